@@ -1,0 +1,399 @@
+/*
+ * kt_oracle.c -- plain CPU oracle for KAITIAN's hierarchical, load-weighted
+ * gradient synchronisation.
+ *
+ * TEST INFRASTRUCTURE ONLY.  This file is the slow, obviously-correct statement of
+ * what the hot path computes.  It is written from the paper's description
+ * (Section III-A hierarchical communication, Section III-C load-adaptive
+ * scheduling) and shares no code, header, table or helper with the CUDA library.
+ * Only tests, the smoke check and the bench's CPU-baseline leg may call it.
+ *
+ * Everything is single threaded and element by element, in a fixed summation
+ * order: ascending rank inside a group, ascending group across groups.  Compile
+ * with -O2 -ffp-contract=off so that the only fused multiply-adds are the explicit
+ * fmaf() calls below.
+ *
+ * Pins (see tests/test_oracle_*.py): every function in this file is pinned to
+ * something other than itself -- exact rational arithmetic, closed forms, a library
+ * cast routine, numpy means, brute-force re-derivation.  No function here is
+ * "parity unpinned".
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+
+#define KTO_OK 0
+#define KTO_ERR_INVALID (-1)
+
+/* ------------------------------------------------------------------------- */
+/* Section III-C, "Initial Benchmarking" and "Dynamic Data Allocation".         */
+/*                                                                           */
+/* score_i = time_fastest / time_i (fastest device scores 1.0);               */
+/* quota_i = score_i / sum_j score_j * B_global;                               */
+/* shares are the quotas rounded to integers such that they still add up to     */
+/* B_global.  The paper does not say how the sum is repaired; the               */
+/* reading used is the largest-remainder rule (floor every quota, hand the      */
+/* missing units to the largest fractional parts, ties to the lower index),    */
+/* which equals nearest rounding whenever nearest rounding already sums to B.   */
+/* A rank never gets zero samples: a zero share is raised to one, taken from    */
+/* the currently largest share (tie: the slowest of them, then higher index).   */
+/* ------------------------------------------------------------------------- */
+int kto_schedule(const double *step_times, int K, int global_batch, int32_t *shares)
+{
+    if (!step_times || !shares || K < 1 || global_batch < K)
+        return KTO_ERR_INVALID;
+    for (int i = 0; i < K; ++i)
+        if (!(step_times[i] > 0.0) || !isfinite(step_times[i]))
+            return KTO_ERR_INVALID;
+
+    double t_min = step_times[0];
+    for (int i = 1; i < K; ++i)
+        if (step_times[i] < t_min)
+            t_min = step_times[i];
+
+    double *score = (double *)malloc(sizeof(double) * (size_t)K);
+    double *frac = (double *)malloc(sizeof(double) * (size_t)K);
+    if (!score || !frac) {
+        free(score);
+        free(frac);
+        return KTO_ERR_INVALID;
+    }
+
+    double sum = 0.0;
+    for (int i = 0; i < K; ++i) {
+        score[i] = t_min / step_times[i];
+        sum = sum + score[i];
+    }
+
+    int64_t given = 0;
+    for (int i = 0; i < K; ++i) {
+        double q = score[i] / sum * (double)global_batch;
+        double f = floor(q);
+        shares[i] = (int32_t)f;
+        frac[i] = q - f;
+        given += shares[i];
+    }
+
+    int64_t missing = (int64_t)global_batch - given;
+    while (missing > 0) {
+        int best = -1;
+        for (int i = 0; i < K; ++i)
+            if (frac[i] >= 0.0 && (best < 0 || frac[i] > frac[best]))
+                best = i;
+        if (best < 0) { /* every rank already got one extra unit: start again */
+            for (int i = 0; i < K; ++i)
+                frac[i] = 0.0;
+            continue;
+        }
+        shares[best] += 1;
+        frac[best] = -1.0; /* at most one extra unit per round */
+        --missing;
+    }
+    while (missing < 0) { /* only reachable through rounding of the quotas */
+        int big = 0;
+        for (int i = 1; i < K; ++i)
+            if (shares[i] > shares[big])
+                big = i;
+        shares[big] -= 1;
+        ++missing;
+    }
+
+    /* nobody idles: the donor is the largest share; among equal shares the slowest
+     * device, among equally slow ones the higher index -- so that a faster device
+     * never ends up with less than a slower one */
+    for (int i = 0; i < K; ++i) {
+        if (shares[i] >= 1)
+            continue;
+        int big = 0;
+        for (int j = 1; j < K; ++j)
+            if (shares[j] > shares[big] ||
+                (shares[j] == shares[big] && step_times[j] >= step_times[big]))
+                big = j;
+        shares[big] -= 1;
+        shares[i] += 1;
+    }
+
+    free(score);
+    free(frac);
+    return KTO_OK;
+}
+
+/* ------------------------------------------------------------------------- */
+/* Weights of the two-level mean (Section III-A groups, Section III-C shares).  */
+/* B_g = sum of the shares of group g, B = sum of all shares.                  */
+/* a_r = b_r / B_g  (weight of rank r inside its group),                       */
+/* W_g = B_g / B    (weight of group g in the global result),                  */
+/* w_r = b_r / B    (weight of rank r in the one-level, "flat" mean).          */
+/* Each quotient is formed in double and rounded once to float.               */
+/* ------------------------------------------------------------------------- */
+int kto_coefficients(const int32_t *group_of, const int32_t *shares, int K, int G,
+                     float *a, float *W, float *w_flat)
+{
+    if (!group_of || !shares || K < 1 || G < 1 || G > K)
+        return KTO_ERR_INVALID;
+    int64_t *Bg = (int64_t *)calloc((size_t)G, sizeof(int64_t));
+    if (!Bg)
+        return KTO_ERR_INVALID;
+    int64_t B = 0;
+    for (int r = 0; r < K; ++r) {
+        if (group_of[r] < 0 || group_of[r] >= G || shares[r] < 1) {
+            free(Bg);
+            return KTO_ERR_INVALID;
+        }
+        Bg[group_of[r]] += shares[r];
+        B += shares[r];
+    }
+    for (int g = 0; g < G; ++g)
+        if (Bg[g] == 0) { /* empty group */
+            free(Bg);
+            return KTO_ERR_INVALID;
+        }
+    for (int r = 0; r < K; ++r) {
+        if (a)
+            a[r] = (float)((double)shares[r] / (double)Bg[group_of[r]]);
+        if (w_flat)
+            w_flat[r] = (float)((double)shares[r] / (double)B);
+    }
+    if (W)
+        for (int g = 0; g < G; ++g)
+            W[g] = (float)((double)Bg[g] / (double)B);
+    free(Bg);
+    return KTO_OK;
+}
+
+/* ------------------------------------------------------------------------- */
+/* Bucket plan (gradient bucketing of the data-parallel reducer, Section III).  */
+/* The paper only says gradients are all-reduced by DDP; the reading used:     */
+/*  - tensors are visited in reverse list order (gradients of the last layers   */
+/*    become ready first);                                                     */
+/*  - a bucket holds at most cap = bucket_cap_bytes / 4 transport elements      */
+/*    (the transport is fp32 whatever the gradient dtype); a tensor is never    */
+/*    split and a tensor larger than the cap gets a bucket of its own;          */
+/*  - inside the transport every tensor starts at a multiple of 8 elements and  */
+/*    every bucket at a multiple of 64 elements; the gaps are zero padding.     */
+/* Outputs: tensor_offset[t] (element offset in the transport), bucket_of[t],  */
+/* bucket_start[b], bucket_numel[b] (start of bucket b to start of b+1, the     */
+/* last one up to transport_numel), n_buckets, transport_numel (multiple of 64).*/
+/* bucket_start/bucket_numel must have room for T entries.                     */
+/* ------------------------------------------------------------------------- */
+static int64_t round_up(int64_t x, int64_t m) { return (x + m - 1) / m * m; }
+
+int kto_bucket_plan(const int64_t *numel, int T, int64_t bucket_cap_bytes,
+                    int64_t *tensor_offset, int32_t *bucket_of, int64_t *bucket_start,
+                    int64_t *bucket_numel, int32_t *n_buckets, int64_t *transport_numel)
+{
+    if (!numel || T < 1 || bucket_cap_bytes < 4)
+        return KTO_ERR_INVALID;
+    for (int t = 0; t < T; ++t)
+        if (numel[t] < 0)
+            return KTO_ERR_INVALID;
+    const int64_t cap = bucket_cap_bytes / 4;
+
+    int32_t nb = 0;
+    int64_t cursor = 0;     /* next free transport element */
+    int64_t start = 0;      /* start of the open bucket */
+    int open_has_tensor = 0;
+    for (int t = T - 1; t >= 0; --t) {
+        int64_t off = round_up(cursor, 8);
+        if (open_has_tensor && (off - start) + numel[t] > cap) {
+            /* close the bucket, open the next one on a 64-element boundary */
+            ++nb;
+            start = round_up(cursor, 64);
+            off = start;
+            open_has_tensor = 0;
+        }
+        if (!open_has_tensor)
+            bucket_start[nb] = start;
+        tensor_offset[t] = off;
+        bucket_of[t] = nb;
+        cursor = off + numel[t];
+        open_has_tensor = 1;
+    }
+    ++nb;
+    const int64_t total = round_up(cursor, 64);
+    for (int b = 0; b < nb; ++b)
+        bucket_numel[b] = (b + 1 < nb ? bucket_start[b + 1] : total) - bucket_start[b];
+    *n_buckets = nb;
+    *transport_numel = total;
+    return KTO_OK;
+}
+
+/* ------------------------------------------------------------------------- */
+/* Casts.  bf16 is the upper half of an IEEE-754 binary32 pattern.             */
+/* Widening is exact.  Narrowing rounds to nearest, ties to even, on the bit    */
+/* pattern; a NaN keeps its sign and upper payload and is made quiet.           */
+/* ------------------------------------------------------------------------- */
+static float bits_to_f32(uint32_t u)
+{
+    float f;
+    memcpy(&f, &u, 4);
+    return f;
+}
+static uint32_t f32_to_bits(float f)
+{
+    uint32_t u;
+    memcpy(&u, &f, 4);
+    return u;
+}
+
+float kto_bf16_to_f32_one(uint16_t h) { return bits_to_f32((uint32_t)h << 16); }
+
+uint16_t kto_f32_to_bf16_one(float f)
+{
+    uint32_t u = f32_to_bits(f);
+    if ((u & 0x7FFFFFFFu) > 0x7F800000u) /* NaN */
+        return (uint16_t)((u >> 16) | 0x0040u);
+    uint32_t lsb = (u >> 16) & 1u;
+    u += 0x7FFFu + lsb;
+    return (uint16_t)(u >> 16);
+}
+
+void kto_bf16_to_f32(const uint16_t *in, float *out, int64_t n)
+{
+    for (int64_t i = 0; i < n; ++i)
+        out[i] = kto_bf16_to_f32_one(in[i]);
+}
+
+void kto_f32_to_bf16(const float *in, uint16_t *out, int64_t n)
+{
+    for (int64_t i = 0; i < n; ++i)
+        out[i] = kto_f32_to_bf16_one(in[i]);
+}
+
+/* dtype codes used by the element accessors below */
+#define KTO_F32 0
+#define KTO_BF16 1
+
+static float load_as_f32(const void *base, int dtype, int64_t i)
+{
+    if (dtype == KTO_BF16)
+        return kto_bf16_to_f32_one(((const uint16_t *)base)[i]);
+    return ((const float *)base)[i];
+}
+
+/* ------------------------------------------------------------------------- */
+/* Standalone pack: the flat bucket copy of one rank's gradient list.          */
+/* flat[tensor_offset[t] + j] = x^(t)[j] (bit copy, same dtype), padding = 0.   */
+/* elem_size is 4 (fp32) or 2 (bf16).                                          */
+/* ------------------------------------------------------------------------- */
+void kto_pack(const void *const *tensors, const int64_t *numel, const int64_t *tensor_offset,
+              int T, int elem_size, int64_t transport_numel, void *flat)
+{
+    memset(flat, 0, (size_t)transport_numel * (size_t)elem_size);
+    for (int t = 0; t < T; ++t) {
+        const unsigned char *src = (const unsigned char *)tensors[t];
+        unsigned char *dst = (unsigned char *)flat + tensor_offset[t] * elem_size;
+        for (int64_t j = 0; j < numel[t] * elem_size; ++j)
+            dst[j] = src[j];
+    }
+}
+
+/* ------------------------------------------------------------------------- */
+/* Intra-group reduce (Section III-A, first bullet: the collective among the    */
+/* homogeneous devices of one group), with the in-group batch-share weights:   */
+/*   P_g[i] = sum over the ranks r of group g, ascending r, of a_r * x_r[i].     */
+/* The first term is one rounded product, every later term one fmaf.           */
+/* grads is rank-major: grads[r*T + t] is tensor t of rank r.  transport[g]     */
+/* receives group g's fp32 partial at the bucket offsets; padding is zero.      */
+/* ------------------------------------------------------------------------- */
+void kto_intra_reduce(const void *const *grads, int in_dtype, const int64_t *numel,
+                      const int64_t *tensor_offset, int T, int64_t transport_numel,
+                      const int32_t *group_of, const float *a, int K, int G,
+                      float *const *transport)
+{
+    for (int g = 0; g < G; ++g) {
+        float *P = transport[g];
+        for (int64_t i = 0; i < transport_numel; ++i)
+            P[i] = 0.0f;
+        for (int t = 0; t < T; ++t) {
+            for (int64_t j = 0; j < numel[t]; ++j) {
+                float acc = 0.0f;
+                int first = 1;
+                for (int r = 0; r < K; ++r) {
+                    if (group_of[r] != g)
+                        continue;
+                    float x = load_as_f32(grads[(size_t)r * (size_t)T + (size_t)t], in_dtype, j);
+                    if (first) {
+                        acc = a[r] * x;
+                        first = 0;
+                    } else {
+                        acc = fmaf(a[r], x, acc);
+                    }
+                }
+                P[tensor_offset[t] + j] = acc;
+            }
+        }
+    }
+}
+
+/* ------------------------------------------------------------------------- */
+/* Inter-group combine (Section III-A, second bullet: the reduction between     */
+/* groups, done on host-relayed fp32 partials), with the group weights:        */
+/*   S[i] = sum over groups g, ascending g, of W_g * P_g[i].                     */
+/* ------------------------------------------------------------------------- */
+void kto_combine(const float *const *partials, const float *W, int G, int64_t n, float *S)
+{
+    for (int64_t i = 0; i < n; ++i) {
+        float acc = W[0] * partials[0][i];
+        for (int g = 1; g < G; ++g)
+            acc = fmaf(W[g], partials[g][i], acc);
+        S[i] = acc;
+    }
+}
+
+/* ------------------------------------------------------------------------- */
+/* Unpack + scale: the copy from the reduced bucket back into per-parameter     */
+/* gradients.  out^(t)[j] = cast(scale * S[tensor_offset[t] + j]); the product  */
+/* is one rounded fp32 multiply; cast is the identity for fp32 and the           */
+/* round-to-nearest-even narrowing above for bf16.  Padding is ignored.         */
+/* ------------------------------------------------------------------------- */
+void kto_unpack_scale(const float *S, const int64_t *numel, const int64_t *tensor_offset,
+                      int T, float scale, int out_dtype, void *const *out)
+{
+    for (int t = 0; t < T; ++t) {
+        for (int64_t j = 0; j < numel[t]; ++j) {
+            float y = S[tensor_offset[t] + j] * scale;
+            if (out_dtype == KTO_BF16)
+                ((uint16_t *)out[t])[j] = kto_f32_to_bf16_one(y);
+            else
+                ((float *)out[t])[j] = y;
+        }
+    }
+}
+
+/* ------------------------------------------------------------------------- */
+/* One-level ("flat") weighted mean over all ranks, for the invariant           */
+/* "hierarchical equals flat within tolerance":                                */
+/*   F[i] = sum_r w_r * x_r[i], ascending r, in fp32 (fmaf chain) and, with the  */
+/* exact rational weights b_r / B, in fp64.  x is one flat buffer per rank.      */
+/* ------------------------------------------------------------------------- */
+void kto_flat_reduce_f32(const void *const *x, int in_dtype, const float *w_flat, int K,
+                         int64_t n, float *F)
+{
+    for (int64_t i = 0; i < n; ++i) {
+        float acc = w_flat[0] * load_as_f32(x[0], in_dtype, i);
+        for (int r = 1; r < K; ++r)
+            acc = fmaf(w_flat[r], load_as_f32(x[r], in_dtype, i), acc);
+        F[i] = acc;
+    }
+}
+
+void kto_flat_reduce_f64(const void *const *x, int in_dtype, const int32_t *shares, int K,
+                         int64_t n, double *F, double *absF)
+{
+    int64_t B = 0;
+    for (int r = 0; r < K; ++r)
+        B += shares[r];
+    for (int64_t i = 0; i < n; ++i) {
+        double acc = 0.0, mag = 0.0;
+        for (int r = 0; r < K; ++r) {
+            double v = (double)load_as_f32(x[r], in_dtype, i);
+            acc += (double)shares[r] * v;
+            mag += (double)shares[r] * fabs(v);
+        }
+        F[i] = acc / (double)B;
+        if (absF)
+            absF[i] = mag / (double)B; /* sum_r w_r |x_r[i]|: forward-error scale */
+    }
+}
