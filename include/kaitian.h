@@ -1,0 +1,194 @@
+/*
+ * kaitian.h -- C ABI of the B200 library for KAITIAN's hierarchical, load-weighted
+ * gradient synchronisation (the data-parallel hot path of a heterogeneous training
+ * step; paper Sections III-A and III-C).
+ *
+ * K simulated ranks, split into G vendor groups, keep their per-parameter gradient
+ * tensors in one GPU's memory.  One synchronisation step is
+ *
+ *   kt_schedule      step times -> integer batch shares            (Section III-C)
+ *   kt_groups_init   rank->group map + shares -> weights            (Sections III-A, III-C)
+ *   kt_bucket_pack   describe the gradient tensors, build buckets   (DDP bucketing, Section III)
+ *   kt_hier_reduce   INTRA: P_g = sum_{r in g} a_r x_r  (fp32 transport, one per group)
+ *   kt_stage_to_host relay of the partials through pinned host RAM  (Section III-A, steps 1-3)
+ *   kt_hier_reduce   INTER: S = sum_g W_g P_g
+ *   kt_unpack_scale  per-parameter gradients = cast(scale * S)
+ *
+ * Conventions
+ *  - Every pointer argument says "host" or "device".  "host array of device pointers"
+ *    means the array itself is read on the host during the call and may be freed after
+ *    it returns; the pointers in it address device memory owned by the caller.
+ *  - The library owns only the kt_ctx and its small device tables (pointer tables, tensor
+ *    table).  Gradient tensors, transport buffers, pinned buffers and streams belong to
+ *    the caller.  `stream` arguments are cudaStream_t values passed as void* (NULL = the
+ *    legacy default stream).
+ *  - All functions return KT_OK (0) or a negative kt_status.  Arguments are validated on
+ *    the host before anything is launched; nothing traps on the device and nothing
+ *    throws across the boundary.  kt_last_error() returns a message for the last failing
+ *    call made by the calling thread.
+ *  - Kernel launches and copies are asynchronous with respect to the given stream.
+ *    kt_schedule, kt_groups_init, kt_set_shares, kt_plan_query are pure host functions.
+ *  - Arithmetic is IEEE fp32 with a fixed order (ascending rank inside a group, ascending
+ *    group): the first term of a sum is one rounded product, every later term one fused
+ *    multiply-add.  bf16 gradients are widened exactly; bf16 outputs are rounded to
+ *    nearest-even.
+ */
+#ifndef KAITIAN_H
+#define KAITIAN_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct kt_ctx kt_ctx;
+
+typedef enum { KT_F32 = 0, KT_BF16 = 1 } kt_dtype;
+
+typedef enum {
+    KT_OK = 0,
+    KT_ERR_INVALID = -1, /* bad argument value (null pointer, range, non-finite time ...) */
+    KT_ERR_SHAPE = -2,   /* sizes inconsistent with the plan (T, R, bucket index ...) */
+    KT_ERR_ALIGN = -3,   /* a transport / flat / combined buffer is not 16-byte aligned */
+    KT_ERR_CUDA = -4,    /* a CUDA runtime call or launch failed; message has the CUDA text */
+    KT_ERR_TIMEOUT = -5, /* kt_stage_wait: the copy had not finished at the deadline */
+    KT_ERR_STATE = -6,   /* call order: e.g. kt_hier_reduce before kt_bucket_pack */
+    KT_ERR_NOMEM = -7    /* host or device allocation of a table failed */
+} kt_status;
+
+typedef enum { KT_INTRA = 1, KT_INTER = 2, KT_BOTH = 3 } kt_phase;
+typedef enum { KT_D2H = 0, KT_H2D = 1 } kt_stage_dir;
+
+#define KT_MAX_RANKS 64
+#define KT_MAX_GROUPS 16
+
+/* Section III-C (initial benchmarking + dynamic data allocation).
+ * step_times[K] (host): measured per-rank step times, each finite and > 0.
+ * shares_out[K] (host): integer batch shares, sum == global_batch, each >= 1.
+ * score_i = t_min / t_i; quota_i = score_i / sum(score) * global_batch; quotas are floored
+ * and the missing units go to the largest fractional parts (tie: lower rank).  A zero
+ * share is raised to one at the expense of the largest share (tie: the slowest of them,
+ * then the higher rank).  Requires 1 <= K <= KT_MAX_RANKS and global_batch >= K.
+ * Errors: KT_ERR_INVALID. */
+int kt_schedule(const double *step_times, int K, int global_batch, int32_t *shares_out);
+
+/* Sections III-A (groups of homogeneous devices) and III-C (shares).
+ * group_of[K] (host): group index of every rank, each in [0, G), no group empty.
+ * shares[K] (host): batch shares, each >= 1.
+ * Computes a_r = b_r / B_g and W_g = B_g / B (double quotient, rounded once to float).
+ * *out receives a new context bound to the current CUDA device; free with kt_destroy.
+ * Errors: KT_ERR_INVALID, KT_ERR_NOMEM, KT_ERR_CUDA. */
+int kt_groups_init(const int32_t *group_of, const int32_t *shares, int K, int G, kt_ctx **out);
+
+/* New shares for the same groups (e.g. after re-running kt_schedule); the bucket plan is
+ * kept.  Takes effect for launches made after the call returns. */
+int kt_set_shares(kt_ctx *ctx, const int32_t *shares);
+
+/* Replace the weights directly: a[K], W[G] (host).  Lets a caller use plain sums across
+ * the hierarchy (a_r = b_r, W_g = 1) with a final scale of 1/B in kt_unpack_scale. */
+int kt_set_coefficients(kt_ctx *ctx, const float *a, const float *W);
+
+/* Read back the weights in use: a_out[K], W_out[G] (host, either may be NULL). */
+int kt_get_coefficients(const kt_ctx *ctx, float *a_out, float *W_out);
+
+/* Gradient bucketing of the data-parallel reducer (Section III: gradients are
+ * all-reduced bucket by bucket; the paper leaves order and size open).
+ * grads: host array of K*T device pointers, rank-major (grads[r*T + t] = tensor t of
+ *        rank r), element type in_dtype, numel[t] elements each (host array, >= 0).
+ *        Pointers need only element alignment; 16-byte aligned tensors take the
+ *        vectorised path.  The pointers are remembered: kt_hier_reduce(KT_INTRA) reads
+ *        the tensors in place, so they must stay valid until re-registered.
+ * Plan: tensors are laid into the fp32 transport in reverse list order; a bucket holds at
+ *        most bucket_cap_bytes / 4 elements (a larger tensor gets a bucket of its own,
+ *        tensors are never split); every tensor starts at a multiple of 8 elements, every
+ *        bucket at a multiple of 64; the gaps are zero padding.
+ * flat_out: NULL, or host array of K device pointers to buffers of transport_numel
+ *        elements of in_dtype, 16-byte aligned: the standalone pack kernel then copies
+ *        every rank's tensors into its flat buffer at the plan's offsets (bit copy,
+ *        padding zero) on `stream`.
+ * Calling it again replaces plan and pointers.  Allocates the device tables (the only
+ * call besides kt_unpack_scale that may allocate).
+ * Errors: KT_ERR_INVALID, KT_ERR_ALIGN, KT_ERR_NOMEM, KT_ERR_CUDA. */
+int kt_bucket_pack(kt_ctx *ctx, const void *const *grads, const int64_t *numel, int T,
+                   int in_dtype, int64_t bucket_cap_bytes, void *const *flat_out, void *stream);
+
+/* The bucket plan alone, as a pure host function (same rules as kt_bucket_pack; no context,
+ * no device): lets a caller size transport buffers before any tensor exists.  Outputs as in
+ * kt_plan_query.  Errors: KT_ERR_INVALID. */
+int kt_plan_buckets(const int64_t *numel, int T, int64_t bucket_cap_bytes, int32_t *n_buckets,
+                    int64_t *bucket_start, int64_t *bucket_numel, int64_t *tensor_offset,
+                    int32_t *bucket_of, int64_t *transport_numel);
+
+/* Plan read-back (all outputs host, each may be NULL).  bucket_start / bucket_numel need
+ * room for n_buckets entries (at most T), tensor_offset for T; offsets and sizes are in
+ * transport elements.  Errors: KT_ERR_STATE before kt_bucket_pack. */
+int kt_plan_query(const kt_ctx *ctx, int32_t *n_buckets, int64_t *bucket_start,
+                  int64_t *bucket_numel, int64_t *tensor_offset, int32_t *bucket_of,
+                  int64_t *transport_numel);
+
+/* The two reductions of Section III-A.
+ * transport: host array of G device pointers, fp32, transport_numel elements each,
+ *        16-byte aligned.
+ * phase KT_INTRA: the fused pack + widen + weighted intra-group reduce.  Reads every
+ *        registered gradient element once and writes P_g = sum_{r in g} a_r x_r at the
+ *        plan's offsets of transport[g], zero in the padding.
+ * phase KT_INTER: combined[i] = sum_g W_g transport[g][i] over the bucket's range
+ *        (combined: device fp32, transport_numel elements, 16-byte aligned).
+ * phase KT_BOTH: KT_INTRA then KT_INTER on the same stream.
+ * bucket: -1 for all buckets, else one bucket index; only that bucket's range of the
+ *        buffers is read or written.
+ * Errors: KT_ERR_STATE, KT_ERR_SHAPE, KT_ERR_INVALID, KT_ERR_ALIGN, KT_ERR_CUDA. */
+int kt_hier_reduce(kt_ctx *ctx, int phase, int bucket, float *const *transport, float *combined,
+                   void *stream);
+
+/* Host relay of Section III-A (device -> host RAM -> [exchange] -> device).
+ * dir KT_D2H: side_stream waits for the work queued so far on main_stream, then copies the
+ *        bucket's range of every transport[g] (device) to host_pinned[g] (host, pinned,
+ *        same element offsets).
+ * dir KT_H2D: side_stream waits for main_stream and for the last KT_D2H of the same
+ *        bucket, then copies host_pinned[g] back into transport[g] (typically a second,
+ *        "receive" set of device buffers).
+ * Both record a completion event that kt_stage_wait consumes.  transport / host_pinned:
+ * host arrays of G pointers.  bucket as in kt_hier_reduce.
+ * Errors: KT_ERR_STATE, KT_ERR_SHAPE, KT_ERR_INVALID, KT_ERR_CUDA. */
+int kt_stage_to_host(kt_ctx *ctx, int dir, int bucket, float *const *transport,
+                     float *const *host_pinned, void *main_stream, void *side_stream);
+
+/* Makes main_stream wait for the last kt_stage_to_host(dir, bucket).  timeout_ms < 0:
+ * returns at once (stream-side wait only).  timeout_ms >= 0: additionally polls the
+ * event on the host until it completes or the deadline passes (KT_ERR_TIMEOUT; the copy
+ * itself is left running).  KT_ERR_STATE if no such copy was queued. */
+int kt_stage_wait(kt_ctx *ctx, int dir, int bucket, void *main_stream, int timeout_ms);
+
+/* Copy-out of the reducer: per-parameter gradients from the reduced bucket.
+ * src: host array of device pointers; from_combined != 0: src[0] is a combined buffer
+ *        (S); from_combined == 0: src[0..G-1] are the group partials and the inter-group
+ *        combine S = sum_g W_g P_g is fused into this kernel (no combined buffer).
+ * out_grads: host array of R*T device pointers (copy-major: out_grads[c*T + t]),
+ *        R = 1, or up to K to hand every rank its own copy; element type out_dtype;
+ *        numel as registered.  16-byte aligned tensors take the vectorised path.
+ * out[t][j] = cast(scale * S[tensor_offset[t] + j]); one rounded multiply; padding ignored.
+ * Errors: KT_ERR_STATE, KT_ERR_SHAPE, KT_ERR_INVALID, KT_ERR_ALIGN, KT_ERR_NOMEM, KT_ERR_CUDA. */
+int kt_unpack_scale(kt_ctx *ctx, const float *const *src, int from_combined,
+                    void *const *out_grads, int R, int out_dtype, float scale, int bucket,
+                    void *stream);
+
+/* Standalone cast kernel: n elements from `in` (device, in_dtype) to `out` (device,
+ * out_dtype); bf16 -> fp32 exact, fp32 -> bf16 round-to-nearest-even, same type = copy.
+ * Errors: KT_ERR_INVALID, KT_ERR_CUDA. */
+int kt_cast(const void *in, int in_dtype, void *out, int out_dtype, int64_t n, void *stream);
+
+/* Number of kernels this context has launched so far (for launch accounting). */
+int64_t kt_launch_count(const kt_ctx *ctx);
+
+/* Message of the last failing call of this thread ("" if none).  ctx may be NULL. */
+const char *kt_last_error(const kt_ctx *ctx);
+
+/* Frees the context, its device tables and events.  NULL is allowed. */
+void kt_destroy(kt_ctx *ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* KAITIAN_H */

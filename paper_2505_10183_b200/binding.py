@@ -1,0 +1,295 @@
+"""Thin ctypes binding over the C-ABI library declared in ``include/kaitian.h``.
+
+Argument marshalling only: every function here has the name of the C entry point it
+calls, turns torch tensors into raw pointers and raises :class:`KtError` on a negative
+status.  All arithmetic runs in the CUDA library.  If the library has not been built the
+import fails: there is no CPU fallback.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from dataclasses import dataclass
+from typing import List, Optional, Sequence, Union
+
+import torch
+
+from . import build as _build
+
+KT_F32, KT_BF16 = 0, 1
+KT_INTRA, KT_INTER, KT_BOTH = 1, 2, 3
+KT_D2H, KT_H2D = 0, 1
+KT_OK, KT_ERR_INVALID, KT_ERR_SHAPE, KT_ERR_ALIGN = 0, -1, -2, -3
+KT_ERR_CUDA, KT_ERR_TIMEOUT, KT_ERR_STATE, KT_ERR_NOMEM = -4, -5, -6, -7
+KT_MAX_RANKS, KT_MAX_GROUPS = 64, 16
+
+EXPORTS = ["kt_schedule", "kt_groups_init", "kt_set_shares", "kt_set_coefficients",
+           "kt_get_coefficients", "kt_bucket_pack", "kt_plan_buckets", "kt_plan_query", "kt_hier_reduce",
+           "kt_stage_to_host", "kt_stage_wait", "kt_unpack_scale", "kt_cast", "kt_launch_count",
+           "kt_last_error", "kt_destroy"]
+
+_DTYPES = {torch.float32: KT_F32, torch.bfloat16: KT_BF16}
+
+
+class KtError(RuntimeError):
+    def __init__(self, status: int, message: str):
+        super().__init__("kaitian status %d: %s" % (status, message))
+        self.status = status
+
+
+def _load() -> C.CDLL:
+    path = _build.LIB
+    if not os.path.exists(path):
+        raise ImportError(
+            "%s is missing: build it with `python -m paper_2505_10183_b200.build` "
+            "(needs nvcc); this package has no CPU fallback" % path)
+    L = C.CDLL(path)
+    vp, i32p, i64p, f32p = C.c_void_p, C.POINTER(C.c_int32), C.POINTER(C.c_int64), C.POINTER(C.c_float)
+    vpp = C.POINTER(C.c_void_p)
+    sigs = {
+        "kt_schedule": ([C.POINTER(C.c_double), C.c_int, C.c_int, i32p], C.c_int),
+        "kt_groups_init": ([i32p, i32p, C.c_int, C.c_int, vpp], C.c_int),
+        "kt_set_shares": ([vp, i32p], C.c_int),
+        "kt_set_coefficients": ([vp, f32p, f32p], C.c_int),
+        "kt_get_coefficients": ([vp, f32p, f32p], C.c_int),
+        "kt_bucket_pack": ([vp, vpp, i64p, C.c_int, C.c_int, C.c_int64, vpp, vp], C.c_int),
+        "kt_plan_buckets": ([i64p, C.c_int, C.c_int64, i32p, i64p, i64p, i64p, i32p, i64p], C.c_int),
+        "kt_plan_query": ([vp, i32p, i64p, i64p, i64p, i32p, i64p], C.c_int),
+        "kt_hier_reduce": ([vp, C.c_int, C.c_int, vpp, vp, vp], C.c_int),
+        "kt_stage_to_host": ([vp, C.c_int, C.c_int, vpp, vpp, vp, vp], C.c_int),
+        "kt_stage_wait": ([vp, C.c_int, C.c_int, vp, C.c_int], C.c_int),
+        "kt_unpack_scale": ([vp, vpp, C.c_int, vpp, C.c_int, C.c_int, C.c_float, C.c_int, vp], C.c_int),
+        "kt_cast": ([vp, C.c_int, vp, C.c_int, C.c_int64, vp], C.c_int),
+        "kt_launch_count": ([vp], C.c_int64),
+        "kt_last_error": ([vp], C.c_char_p),
+        "kt_destroy": ([vp], None),
+    }
+    for name, (args, res) in sigs.items():
+        fn = getattr(L, name)
+        fn.argtypes = args
+        fn.restype = res
+    return L
+
+
+_lib = _load()
+
+
+def _check(rc: int) -> None:
+    if rc != 0:
+        raise KtError(rc, _lib.kt_last_error(None).decode("utf-8", "replace"))
+
+
+class PtrArray:
+    """A host array of raw pointers built once from tensors (keeps them alive)."""
+
+    def __init__(self, tensors: Sequence[torch.Tensor]):
+        self.tensors = list(tensors)
+        self.n = len(self.tensors)
+        self.array = (C.c_void_p * max(self.n, 1))()
+        for i, t in enumerate(self.tensors):
+            self.array[i] = t.data_ptr() if t.numel() > 0 else (t.data_ptr() or None)
+
+
+Ptrs = Union[PtrArray, Sequence[torch.Tensor]]
+
+
+def kt_ptrs(tensors: Ptrs) -> PtrArray:
+    return tensors if isinstance(tensors, PtrArray) else PtrArray(tensors)
+
+
+def _stream(stream) -> C.c_void_p:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return C.c_void_p(stream.cuda_stream if hasattr(stream, "cuda_stream") else int(stream))
+
+
+def _i32(values) -> C.Array:
+    return (C.c_int32 * len(values))(*[int(v) for v in values])
+
+
+@dataclass
+class Plan:
+    n_buckets: int
+    bucket_start: List[int]
+    bucket_numel: List[int]
+    tensor_offset: List[int]
+    bucket_of: List[int]
+    transport_numel: int
+
+
+class Ctx:
+    """Opaque handle returned by :func:`kt_groups_init`."""
+
+    def __init__(self, handle: int, K: int, G: int):
+        self.handle = C.c_void_p(handle)
+        self.K, self.G, self.T = K, G, 0
+        self._keep = {}
+
+    def __del__(self):
+        try:
+            kt_destroy(self)
+        except Exception:
+            pass
+
+
+# --------------------------------------------------------------------------- entry points
+def kt_schedule(step_times: Sequence[float], global_batch: int) -> List[int]:
+    K = len(step_times)
+    t = (C.c_double * max(K, 1))(*[float(x) for x in step_times])
+    out = (C.c_int32 * max(K, 1))()
+    _check(_lib.kt_schedule(t, K, int(global_batch), out))
+    return [int(out[i]) for i in range(K)]
+
+
+def kt_groups_init(group_of: Sequence[int], shares: Sequence[int], G: Optional[int] = None) -> Ctx:
+    K = len(group_of)
+    if len(shares) != K:
+        raise KtError(KT_ERR_SHAPE, "group_of and shares differ in length")
+    G = (max(group_of) + 1 if K else 0) if G is None else G
+    h = C.c_void_p()
+    _check(_lib.kt_groups_init(_i32(group_of), _i32(shares), K, int(G), C.byref(h)))
+    return Ctx(h.value, K, int(G))
+
+
+def kt_set_shares(ctx: Ctx, shares: Sequence[int]) -> None:
+    if len(shares) != ctx.K:
+        raise KtError(KT_ERR_SHAPE, "expected %d shares" % ctx.K)
+    _check(_lib.kt_set_shares(ctx.handle, _i32(shares)))
+
+
+def kt_set_coefficients(ctx: Ctx, a: Sequence[float], W: Sequence[float]) -> None:
+    if len(a) != ctx.K or len(W) != ctx.G:
+        raise KtError(KT_ERR_SHAPE, "expected %d rank and %d group weights" % (ctx.K, ctx.G))
+    _check(_lib.kt_set_coefficients(ctx.handle, (C.c_float * ctx.K)(*a), (C.c_float * ctx.G)(*W)))
+
+
+def kt_get_coefficients(ctx: Ctx):
+    a = (C.c_float * ctx.K)()
+    W = (C.c_float * ctx.G)()
+    _check(_lib.kt_get_coefficients(ctx.handle, a, W))
+    return list(a), list(W)
+
+
+def kt_bucket_pack(ctx: Ctx, grads: Sequence[Sequence[torch.Tensor]], bucket_cap_bytes: int,
+                   flat_out: Optional[Ptrs] = None, stream=None) -> None:
+    """grads[r][t]: tensor t of rank r (contiguous, all of one dtype, same shapes per rank)."""
+    if len(grads) != ctx.K:
+        raise KtError(KT_ERR_SHAPE, "expected gradient lists of %d ranks" % ctx.K)
+    T = len(grads[0])
+    flat = []
+    for r in range(ctx.K):
+        if len(grads[r]) != T:
+            raise KtError(KT_ERR_SHAPE, "rank %d holds %d tensors, rank 0 holds %d" % (r, len(grads[r]), T))
+        for t in range(T):
+            g = grads[r][t]
+            if g.dtype != grads[0][0].dtype or g.numel() != grads[0][t].numel() or not g.is_contiguous():
+                raise KtError(KT_ERR_SHAPE, "grads[%d][%d]: dtype, size or layout mismatch" % (r, t))
+            flat.append(g)
+    if T and grads[0][0].dtype not in _DTYPES:
+        raise KtError(KT_ERR_INVALID, "unsupported gradient dtype %s" % grads[0][0].dtype)
+    pa = PtrArray(flat)
+    numel = (C.c_int64 * max(T, 1))(*[int(g.numel()) for g in grads[0]])
+    fo = kt_ptrs(flat_out) if flat_out is not None else None
+    dt = _DTYPES[grads[0][0].dtype] if T else KT_F32
+    _check(_lib.kt_bucket_pack(ctx.handle, pa.array, numel, T, dt, int(bucket_cap_bytes),
+                               fo.array if fo is not None else None, _stream(stream)))
+    ctx.T = T
+    ctx._keep["grads"] = pa
+
+
+def kt_plan_buckets(numel: Sequence[int], bucket_cap_bytes: int) -> Plan:
+    T = len(numel)
+    n = (C.c_int64 * max(T, 1))(*[int(v) for v in numel])
+    nb = C.c_int32()
+    total = C.c_int64()
+    bs = (C.c_int64 * max(T, 1))()
+    bn = (C.c_int64 * max(T, 1))()
+    off = (C.c_int64 * max(T, 1))()
+    bof = (C.c_int32 * max(T, 1))()
+    _check(_lib.kt_plan_buckets(n, T, int(bucket_cap_bytes), C.byref(nb), bs, bn, off, bof, C.byref(total)))
+    return Plan(nb.value, list(bs)[: nb.value], list(bn)[: nb.value], list(off)[:T], list(bof)[:T], total.value)
+
+
+def kt_plan_query(ctx: Ctx) -> Plan:
+    nb = C.c_int32()
+    total = C.c_int64()
+    _check(_lib.kt_plan_query(ctx.handle, C.byref(nb), None, None, None, None, C.byref(total)))
+    bs = (C.c_int64 * nb.value)()
+    bn = (C.c_int64 * nb.value)()
+    off = (C.c_int64 * ctx.T)()
+    bof = (C.c_int32 * ctx.T)()
+    _check(_lib.kt_plan_query(ctx.handle, None, bs, bn, off, bof, None))
+    return Plan(nb.value, list(bs), list(bn), list(off), list(bof), total.value)
+
+
+def kt_hier_reduce(ctx: Ctx, phase: int, transport: Ptrs, combined: Optional[torch.Tensor] = None,
+                   bucket: int = -1, stream=None) -> None:
+    tr = kt_ptrs(transport)
+    if tr.n != ctx.G:
+        raise KtError(KT_ERR_SHAPE, "expected %d transport buffers" % ctx.G)
+    _check(_lib.kt_hier_reduce(ctx.handle, int(phase), int(bucket), tr.array,
+                               C.c_void_p(combined.data_ptr()) if combined is not None else None,
+                               _stream(stream)))
+
+
+def kt_stage_to_host(ctx: Ctx, direction: int, transport: Ptrs, host_pinned: Ptrs, bucket: int = -1,
+                     main_stream=None, side_stream=None) -> None:
+    tr, hp = kt_ptrs(transport), kt_ptrs(host_pinned)
+    if tr.n != ctx.G or hp.n != ctx.G:
+        raise KtError(KT_ERR_SHAPE, "expected %d device and %d host buffers" % (ctx.G, ctx.G))
+    _check(_lib.kt_stage_to_host(ctx.handle, int(direction), int(bucket), tr.array, hp.array,
+                                 _stream(main_stream), _stream(side_stream)))
+
+
+def kt_stage_wait(ctx: Ctx, direction: int, bucket: int = -1, main_stream=None, timeout_ms: int = -1) -> None:
+    _check(_lib.kt_stage_wait(ctx.handle, int(direction), int(bucket), _stream(main_stream), int(timeout_ms)))
+
+
+def kt_unpack_scale(ctx: Ctx, src: Ptrs, out_grads: Union[PtrArray, Sequence[Sequence[torch.Tensor]]],
+                    scale: float = 1.0, from_combined: bool = False, bucket: int = -1,
+                    out_dtype: Optional[int] = None, R: Optional[int] = None, stream=None) -> None:
+    """out_grads[c][t]: copy c of tensor t (or a PtrArray of R*T pointers with R, out_dtype given)."""
+    sp = kt_ptrs(src)
+    if sp.n != (1 if from_combined else ctx.G):
+        raise KtError(KT_ERR_SHAPE, "wrong number of source buffers")
+    if isinstance(out_grads, PtrArray):
+        op = out_grads
+        if R is None or out_dtype is None:
+            raise KtError(KT_ERR_INVALID, "R and out_dtype are required with a PtrArray")
+    else:
+        R = len(out_grads)
+        flat = [t for copy in out_grads for t in copy]
+        if any(len(copy) != ctx.T for copy in out_grads):
+            raise KtError(KT_ERR_SHAPE, "every copy needs %d tensors" % ctx.T)
+        if any(t.dtype != flat[0].dtype or not t.is_contiguous() for t in flat):
+            raise KtError(KT_ERR_SHAPE, "out_grads: dtype or layout mismatch")
+        if flat and flat[0].dtype not in _DTYPES:
+            raise KtError(KT_ERR_INVALID, "unsupported output dtype %s" % flat[0].dtype)
+        out_dtype = _DTYPES[flat[0].dtype] if flat else KT_F32
+        op = PtrArray(flat)
+    if op.n != R * ctx.T:
+        raise KtError(KT_ERR_SHAPE, "expected %d output pointers" % (R * ctx.T))
+    _check(_lib.kt_unpack_scale(ctx.handle, sp.array, 1 if from_combined else 0, op.array, int(R),
+                                int(out_dtype), C.c_float(scale), int(bucket), _stream(stream)))
+    ctx._keep["out"] = op
+
+
+def kt_cast(inp: torch.Tensor, out: torch.Tensor, stream=None) -> None:
+    if inp.numel() != out.numel() or inp.dtype not in _DTYPES or out.dtype not in _DTYPES:
+        raise KtError(KT_ERR_SHAPE, "kt_cast: size or dtype mismatch")
+    _check(_lib.kt_cast(C.c_void_p(inp.data_ptr()), _DTYPES[inp.dtype], C.c_void_p(out.data_ptr()),
+                        _DTYPES[out.dtype], inp.numel(), _stream(stream)))
+
+
+def kt_launch_count(ctx: Ctx) -> int:
+    return int(_lib.kt_launch_count(ctx.handle))
+
+
+def kt_last_error() -> str:
+    return _lib.kt_last_error(None).decode("utf-8", "replace")
+
+
+def kt_destroy(ctx: Ctx) -> None:
+    if ctx.handle is not None and ctx.handle.value:
+        _lib.kt_destroy(ctx.handle)
+        ctx.handle = C.c_void_p(None)

@@ -1,0 +1,1102 @@
+// kaitian.cu -- sm_100a kernels and C ABI for KAITIAN's hierarchical, load-weighted
+// gradient synchronisation (paper Sections III-A and III-C).  See include/kaitian.h for
+// the contract of every entry point.
+//
+// Data layout in device memory
+//   gradients   K*T caller-owned tensors (fp32 or bf16), read in place through a pointer
+//               table [K][T] kept in group-major rank order and transport tensor order
+//   transport   G caller-owned fp32 buffers of transport_numel elements: tensors laid end
+//               to end in reverse list order, each at a multiple of 8 elements, buckets at
+//               multiples of 64, zero padding in the gaps
+//   tensor table  one 32-byte record per tensor (transport offset, numel, numel + padding,
+//               flags) and a prefix sum of TILE-sized work units per tensor
+// Work decomposition: the transport is cut into tiles of TILE elements that never cross a
+// tensor boundary.  A CTA walks tiles in a grid-stride loop, finds the tensor of a tile by
+// binary search in the prefix (shared memory), and streams the K rank buffers of that tile
+// with 128-bit loads.  Interior tiles of 16-byte aligned tensors take a branch-free vector
+// path; ragged tails, padding and misaligned tensors take an element-wise path.
+//
+// Arithmetic order is fixed: first member of a group acc = a*x (one rounded multiply),
+// later members acc = fma(a, x, acc); the same across groups with W_g.
+
+#include "../../include/kaitian.h"
+
+#include <cuda_runtime.h>
+
+#include <chrono>
+#include <cmath>
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <thread>
+#include <utility>
+#include <vector>
+
+namespace {
+
+constexpr int NT = 256;          // threads per CTA
+constexpr int TILE = 2048;       // transport elements per work unit
+constexpr int FLAG_ALIGNED = 1;  // all K sources of the tensor are 16-byte aligned
+
+// ------------------------------------------------------------------ error reporting
+thread_local char g_err[512] = "";
+
+int fail(int code, const char *fmt, ...) {
+    va_list ap;
+    va_start(ap, fmt);
+    vsnprintf(g_err, sizeof(g_err), fmt, ap);
+    va_end(ap);
+    return code;
+}
+
+#define KT_CUDA(call)                                                                       \
+    do {                                                                                    \
+        cudaError_t e_ = (call);                                                            \
+        if (e_ != cudaSuccess)                                                              \
+            return fail(KT_ERR_CUDA, "%s: %s", #call, cudaGetErrorString(e_));              \
+    } while (0)
+
+// ------------------------------------------------------------------ device tables
+struct TInfo {            // one per tensor, transport order
+    long long dst_off;    // element offset in the transport
+    long long numel;      // gradient elements
+    long long ext;        // numel + zero padding up to the next tensor (multiple of 8 apart)
+    int flags;
+    int pad_;
+};
+
+struct RankTab {          // ranks in group-major order (ascending rank inside a group)
+    float coef[KT_MAX_RANKS];
+    signed char gid[KT_MAX_RANKS];
+    unsigned char first[KT_MAX_RANKS];   // first member of its group
+    unsigned char last[KT_MAX_RANKS];    // last member of its group
+    int K;
+};
+
+struct GroupTab {
+    float W[KT_MAX_GROUPS];
+    int G;
+};
+
+struct TilePlan {         // which tiles a launch covers and how to decode them
+    const int *prefix;    // [T+1] tiles before tensor u
+    const TInfo *info;    // [T]
+    int T;
+    int u_lo, u_hi;       // tensors [u_lo, u_hi) take part
+    int tile_lo;          // prefix[u_lo]
+    int n_tiles;          // prefix[u_hi] - prefix[u_lo]
+    int prefix_in_smem;   // stage prefix[u_lo .. u_hi] in shared memory
+};
+
+struct K1Params {
+    TilePlan tp;
+    const void *const *ptrs;           // [K][T] device pointer table
+    float *transport[KT_MAX_GROUPS];
+    RankTab rt;
+};
+
+struct K2Params {
+    TilePlan tp;
+    const float *src[KT_MAX_GROUPS];   // partials (or one combined buffer)
+    GroupTab gt;
+    void *const *out_ptrs;             // [R][T] device pointer table
+    const unsigned char *out_aligned;  // [T] all R destinations 16-byte aligned
+    int R;
+    float scale;
+};
+
+struct PackParams {
+    TilePlan tp;
+    const void *const *ptrs;           // [K][T], group-major rank order
+    void *flat[KT_MAX_RANKS];          // same rank order
+    int K;
+};
+
+// ------------------------------------------------------------------ device helpers
+__device__ __forceinline__ uint4 ld_stream(const void *p) {
+    // read-once data: keep it out of L1
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                 : "l"(p));
+    return v;
+}
+
+template <typename P>
+__device__ __forceinline__ P *ldg_ptr(P *const *slot) {
+    // pointer tables are read-only for the lifetime of a launch
+    return reinterpret_cast<P *>(__ldg(reinterpret_cast<const unsigned long long *>(slot)));
+}
+
+__device__ __forceinline__ unsigned pack_bf16x2(float lo, float hi) {
+    unsigned d;   // round-to-nearest-even narrowing of two floats; hi lands in the upper half
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
+    return d;
+}
+
+template <typename T> struct Elem;
+template <> struct Elem<float> {
+    static constexpr int VEC = 4;
+    __device__ static __forceinline__ float widen(float v) { return v; }
+    __device__ static __forceinline__ void unpack(const uint4 &v, float (&x)[4]) {
+        x[0] = __uint_as_float(v.x); x[1] = __uint_as_float(v.y);
+        x[2] = __uint_as_float(v.z); x[3] = __uint_as_float(v.w);
+    }
+};
+template <> struct Elem<unsigned short> {
+    static constexpr int VEC = 8;
+    __device__ static __forceinline__ float widen(unsigned short v) {
+        return __uint_as_float(static_cast<unsigned>(v) << 16);
+    }
+    __device__ static __forceinline__ void unpack(const uint4 &v, float (&x)[8]) {
+        x[0] = __uint_as_float(v.x << 16); x[1] = __uint_as_float(v.x & 0xFFFF0000u);
+        x[2] = __uint_as_float(v.y << 16); x[3] = __uint_as_float(v.y & 0xFFFF0000u);
+        x[4] = __uint_as_float(v.z << 16); x[5] = __uint_as_float(v.z & 0xFFFF0000u);
+        x[6] = __uint_as_float(v.w << 16); x[7] = __uint_as_float(v.w & 0xFFFF0000u);
+    }
+};
+
+// Stage the tile prefix of the participating tensors in shared memory (or leave it global).
+__device__ __forceinline__ const int *stage_prefix(const TilePlan &tp, int *smem) {
+    if (!tp.prefix_in_smem) return tp.prefix + tp.u_lo;
+    const int n = tp.u_hi - tp.u_lo + 1;
+    for (int i = threadIdx.x; i < n; i += NT) smem[i] = tp.prefix[tp.u_lo + i];
+    __syncthreads();
+    return smem;
+}
+
+// Largest u in [0, n) with pre[u] <= tile (pre is non-decreasing, pre[n] > tile).
+__device__ __forceinline__ int find_tensor(const int *pre, int n, int tile) {
+    int lo = 0, hi = n;
+    while (hi - lo > 1) {
+        const int mid = (lo + hi) >> 1;
+        if (pre[mid] <= tile) lo = mid; else hi = mid;
+    }
+    return lo;
+}
+
+// ------------------------------------------------------------------ K1: fused pack + widen + weighted intra-group reduce
+// P_g[off_u + e] = sum_{r in g} a_r * f32(x_r^(u)[e]), zero in the padding.
+template <typename Tin, int KB>
+__global__ void __launch_bounds__(NT) k1_intra_reduce(const __grid_constant__ K1Params p) {
+    constexpr int VEC = Elem<Tin>::VEC;
+    constexpr int ITERS = TILE / (NT * VEC);
+    extern __shared__ int smem_prefix[];
+    const int *pre = stage_prefix(p.tp, smem_prefix);
+    const int nu = p.tp.u_hi - p.tp.u_lo;
+    const int K = p.rt.K;
+    const int T = p.tp.T;
+
+    for (int tile = blockIdx.x; tile < p.tp.n_tiles; tile += gridDim.x) {
+        const int gt = tile + p.tp.tile_lo;
+        const int ul = find_tensor(pre, nu, gt);
+        const int u = ul + p.tp.u_lo;
+        const TInfo ti = p.tp.info[u];
+        const long long e0 = static_cast<long long>(gt - pre[ul]) * TILE;
+
+        if ((ti.flags & FLAG_ALIGNED) && e0 + TILE <= ti.numel) {
+            // ---- interior tile, every source 16-byte aligned: branch-free vector path
+            const long long v0 = (e0 / VEC) + threadIdx.x;       // 16-byte vector index
+            float acc[ITERS][VEC];
+            for (int kb = 0; kb < K; kb += KB) {
+                uint4 raw[KB][ITERS];
+#pragma unroll
+                for (int j = 0; j < KB; ++j) {
+                    if (kb + j < K) {
+                        const uint4 *s = static_cast<const uint4 *>(
+                            ldg_ptr(&p.ptrs[static_cast<size_t>(kb + j) * T + u])) + v0;
+#pragma unroll
+                        for (int it = 0; it < ITERS; ++it) raw[j][it] = ld_stream(s + it * NT);
+                    }
+                }
+#pragma unroll
+                for (int j = 0; j < KB; ++j) {
+                    if (kb + j < K) {
+                        const float a = p.rt.coef[kb + j];
+                        const bool first = p.rt.first[kb + j];
+#pragma unroll
+                        for (int it = 0; it < ITERS; ++it) {
+                            float x[VEC];
+                            Elem<Tin>::unpack(raw[j][it], x);
+#pragma unroll
+                            for (int c = 0; c < VEC; ++c)
+                                acc[it][c] = first ? __fmul_rn(a, x[c]) : __fmaf_rn(a, x[c], acc[it][c]);
+                        }
+                        if (p.rt.last[kb + j]) {
+                            float *d = p.transport[p.rt.gid[kb + j]] + ti.dst_off + e0;
+#pragma unroll
+                            for (int it = 0; it < ITERS; ++it) {
+                                float4 *dv = reinterpret_cast<float4 *>(d + (it * NT + threadIdx.x) * VEC);
+#pragma unroll
+                                for (int q = 0; q < VEC / 4; ++q)
+                                    dv[q] = make_float4(acc[it][4 * q], acc[it][4 * q + 1],
+                                                        acc[it][4 * q + 2], acc[it][4 * q + 3]);
+                            }
+                        }
+                    }
+                }
+            }
+        } else {
+            // ---- ragged tail, padding or misaligned tensor: groups of 4 elements, element loads
+            for (long long e = e0 + 4 * threadIdx.x; e < e0 + TILE && e < ti.ext; e += 4 * NT) {
+                float acc[4] = {0.f, 0.f, 0.f, 0.f};
+                for (int k = 0; k < K; ++k) {
+                    const Tin *s = static_cast<const Tin *>(ldg_ptr(&p.ptrs[static_cast<size_t>(k) * T + u]));
+                    const float a = p.rt.coef[k];
+                    const bool first = p.rt.first[k];
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) {
+                        if (e + c < ti.numel) {
+                            const float x = Elem<Tin>::widen(s[e + c]);
+                            acc[c] = first ? __fmul_rn(a, x) : __fmaf_rn(a, x, acc[c]);
+                        } else {
+                            acc[c] = 0.f;
+                        }
+                    }
+                    if (p.rt.last[k])
+                        *reinterpret_cast<float4 *>(p.transport[p.rt.gid[k]] + ti.dst_off + e) =
+                            make_float4(acc[0], acc[1], acc[2], acc[3]);
+                }
+            }
+        }
+    }
+}
+
+// ------------------------------------------------------------------ K2: inter-group combine + scale + cast + unpack
+// out_c^(u)[e] = cast(scale * sum_g W_g P_g[off_u + e]) for every copy c < R.
+template <typename Tout>
+__global__ void __launch_bounds__(NT) k2_combine_unpack(const __grid_constant__ K2Params p) {
+    constexpr int VEC = Elem<Tout>::VEC;
+    constexpr int ITERS = TILE / (NT * VEC);
+    extern __shared__ int smem_prefix[];
+    const int *pre = stage_prefix(p.tp, smem_prefix);
+    const int nu = p.tp.u_hi - p.tp.u_lo;
+    const int G = p.gt.G;
+    const int T = p.tp.T;
+
+    for (int tile = blockIdx.x; tile < p.tp.n_tiles; tile += gridDim.x) {
+        const int gt = tile + p.tp.tile_lo;
+        const int ul = find_tensor(pre, nu, gt);
+        const int u = ul + p.tp.u_lo;
+        const TInfo ti = p.tp.info[u];
+        const long long e0 = static_cast<long long>(gt - pre[ul]) * TILE;
+
+        if (p.out_aligned[u] && e0 + TILE <= ti.numel) {
+            float acc[ITERS][VEC];
+#pragma unroll
+            for (int it = 0; it < ITERS; ++it) {
+                const long long e = e0 + (it * NT + threadIdx.x) * VEC;
+                for (int g = 0; g < G; ++g) {
+                    const float4 *s = reinterpret_cast<const float4 *>(p.src[g] + ti.dst_off + e);
+                    const float w = p.gt.W[g];
+#pragma unroll
+                    for (int q = 0; q < VEC / 4; ++q) {
+                        const float4 v = s[q];
+                        if (g == 0) {
+                            acc[it][4 * q] = __fmul_rn(w, v.x); acc[it][4 * q + 1] = __fmul_rn(w, v.y);
+                            acc[it][4 * q + 2] = __fmul_rn(w, v.z); acc[it][4 * q + 3] = __fmul_rn(w, v.w);
+                        } else {
+                            acc[it][4 * q] = __fmaf_rn(w, v.x, acc[it][4 * q]);
+                            acc[it][4 * q + 1] = __fmaf_rn(w, v.y, acc[it][4 * q + 1]);
+                            acc[it][4 * q + 2] = __fmaf_rn(w, v.z, acc[it][4 * q + 2]);
+                            acc[it][4 * q + 3] = __fmaf_rn(w, v.w, acc[it][4 * q + 3]);
+                        }
+                    }
+                }
+            }
+#pragma unroll
+            for (int it = 0; it < ITERS; ++it) {
+                uint4 o;
+                float y[VEC];
+#pragma unroll
+                for (int c = 0; c < VEC; ++c) y[c] = __fmul_rn(acc[it][c], p.scale);
+                if constexpr (VEC == 4) {
+                    o = make_uint4(__float_as_uint(y[0]), __float_as_uint(y[1]), __float_as_uint(y[2]),
+                                   __float_as_uint(y[3]));
+                } else {
+                    o = make_uint4(pack_bf16x2(y[0], y[1]), pack_bf16x2(y[2], y[3]),
+                                   pack_bf16x2(y[4], y[5]), pack_bf16x2(y[6], y[7]));
+                }
+                const long long vi = e0 / VEC + it * NT + threadIdx.x;
+                for (int c = 0; c < p.R; ++c)
+                    static_cast<uint4 *>(ldg_ptr(&p.out_ptrs[static_cast<size_t>(c) * T + u]))[vi] = o;
+            }
+        } else {
+            for (long long e = e0 + threadIdx.x; e < e0 + TILE && e < ti.numel; e += NT) {
+                float acc = __fmul_rn(p.gt.W[0], p.src[0][ti.dst_off + e]);
+                for (int g = 1; g < G; ++g) acc = __fmaf_rn(p.gt.W[g], p.src[g][ti.dst_off + e], acc);
+                const float y = __fmul_rn(acc, p.scale);
+                for (int c = 0; c < p.R; ++c) {
+                    void *d = ldg_ptr(&p.out_ptrs[static_cast<size_t>(c) * T + u]);
+                    if (VEC == 4) static_cast<float *>(d)[e] = y;
+                    else static_cast<unsigned short *>(d)[e] = static_cast<unsigned short>(pack_bf16x2(y, 0.f) & 0xFFFFu);
+                }
+            }
+        }
+    }
+}
+
+// ------------------------------------------------------------------ flat inter-group combine into a combined buffer
+__global__ void __launch_bounds__(NT) k_combine_flat(const __grid_constant__ K2Params p, float *combined,
+                                                     long long lo, long long n4) {
+    const int G = p.gt.G;
+    for (long long i = blockIdx.x * static_cast<long long>(NT) + threadIdx.x; i < n4;
+         i += static_cast<long long>(gridDim.x) * NT) {
+        const long long e = lo + 4 * i;
+        float4 v = *reinterpret_cast<const float4 *>(p.src[0] + e);
+        const float w0 = p.gt.W[0];
+        float4 acc = make_float4(__fmul_rn(w0, v.x), __fmul_rn(w0, v.y), __fmul_rn(w0, v.z), __fmul_rn(w0, v.w));
+        for (int g = 1; g < G; ++g) {
+            v = *reinterpret_cast<const float4 *>(p.src[g] + e);
+            const float w = p.gt.W[g];
+            acc.x = __fmaf_rn(w, v.x, acc.x); acc.y = __fmaf_rn(w, v.y, acc.y);
+            acc.z = __fmaf_rn(w, v.z, acc.z); acc.w = __fmaf_rn(w, v.w, acc.w);
+        }
+        *reinterpret_cast<float4 *>(combined + e) = acc;
+    }
+}
+
+// ------------------------------------------------------------------ standalone pack (bit copy of every rank's tensors into its flat buffer)
+template <typename Tin>
+__global__ void __launch_bounds__(NT) k_pack(const __grid_constant__ PackParams p) {
+    constexpr int VEC = Elem<Tin>::VEC;
+    constexpr int ITERS = TILE / (NT * VEC);
+    extern __shared__ int smem_prefix[];
+    const int *pre = stage_prefix(p.tp, smem_prefix);
+    const int nu = p.tp.u_hi - p.tp.u_lo;
+    const int T = p.tp.T;
+    const int k = blockIdx.y;
+    Tin *flat = static_cast<Tin *>(p.flat[k]);
+
+    for (int tile = blockIdx.x; tile < p.tp.n_tiles; tile += gridDim.x) {
+        const int gt = tile + p.tp.tile_lo;
+        const int ul = find_tensor(pre, nu, gt);
+        const int u = ul + p.tp.u_lo;
+        const TInfo ti = p.tp.info[u];
+        const long long e0 = static_cast<long long>(gt - pre[ul]) * TILE;
+        const Tin *s = static_cast<const Tin *>(ldg_ptr(&p.ptrs[static_cast<size_t>(k) * T + u]));
+        if ((ti.flags & FLAG_ALIGNED) && e0 + TILE <= ti.numel) {
+            const uint4 *sv = reinterpret_cast<const uint4 *>(s + e0) + threadIdx.x;
+            uint4 *dv = reinterpret_cast<uint4 *>(flat + ti.dst_off + e0) + threadIdx.x;
+            uint4 raw[ITERS];
+#pragma unroll
+            for (int it = 0; it < ITERS; ++it) raw[it] = ld_stream(sv + it * NT);
+#pragma unroll
+            for (int it = 0; it < ITERS; ++it) dv[it * NT] = raw[it];
+        } else {
+            for (long long e = e0 + threadIdx.x; e < e0 + TILE && e < ti.ext; e += NT)
+                flat[ti.dst_off + e] = e < ti.numel ? s[e] : Tin(0);
+        }
+    }
+}
+
+// ------------------------------------------------------------------ standalone casts
+__global__ void __launch_bounds__(NT) k_cast_bf16_to_f32(const unsigned short *in, float *out, long long n) {
+    for (long long i = blockIdx.x * static_cast<long long>(NT) + threadIdx.x; i < n;
+         i += static_cast<long long>(gridDim.x) * NT)
+        out[i] = __uint_as_float(static_cast<unsigned>(in[i]) << 16);
+}
+__global__ void __launch_bounds__(NT) k_cast_f32_to_bf16(const float *in, unsigned short *out, long long n) {
+    for (long long i = blockIdx.x * static_cast<long long>(NT) + threadIdx.x; i < n;
+         i += static_cast<long long>(gridDim.x) * NT)
+        out[i] = static_cast<unsigned short>(pack_bf16x2(in[i], 0.f) & 0xFFFFu);
+}
+
+// ------------------------------------------------------------------ host-side state
+struct StageSlot {
+    cudaEvent_t done = nullptr;
+    bool recorded = false;
+};
+
+}  // namespace
+
+struct kt_ctx {
+    int device = 0;
+    int sm_count = 0;
+    int K = 0, G = 0;
+    std::vector<int32_t> group_of, shares;
+    std::vector<int> order;          // group-major rank order
+    RankTab rt{};
+    GroupTab gt{};
+
+    // plan (valid once planned)
+    bool planned = false;
+    int T = 0;
+    int in_dtype = KT_F32;
+    std::vector<int64_t> numel, tensor_offset;       // user tensor order
+    std::vector<int32_t> bucket_of;
+    std::vector<int64_t> bucket_start, bucket_numel;
+    std::vector<int> bucket_u_lo, bucket_u_hi;       // transport-order tensor range per bucket
+    int64_t transport_numel = 0;
+    std::vector<int> prefix;                         // [T+1], transport order
+    std::vector<TInfo> info;                         // [T], transport order
+
+    // device tables
+    void *d_tables = nullptr;        // one allocation: prefix | info | grad ptrs
+    int *d_prefix = nullptr;
+    TInfo *d_info = nullptr;
+    const void **d_ptrs = nullptr;
+    void *d_out = nullptr;           // out pointer table + aligned flags
+    size_t d_out_cap = 0;
+    std::vector<void *> out_cached;  // host copy of the uploaded out pointers
+    int out_R = 0, out_dtype = -1;
+
+    cudaEvent_t ev_main = nullptr;
+    std::vector<StageSlot> slots[2]; // per direction: index 0 = all buckets, 1 + b = bucket b
+    int64_t launches = 0;
+    std::vector<std::pair<const void *, int>> occupancy;   // resident CTAs per SM, per kernel
+};
+
+namespace {
+
+int64_t round_up(int64_t x, int64_t m) { return (x + m - 1) / m * m; }
+
+// Bucket plan: tensors in reverse list order, greedy fill up to cap elements, tensors never
+// split, every tensor at a multiple of 8 elements, every bucket at a multiple of 64.
+struct BucketPlan {
+    std::vector<int64_t> offset;      // [T] list order
+    std::vector<int32_t> bucket_of;   // [T] list order
+    std::vector<int64_t> start;       // [n_buckets]
+    std::vector<int> u_lo, u_hi;      // transport-order tensor range of each bucket
+    int64_t total = 0;
+};
+
+void plan_buckets(const int64_t *numel, int T, int64_t bucket_cap_bytes, BucketPlan *bp) {
+    const int64_t cap = bucket_cap_bytes / 4;
+    bp->offset.assign(T, 0);
+    bp->bucket_of.assign(T, 0);
+    bp->start.assign(1, 0);
+    bp->u_lo.assign(1, 0);
+    bp->u_hi.clear();
+    int64_t next = 0, open_start = 0;
+    bool open_empty = true;
+    for (int u = 0; u < T; ++u) {                 // u: transport order, t: list order
+        const int t = T - 1 - u;
+        int64_t at = round_up(next, 8);
+        if (!open_empty && (at - open_start) + numel[t] > cap) {
+            open_start = round_up(next, 64);
+            at = open_start;
+            bp->start.push_back(open_start);
+            bp->u_hi.push_back(u);
+            bp->u_lo.push_back(u);
+        }
+        bp->offset[t] = at;
+        bp->bucket_of[t] = static_cast<int32_t>(bp->start.size() - 1);
+        next = at + numel[t];
+        open_empty = false;
+    }
+    bp->u_hi.push_back(T);
+    bp->total = round_up(next, 64);
+}
+
+int compute_coefficients(kt_ctx *c) {
+    std::vector<int64_t> Bg(c->G, 0);
+    int64_t B = 0;
+    for (int r = 0; r < c->K; ++r) {
+        Bg[c->group_of[r]] += c->shares[r];
+        B += c->shares[r];
+    }
+    c->order.clear();
+    for (int g = 0; g < c->G; ++g)
+        for (int r = 0; r < c->K; ++r)
+            if (c->group_of[r] == g) c->order.push_back(r);
+    std::memset(&c->rt, 0, sizeof(c->rt));
+    c->rt.K = c->K;
+    for (int k = 0; k < c->K; ++k) {
+        const int r = c->order[k];
+        const int g = c->group_of[r];
+        c->rt.coef[k] = static_cast<float>(static_cast<double>(c->shares[r]) / static_cast<double>(Bg[g]));
+        c->rt.gid[k] = static_cast<signed char>(g);
+        c->rt.first[k] = (k == 0 || c->group_of[c->order[k - 1]] != g);
+        c->rt.last[k] = (k == c->K - 1 || c->group_of[c->order[k + 1]] != g);
+    }
+    std::memset(&c->gt, 0, sizeof(c->gt));
+    c->gt.G = c->G;
+    for (int g = 0; g < c->G; ++g)
+        c->gt.W[g] = static_cast<float>(static_cast<double>(Bg[g]) / static_cast<double>(B));
+    return KT_OK;
+}
+
+int check_shares(const int32_t *shares, int K) {
+    if (!shares) return fail(KT_ERR_INVALID, "shares is NULL");
+    for (int r = 0; r < K; ++r)
+        if (shares[r] < 1) return fail(KT_ERR_INVALID, "shares[%d] = %d, must be >= 1", r, shares[r]);
+    return KT_OK;
+}
+
+bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// Grid of a grid-stride kernel: one wave of resident CTAs (SM count x occupancy), or
+// fewer when there is less work.  Occupancy is queried once per kernel and cached.
+template <typename Kern>
+int grid_for(kt_ctx *c, Kern kernel, size_t smem, long long units) {
+    const void *key = reinterpret_cast<const void *>(kernel);
+    int per_sm = 0;
+    for (const auto &kv : c->occupancy)
+        if (kv.first == key) per_sm = kv.second;
+    if (!per_sm) {
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, NT, smem) != cudaSuccess || per_sm < 1) {
+            cudaGetLastError();
+            per_sm = 1;
+        }
+        c->occupancy.emplace_back(key, per_sm);
+    }
+    const long long cap = static_cast<long long>(c->sm_count) * per_sm;
+    const long long g = units < cap ? units : cap;
+    return static_cast<int>(g < 1 ? 1 : g);
+}
+
+// tile range of a bucket (or of everything for bucket == -1)
+int make_tile_plan(const kt_ctx *c, int bucket, TilePlan *tp) {
+    if (bucket < -1 || bucket >= static_cast<int>(c->bucket_start.size()))
+        return fail(KT_ERR_SHAPE, "bucket %d out of range [-1, %d)", bucket, (int)c->bucket_start.size());
+    tp->prefix = c->d_prefix;
+    tp->info = c->d_info;
+    tp->T = c->T;
+    tp->u_lo = bucket < 0 ? 0 : c->bucket_u_lo[bucket];
+    tp->u_hi = bucket < 0 ? c->T : c->bucket_u_hi[bucket];
+    tp->tile_lo = c->prefix[tp->u_lo];
+    tp->n_tiles = c->prefix[tp->u_hi] - tp->tile_lo;
+    tp->prefix_in_smem = (tp->u_hi - tp->u_lo + 1) * sizeof(int) <= 32 * 1024;
+    return KT_OK;
+}
+
+size_t prefix_smem(const TilePlan &tp) {
+    return tp.prefix_in_smem ? (tp.u_hi - tp.u_lo + 1) * sizeof(int) : 0;
+}
+
+void bucket_range(const kt_ctx *c, int bucket, int64_t *lo, int64_t *n) {
+    if (bucket < 0) {
+        *lo = 0;
+        *n = c->transport_numel;
+    } else {
+        *lo = c->bucket_start[bucket];
+        *n = c->bucket_numel[bucket];
+    }
+}
+
+int check_ctx(const kt_ctx *c, bool need_plan) {
+    if (!c) return fail(KT_ERR_INVALID, "ctx is NULL");
+    if (need_plan && !c->planned) return fail(KT_ERR_STATE, "kt_bucket_pack has not been called on this context");
+    return KT_OK;
+}
+
+int check_buffers(const kt_ctx *c, const float *const *bufs, int n, const char *what) {
+    if (!bufs) return fail(KT_ERR_INVALID, "%s is NULL", what);
+    for (int g = 0; g < n; ++g) {
+        if (!bufs[g]) return fail(KT_ERR_INVALID, "%s[%d] is NULL", what, g);
+        if (!aligned16(bufs[g])) return fail(KT_ERR_ALIGN, "%s[%d] is not 16-byte aligned", what, g);
+    }
+    (void)c;
+    return KT_OK;
+}
+
+template <typename Tin>
+int launch_k1(kt_ctx *c, const K1Params &p, cudaStream_t s) {
+    const size_t sm = prefix_smem(p.tp);
+    if (c->K <= 4)
+        k1_intra_reduce<Tin, 4><<<grid_for(c, k1_intra_reduce<Tin, 4>, sm, p.tp.n_tiles), NT, sm, s>>>(p);
+    else
+        k1_intra_reduce<Tin, 8><<<grid_for(c, k1_intra_reduce<Tin, 8>, sm, p.tp.n_tiles), NT, sm, s>>>(p);
+    c->launches += 1;
+    KT_CUDA(cudaGetLastError());
+    return KT_OK;
+}
+
+}  // namespace
+
+// ====================================================================== C ABI
+extern "C" {
+
+int kt_schedule(const double *step_times, int K, int global_batch, int32_t *shares_out) {
+    if (!step_times || !shares_out) return fail(KT_ERR_INVALID, "NULL argument");
+    if (K < 1 || K > KT_MAX_RANKS) return fail(KT_ERR_INVALID, "K = %d outside [1, %d]", K, KT_MAX_RANKS);
+    if (global_batch < K) return fail(KT_ERR_INVALID, "global_batch %d < K %d: some rank would idle", global_batch, K);
+    double t_min = INFINITY;
+    for (int i = 0; i < K; ++i) {
+        const double t = step_times[i];
+        if (!(t > 0.0) || !std::isfinite(t)) return fail(KT_ERR_INVALID, "step_times[%d] must be finite and > 0", i);
+        t_min = t < t_min ? t : t_min;
+    }
+    std::vector<double> score(K), rem(K);
+    double total = 0.0;
+    for (int i = 0; i < K; ++i) {
+        score[i] = t_min / step_times[i];
+        total = total + score[i];
+    }
+    long long assigned = 0;
+    for (int i = 0; i < K; ++i) {
+        const double quota = score[i] / total * static_cast<double>(global_batch);
+        const double whole = std::floor(quota);
+        shares_out[i] = static_cast<int32_t>(whole);
+        rem[i] = quota - whole;
+        assigned += shares_out[i];
+    }
+    // largest remainders first (tie: lower rank); fewer than K units can be missing
+    std::vector<char> served(K, 0);
+    long long left = global_batch - assigned;
+    while (left > 0) {
+        int pick = -1;
+        for (int i = 0; i < K; ++i)
+            if (!served[i] && (pick < 0 || rem[i] > rem[pick])) pick = i;
+        if (pick < 0) {          // every rank served once already: next round
+            served.assign(K, 0);
+            continue;
+        }
+        served[pick] = 1;
+        shares_out[pick] += 1;
+        --left;
+    }
+    for (long long over = assigned - global_batch; over > 0; --over) {   // rounding noise only
+        int pick = 0;
+        for (int i = 1; i < K; ++i)
+            if (shares_out[i] > shares_out[pick]) pick = i;
+        shares_out[pick] -= 1;
+    }
+    // nobody idles: take from the largest share (tie: slowest, then higher rank)
+    for (int i = 0; i < K; ++i) {
+        if (shares_out[i] >= 1) continue;
+        int donor = 0;
+        for (int j = 1; j < K; ++j)
+            if (shares_out[j] > shares_out[donor] ||
+                (shares_out[j] == shares_out[donor] && step_times[j] >= step_times[donor]))
+                donor = j;
+        shares_out[donor] -= 1;
+        shares_out[i] += 1;
+    }
+    return KT_OK;
+}
+
+int kt_groups_init(const int32_t *group_of, const int32_t *shares, int K, int G, kt_ctx **out) {
+    if (!out) return fail(KT_ERR_INVALID, "out is NULL");
+    *out = nullptr;
+    if (!group_of) return fail(KT_ERR_INVALID, "group_of is NULL");
+    if (K < 1 || K > KT_MAX_RANKS) return fail(KT_ERR_INVALID, "K = %d outside [1, %d]", K, KT_MAX_RANKS);
+    if (G < 1 || G > KT_MAX_GROUPS || G > K) return fail(KT_ERR_INVALID, "G = %d outside [1, min(K, %d)]", G, KT_MAX_GROUPS);
+    if (int rc = check_shares(shares, K)) return rc;
+    std::vector<int> members(G, 0);
+    for (int r = 0; r < K; ++r) {
+        if (group_of[r] < 0 || group_of[r] >= G) return fail(KT_ERR_INVALID, "group_of[%d] = %d outside [0, %d)", r, group_of[r], G);
+        members[group_of[r]] += 1;
+    }
+    for (int g = 0; g < G; ++g)
+        if (!members[g]) return fail(KT_ERR_INVALID, "group %d has no rank", g);
+
+    kt_ctx *c = new (std::nothrow) kt_ctx();
+    if (!c) return fail(KT_ERR_NOMEM, "out of host memory");
+    c->K = K;
+    c->G = G;
+    c->group_of.assign(group_of, group_of + K);
+    c->shares.assign(shares, shares + K);
+    compute_coefficients(c);
+    cudaError_t e = cudaGetDevice(&c->device);
+    if (e == cudaSuccess) e = cudaDeviceGetAttribute(&c->sm_count, cudaDevAttrMultiProcessorCount, c->device);
+    if (e == cudaSuccess) e = cudaEventCreateWithFlags(&c->ev_main, cudaEventDisableTiming);
+    if (e != cudaSuccess) {
+        delete c;
+        return fail(KT_ERR_CUDA, "kt_groups_init: %s", cudaGetErrorString(e));
+    }
+    *out = c;
+    return KT_OK;
+}
+
+int kt_set_shares(kt_ctx *c, const int32_t *shares) {
+    if (int rc = check_ctx(c, false)) return rc;
+    if (int rc = check_shares(shares, c->K)) return rc;
+    c->shares.assign(shares, shares + c->K);
+    return compute_coefficients(c);
+}
+
+int kt_set_coefficients(kt_ctx *c, const float *a, const float *W) {
+    if (int rc = check_ctx(c, false)) return rc;
+    if (!a || !W) return fail(KT_ERR_INVALID, "NULL argument");
+    for (int k = 0; k < c->K; ++k) c->rt.coef[k] = a[c->order[k]];
+    for (int g = 0; g < c->G; ++g) c->gt.W[g] = W[g];
+    return KT_OK;
+}
+
+int kt_get_coefficients(const kt_ctx *c, float *a_out, float *W_out) {
+    if (int rc = check_ctx(c, false)) return rc;
+    if (a_out)
+        for (int k = 0; k < c->K; ++k) a_out[c->order[k]] = c->rt.coef[k];
+    if (W_out)
+        for (int g = 0; g < c->G; ++g) W_out[g] = c->gt.W[g];
+    return KT_OK;
+}
+
+int kt_bucket_pack(kt_ctx *c, const void *const *grads, const int64_t *numel, int T, int in_dtype,
+                   int64_t bucket_cap_bytes, void *const *flat_out, void *stream) {
+    if (int rc = check_ctx(c, false)) return rc;
+    if (!grads || !numel) return fail(KT_ERR_INVALID, "NULL argument");
+    if (T < 1) return fail(KT_ERR_INVALID, "T = %d must be >= 1", T);
+    if (in_dtype != KT_F32 && in_dtype != KT_BF16) return fail(KT_ERR_INVALID, "unknown in_dtype %d", in_dtype);
+    if (bucket_cap_bytes < 4) return fail(KT_ERR_INVALID, "bucket_cap_bytes must be >= 4");
+    const size_t es = in_dtype == KT_F32 ? 4 : 2;
+    for (int t = 0; t < T; ++t) {
+        if (numel[t] < 0) return fail(KT_ERR_INVALID, "numel[%d] is negative", t);
+        for (int r = 0; r < c->K; ++r) {
+            const void *p = grads[static_cast<size_t>(r) * T + t];
+            if (numel[t] > 0 && !p) return fail(KT_ERR_INVALID, "grads[%d][%d] is NULL", r, t);
+            if (reinterpret_cast<uintptr_t>(p) % es) return fail(KT_ERR_ALIGN, "grads[%d][%d] is not element aligned", r, t);
+        }
+    }
+    if (flat_out)
+        for (int r = 0; r < c->K; ++r) {
+            if (!flat_out[r]) return fail(KT_ERR_INVALID, "flat_out[%d] is NULL", r);
+            if (!aligned16(flat_out[r])) return fail(KT_ERR_ALIGN, "flat_out[%d] is not 16-byte aligned", r);
+        }
+
+    BucketPlan bp;
+    plan_buckets(numel, T, bucket_cap_bytes, &bp);
+    const std::vector<int64_t> &offset = bp.offset;
+    const std::vector<int32_t> &bof = bp.bucket_of;
+    const std::vector<int64_t> &bstart = bp.start;
+    const std::vector<int> &b_lo = bp.u_lo, &b_hi = bp.u_hi;
+    const int64_t total = bp.total;
+    const int nb = static_cast<int>(bstart.size());
+
+    // ---- tile tables in transport order
+    std::vector<int> prefix(T + 1, 0);
+    std::vector<TInfo> info(T);
+    for (int u = 0; u < T; ++u) {
+        const int t = T - 1 - u;
+        const int64_t end = (u + 1 < T) ? offset[T - 2 - u] : total;
+        TInfo &ti = info[u];
+        ti.dst_off = offset[t];
+        ti.numel = numel[t];
+        ti.ext = end - offset[t];
+        ti.flags = FLAG_ALIGNED;
+        ti.pad_ = 0;
+        for (int r = 0; r < c->K; ++r)
+            if (!aligned16(grads[static_cast<size_t>(r) * T + t])) ti.flags = 0;
+        const int64_t tiles = (ti.ext + TILE - 1) / TILE;
+        if (prefix[u] + tiles > 0x7FFFFFF0LL) return fail(KT_ERR_SHAPE, "too many elements for one plan");
+        prefix[u + 1] = prefix[u] + static_cast<int>(tiles);
+    }
+    std::vector<const void *> ptrs(static_cast<size_t>(c->K) * T);
+    for (int k = 0; k < c->K; ++k)
+        for (int u = 0; u < T; ++u)
+            ptrs[static_cast<size_t>(k) * T + u] = grads[static_cast<size_t>(c->order[k]) * T + (T - 1 - u)];
+
+    // ---- upload (one allocation, three 256-byte aligned regions)
+    KT_CUDA(cudaSetDevice(c->device));
+    const size_t sz_prefix = round_up((T + 1) * sizeof(int), 256);
+    const size_t sz_info = round_up(T * sizeof(TInfo), 256);
+    const size_t sz_ptrs = round_up(ptrs.size() * sizeof(void *), 256);
+    void *d = nullptr;
+    if (cudaMalloc(&d, sz_prefix + sz_info + sz_ptrs) != cudaSuccess) {
+        cudaGetLastError();
+        return fail(KT_ERR_NOMEM, "device allocation of %zu bytes failed", sz_prefix + sz_info + sz_ptrs);
+    }
+    std::vector<char> staging(sz_prefix + sz_info + sz_ptrs, 0);
+    std::memcpy(staging.data(), prefix.data(), (T + 1) * sizeof(int));
+    std::memcpy(staging.data() + sz_prefix, info.data(), T * sizeof(TInfo));
+    std::memcpy(staging.data() + sz_prefix + sz_info, ptrs.data(), ptrs.size() * sizeof(void *));
+    cudaError_t e = cudaMemcpy(d, staging.data(), staging.size(), cudaMemcpyHostToDevice);
+    if (e != cudaSuccess) {
+        cudaFree(d);
+        return fail(KT_ERR_CUDA, "table upload: %s", cudaGetErrorString(e));
+    }
+    if (c->d_tables) cudaFree(c->d_tables);
+    c->d_tables = d;
+    c->d_prefix = static_cast<int *>(d);
+    c->d_info = reinterpret_cast<TInfo *>(static_cast<char *>(d) + sz_prefix);
+    c->d_ptrs = reinterpret_cast<const void **>(static_cast<char *>(d) + sz_prefix + sz_info);
+
+    c->T = T;
+    c->in_dtype = in_dtype;
+    c->numel.assign(numel, numel + T);
+    c->tensor_offset = offset;
+    c->bucket_of = bof;
+    c->bucket_start = bstart;
+    c->bucket_numel.resize(nb);
+    for (int b = 0; b < nb; ++b) c->bucket_numel[b] = (b + 1 < nb ? bstart[b + 1] : total) - bstart[b];
+    c->bucket_u_lo = b_lo;
+    c->bucket_u_hi = b_hi;
+    c->transport_numel = total;
+    c->prefix = prefix;
+    c->info = info;
+    c->planned = true;
+    c->out_cached.clear();
+    for (int dir = 0; dir < 2; ++dir) {
+        for (auto &s : c->slots[dir]) s.recorded = false;
+        while (static_cast<int>(c->slots[dir].size()) < nb + 1) {
+            StageSlot s;
+            KT_CUDA(cudaEventCreateWithFlags(&s.done, cudaEventDisableTiming));
+            c->slots[dir].push_back(s);
+        }
+    }
+
+    if (flat_out) {
+        PackParams p{};
+        if (int rc = make_tile_plan(c, -1, &p.tp)) return rc;
+        p.ptrs = c->d_ptrs;
+        p.K = c->K;
+        for (int k = 0; k < c->K; ++k) p.flat[k] = flat_out[c->order[k]];
+        if (p.tp.n_tiles > 0) {
+            const size_t sm = prefix_smem(p.tp);
+            cudaStream_t s = static_cast<cudaStream_t>(stream);
+            if (in_dtype == KT_F32)
+                k_pack<float><<<dim3(grid_for(c, k_pack<float>, sm, p.tp.n_tiles), c->K), NT, sm, s>>>(p);
+            else
+                k_pack<unsigned short><<<dim3(grid_for(c, k_pack<unsigned short>, sm, p.tp.n_tiles), c->K), NT, sm, s>>>(p);
+            c->launches += 1;
+            KT_CUDA(cudaGetLastError());
+        }
+    }
+    return KT_OK;
+}
+
+int kt_plan_buckets(const int64_t *numel, int T, int64_t bucket_cap_bytes, int32_t *n_buckets,
+                    int64_t *bucket_start, int64_t *bucket_numel, int64_t *tensor_offset, int32_t *bucket_of,
+                    int64_t *transport_numel) {
+    if (!numel) return fail(KT_ERR_INVALID, "numel is NULL");
+    if (T < 1) return fail(KT_ERR_INVALID, "T = %d must be >= 1", T);
+    if (bucket_cap_bytes < 4) return fail(KT_ERR_INVALID, "bucket_cap_bytes must be >= 4");
+    for (int t = 0; t < T; ++t)
+        if (numel[t] < 0) return fail(KT_ERR_INVALID, "numel[%d] is negative", t);
+    BucketPlan bp;
+    plan_buckets(numel, T, bucket_cap_bytes, &bp);
+    const int nb = static_cast<int>(bp.start.size());
+    if (n_buckets) *n_buckets = nb;
+    for (int b = 0; b < nb; ++b) {
+        if (bucket_start) bucket_start[b] = bp.start[b];
+        if (bucket_numel) bucket_numel[b] = (b + 1 < nb ? bp.start[b + 1] : bp.total) - bp.start[b];
+    }
+    if (tensor_offset) std::memcpy(tensor_offset, bp.offset.data(), T * sizeof(int64_t));
+    if (bucket_of) std::memcpy(bucket_of, bp.bucket_of.data(), T * sizeof(int32_t));
+    if (transport_numel) *transport_numel = bp.total;
+    return KT_OK;
+}
+
+int kt_plan_query(const kt_ctx *c, int32_t *n_buckets, int64_t *bucket_start, int64_t *bucket_numel,
+                  int64_t *tensor_offset, int32_t *bucket_of, int64_t *transport_numel) {
+    if (int rc = check_ctx(c, true)) return rc;
+    const int nb = static_cast<int>(c->bucket_start.size());
+    if (n_buckets) *n_buckets = nb;
+    if (bucket_start) std::memcpy(bucket_start, c->bucket_start.data(), nb * sizeof(int64_t));
+    if (bucket_numel) std::memcpy(bucket_numel, c->bucket_numel.data(), nb * sizeof(int64_t));
+    if (tensor_offset) std::memcpy(tensor_offset, c->tensor_offset.data(), c->T * sizeof(int64_t));
+    if (bucket_of) std::memcpy(bucket_of, c->bucket_of.data(), c->T * sizeof(int32_t));
+    if (transport_numel) *transport_numel = c->transport_numel;
+    return KT_OK;
+}
+
+int kt_hier_reduce(kt_ctx *c, int phase, int bucket, float *const *transport, float *combined, void *stream) {
+    if (int rc = check_ctx(c, true)) return rc;
+    if (phase != KT_INTRA && phase != KT_INTER && phase != KT_BOTH) return fail(KT_ERR_INVALID, "unknown phase %d", phase);
+    if (int rc = check_buffers(c, transport, c->G, "transport")) return rc;
+    if (phase & KT_INTER) {
+        if (!combined) return fail(KT_ERR_INVALID, "combined is NULL");
+        if (!aligned16(combined)) return fail(KT_ERR_ALIGN, "combined is not 16-byte aligned");
+    }
+    TilePlan tp{};
+    if (int rc = make_tile_plan(c, bucket, &tp)) return rc;
+    KT_CUDA(cudaSetDevice(c->device));
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+
+    if ((phase & KT_INTRA) && tp.n_tiles > 0) {
+        K1Params p{};
+        p.tp = tp;
+        p.ptrs = c->d_ptrs;
+        p.rt = c->rt;
+        for (int g = 0; g < c->G; ++g) p.transport[g] = transport[g];
+        const int rc = c->in_dtype == KT_F32 ? launch_k1<float>(c, p, s) : launch_k1<unsigned short>(c, p, s);
+        if (rc) return rc;
+    }
+    if (phase & KT_INTER) {
+        int64_t lo, n;
+        bucket_range(c, bucket, &lo, &n);
+        if (n > 0) {
+            K2Params p{};
+            p.gt = c->gt;
+            for (int g = 0; g < c->G; ++g) p.src[g] = transport[g];
+            const long long n4 = n / 4;   // bucket ranges are multiples of 64 elements
+            k_combine_flat<<<grid_for(c, k_combine_flat, 0, (n4 + NT - 1) / NT), NT, 0, s>>>(p, combined, lo, n4);
+            c->launches += 1;
+            KT_CUDA(cudaGetLastError());
+        }
+    }
+    return KT_OK;
+}
+
+int kt_stage_to_host(kt_ctx *c, int dir, int bucket, float *const *transport, float *const *host_pinned,
+                     void *main_stream, void *side_stream) {
+    if (int rc = check_ctx(c, true)) return rc;
+    if (dir != KT_D2H && dir != KT_H2D) return fail(KT_ERR_INVALID, "unknown direction %d", dir);
+    if (!transport || !host_pinned) return fail(KT_ERR_INVALID, "NULL argument");
+    if (bucket < -1 || bucket >= static_cast<int>(c->bucket_start.size()))
+        return fail(KT_ERR_SHAPE, "bucket %d out of range", bucket);
+    for (int g = 0; g < c->G; ++g)
+        if (!transport[g] || !host_pinned[g]) return fail(KT_ERR_INVALID, "buffer %d is NULL", g);
+    int64_t lo, n;
+    bucket_range(c, bucket, &lo, &n);
+    KT_CUDA(cudaSetDevice(c->device));
+    cudaStream_t ms = static_cast<cudaStream_t>(main_stream), ss = static_cast<cudaStream_t>(side_stream);
+    KT_CUDA(cudaEventRecord(c->ev_main, ms));
+    KT_CUDA(cudaStreamWaitEvent(ss, c->ev_main, 0));
+    if (dir == KT_H2D) {
+        StageSlot &d2h = c->slots[KT_D2H][bucket + 1];
+        if (d2h.recorded) KT_CUDA(cudaStreamWaitEvent(ss, d2h.done, 0));
+        StageSlot &all = c->slots[KT_D2H][0];
+        if (bucket >= 0 && all.recorded) KT_CUDA(cudaStreamWaitEvent(ss, all.done, 0));
+    }
+    for (int g = 0; g < c->G && n > 0; ++g) {
+        if (dir == KT_D2H)
+            KT_CUDA(cudaMemcpyAsync(host_pinned[g] + lo, transport[g] + lo, n * sizeof(float), cudaMemcpyDeviceToHost, ss));
+        else
+            KT_CUDA(cudaMemcpyAsync(transport[g] + lo, host_pinned[g] + lo, n * sizeof(float), cudaMemcpyHostToDevice, ss));
+    }
+    StageSlot &slot = c->slots[dir][bucket + 1];
+    KT_CUDA(cudaEventRecord(slot.done, ss));
+    slot.recorded = true;
+    return KT_OK;
+}
+
+int kt_stage_wait(kt_ctx *c, int dir, int bucket, void *main_stream, int timeout_ms) {
+    if (int rc = check_ctx(c, true)) return rc;
+    if (dir != KT_D2H && dir != KT_H2D) return fail(KT_ERR_INVALID, "unknown direction %d", dir);
+    if (bucket < -1 || bucket >= static_cast<int>(c->bucket_start.size()))
+        return fail(KT_ERR_SHAPE, "bucket %d out of range", bucket);
+    StageSlot &slot = c->slots[dir][bucket + 1];
+    if (!slot.recorded) return fail(KT_ERR_STATE, "no staging copy queued for direction %d, bucket %d", dir, bucket);
+    KT_CUDA(cudaStreamWaitEvent(static_cast<cudaStream_t>(main_stream), slot.done, 0));
+    if (timeout_ms < 0) return KT_OK;
+    const auto deadline = std::chrono::steady_clock::now() + std::chrono::milliseconds(timeout_ms);
+    for (;;) {
+        const cudaError_t e = cudaEventQuery(slot.done);
+        if (e == cudaSuccess) return KT_OK;
+        if (e != cudaErrorNotReady) return fail(KT_ERR_CUDA, "cudaEventQuery: %s", cudaGetErrorString(e));
+        if (std::chrono::steady_clock::now() >= deadline)
+            return fail(KT_ERR_TIMEOUT, "staging copy (direction %d, bucket %d) not finished after %d ms", dir, bucket, timeout_ms);
+        std::this_thread::sleep_for(std::chrono::microseconds(50));
+    }
+}
+
+int kt_unpack_scale(kt_ctx *c, const float *const *src, int from_combined, void *const *out_grads, int R,
+                    int out_dtype, float scale, int bucket, void *stream) {
+    if (int rc = check_ctx(c, true)) return rc;
+    if (!out_grads) return fail(KT_ERR_INVALID, "out_grads is NULL");
+    if (R < 1 || R > c->K) return fail(KT_ERR_SHAPE, "R = %d outside [1, K = %d]", R, c->K);
+    if (out_dtype != KT_F32 && out_dtype != KT_BF16) return fail(KT_ERR_INVALID, "unknown out_dtype %d", out_dtype);
+    const int nsrc = from_combined ? 1 : c->G;
+    if (int rc = check_buffers(c, src, nsrc, "src")) return rc;
+    const size_t es = out_dtype == KT_F32 ? 4 : 2;
+    const int T = c->T;
+    const size_t np = static_cast<size_t>(R) * T;
+    for (size_t i = 0; i < np; ++i) {
+        if (c->numel[i % T] > 0 && !out_grads[i]) return fail(KT_ERR_INVALID, "out_grads[%zu] is NULL", i);
+        if (reinterpret_cast<uintptr_t>(out_grads[i]) % es) return fail(KT_ERR_ALIGN, "out_grads[%zu] is not element aligned", i);
+    }
+    TilePlan tp{};
+    if (int rc = make_tile_plan(c, bucket, &tp)) return rc;
+    KT_CUDA(cudaSetDevice(c->device));
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+
+    // (re)upload the destination table only when it changed
+    const bool same = c->out_R == R && c->out_dtype == out_dtype && c->out_cached.size() == np &&
+                      std::memcmp(c->out_cached.data(), out_grads, np * sizeof(void *)) == 0;
+    const size_t sz_ptrs = round_up(np * sizeof(void *), 256);
+    if (!same) {
+        const size_t need = sz_ptrs + round_up(T, 256);
+        if (need > c->d_out_cap) {
+            // the previous table may still be in use by queued kernels: release it once they are done
+            if (c->d_out) {
+                KT_CUDA(cudaDeviceSynchronize());
+                cudaFree(c->d_out);
+                c->d_out = nullptr;
+                c->d_out_cap = 0;
+            }
+            if (cudaMalloc(&c->d_out, need) != cudaSuccess) {
+                cudaGetLastError();
+                return fail(KT_ERR_NOMEM, "device allocation of %zu bytes failed", need);
+            }
+            c->d_out_cap = need;
+        } else {
+            KT_CUDA(cudaStreamSynchronize(s));   // queued kernels may still read the old table
+        }
+        std::vector<char> staging(sz_ptrs + T, 0);
+        for (int cpy = 0; cpy < R; ++cpy)
+            for (int u = 0; u < T; ++u)
+                reinterpret_cast<void **>(staging.data())[static_cast<size_t>(cpy) * T + u] =
+                    out_grads[static_cast<size_t>(cpy) * T + (T - 1 - u)];
+        for (int u = 0; u < T; ++u) {
+            bool al = true;
+            for (int cpy = 0; cpy < R; ++cpy) al = al && aligned16(out_grads[static_cast<size_t>(cpy) * T + (T - 1 - u)]);
+            staging[sz_ptrs + u] = al ? 1 : 0;
+        }
+        KT_CUDA(cudaMemcpy(c->d_out, staging.data(), staging.size(), cudaMemcpyHostToDevice));
+        c->out_cached.assign(out_grads, out_grads + np);
+        c->out_R = R;
+        c->out_dtype = out_dtype;
+    }
+    if (tp.n_tiles == 0) return KT_OK;
+
+    K2Params p{};
+    p.tp = tp;
+    if (from_combined) {
+        p.gt.G = 1;
+        p.gt.W[0] = 1.0f;     // multiplying by one is exact: S passes through unchanged
+        p.src[0] = src[0];
+    } else {
+        p.gt = c->gt;
+        for (int g = 0; g < c->G; ++g) p.src[g] = src[g];
+    }
+    p.out_ptrs = static_cast<void *const *>(c->d_out);
+    p.out_aligned = static_cast<const unsigned char *>(c->d_out) + sz_ptrs;
+    p.R = R;
+    p.scale = scale;
+    const size_t sm = prefix_smem(tp);
+    if (out_dtype == KT_F32)
+        k2_combine_unpack<float><<<grid_for(c, k2_combine_unpack<float>, sm, tp.n_tiles), NT, sm, s>>>(p);
+    else
+        k2_combine_unpack<unsigned short><<<grid_for(c, k2_combine_unpack<unsigned short>, sm, tp.n_tiles), NT, sm, s>>>(p);
+    c->launches += 1;
+    KT_CUDA(cudaGetLastError());
+    return KT_OK;
+}
+
+int kt_cast(const void *in, int in_dtype, void *out, int out_dtype, int64_t n, void *stream) {
+    if (n < 0) return fail(KT_ERR_INVALID, "n is negative");
+    if (n == 0) return KT_OK;
+    if (!in || !out) return fail(KT_ERR_INVALID, "NULL argument");
+    if ((in_dtype != KT_F32 && in_dtype != KT_BF16) || (out_dtype != KT_F32 && out_dtype != KT_BF16))
+        return fail(KT_ERR_INVALID, "unknown dtype");
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (in_dtype == out_dtype) {
+        KT_CUDA(cudaMemcpyAsync(out, in, n * (in_dtype == KT_F32 ? 4 : 2), cudaMemcpyDeviceToDevice, s));
+        return KT_OK;
+    }
+    int dev = 0, sms = 0;
+    KT_CUDA(cudaGetDevice(&dev));
+    KT_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    long long blocks = (n + NT - 1) / NT;
+    const long long cap = static_cast<long long>(sms) * 8;
+    const int grid = static_cast<int>(blocks < cap ? blocks : cap);
+    if (in_dtype == KT_BF16)
+        k_cast_bf16_to_f32<<<grid, NT, 0, s>>>(static_cast<const unsigned short *>(in), static_cast<float *>(out), n);
+    else
+        k_cast_f32_to_bf16<<<grid, NT, 0, s>>>(static_cast<const float *>(in), static_cast<unsigned short *>(out), n);
+    KT_CUDA(cudaGetLastError());
+    return KT_OK;
+}
+
+int64_t kt_launch_count(const kt_ctx *c) { return c ? c->launches : 0; }
+
+const char *kt_last_error(const kt_ctx *) { return g_err; }
+
+void kt_destroy(kt_ctx *c) {
+    if (!c) return;
+    cudaSetDevice(c->device);
+    if (c->d_tables || c->d_out) cudaDeviceSynchronize();
+    if (c->d_tables) cudaFree(c->d_tables);
+    if (c->d_out) cudaFree(c->d_out);
+    if (c->ev_main) cudaEventDestroy(c->ev_main);
+    for (int dir = 0; dir < 2; ++dir)
+        for (auto &s : c->slots[dir])
+            if (s.done) cudaEventDestroy(s.done);
+    delete c;
+}
+
+}  // extern "C"

@@ -1,0 +1,110 @@
+"""No-GPU checks of the C-ABI library: it builds, loads, exports every symbol the header
+declares, and its pure host functions (scheduler, bucket plan, argument validation) agree
+with the oracle bit for bit."""
+import ctypes
+import os
+import random
+import re
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def kt():
+    from paper_2505_10183_b200 import build
+    build.build()
+    from paper_2505_10183_b200 import binding
+    return binding
+
+
+def declared_symbols():
+    text = open(os.path.join(ROOT, "include", "kaitian.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(kt_[a-z_]+)\s*\(", text)))
+
+
+def test_library_exports_every_declared_symbol(kt):
+    from paper_2505_10183_b200 import build
+    lib = ctypes.CDLL(build.LIB)
+    names = declared_symbols()
+    assert len(names) >= 15
+    for name in names:
+        assert hasattr(lib, name), name
+    assert sorted(kt.EXPORTS) == names          # the binding covers the same set
+    for name in names:
+        assert callable(getattr(kt, name)), name
+
+
+def test_schedule_bit_exact_against_oracle(kt, oracle):
+    rnd = random.Random(42)
+    for _ in range(2000):
+        K = rnd.randint(1, 64)
+        times = [rnd.choice([1.0, 1.4, 1.6, 2.1, rnd.uniform(0.05, 9.0)]) for _ in range(K)]
+        B = rnd.randint(K, 4096)
+        assert kt.kt_schedule(times, B) == oracle.schedule(times, B).tolist(), (times, B)
+    # tiny batches exercise the nobody-idles rule
+    for _ in range(500):
+        K = rnd.randint(2, 12)
+        times = [rnd.choice([1.0, 3.0, 50.0, 1000.0]) for _ in range(K)]
+        B = rnd.randint(K, K + 6)
+        assert kt.kt_schedule(times, B) == oracle.schedule(times, B).tolist(), (times, B)
+
+
+@pytest.mark.parametrize("times,B", [([1.0, 0.0], 8), ([1.0, -1.0], 8), ([1.0, float("nan")], 8),
+                                     ([1.0, float("inf")], 8), ([1.0] * 3, 2), ([], 4), ([1.0] * 65, 100)])
+def test_schedule_rejects_invalid(kt, times, B):
+    with pytest.raises(kt.KtError) as e:
+        kt.kt_schedule(times, B)
+    assert e.value.status == kt.KT_ERR_INVALID
+    assert kt.kt_last_error() != ""
+
+
+def test_plan_buckets_against_oracle(kt, oracle):
+    from paper_2505_10183_b200 import workloads as W
+    cases = [(W.tiny().numel, 25 << 20), (W.resnet18().numel, 25 << 20), (W.resnet50().numel, 25 << 20),
+             (W.mobilenet_v2().numel, 25 << 20), (W.mobilenet_v2().numel, 1 << 20), ([1 << 28], 1 << 62)]
+    rnd = random.Random(3)
+    for _ in range(300):
+        T = rnd.randint(1, 50)
+        cases.append(([rnd.choice([0, 1, 7, 8, 9, 63, 64, 65, 100, 1000, 4097, 70000]) for _ in range(T)],
+                      rnd.choice([4, 32, 256, 1000, 4096, 20000, 1 << 22, 1 << 40])))
+    for numel, cap in cases:
+        p = kt.kt_plan_buckets(numel, cap)
+        o = oracle.bucket_plan(numel, cap)
+        assert p.n_buckets == o.n_buckets
+        assert p.tensor_offset == o.tensor_offset.tolist()
+        assert p.bucket_of == o.bucket_of.tolist()
+        assert p.bucket_start == o.bucket_start.tolist()
+        assert p.bucket_numel == o.bucket_numel.tolist()
+        assert p.transport_numel == o.transport_numel
+
+
+def test_argument_validation_needs_no_device(kt):
+    E = kt.KtError
+    for args in (([0, 2], [1, 1], 3), ([0, 1], [1, 0], 2), ([0, -1], [1, 1], 2), ([0, 0], [1, 1], 3),
+                 ([], [], 0), ([0] * 65, [1] * 65, 1)):
+        with pytest.raises(E) as e:
+            kt.kt_groups_init(*args)
+        assert e.value.status == kt.KT_ERR_INVALID
+    with pytest.raises(E):
+        kt.kt_plan_buckets([4, -1], 1024)
+    with pytest.raises(E):
+        kt.kt_plan_buckets([4], 2)
+
+
+def test_missing_library_fails_loudly(tmp_path, monkeypatch):
+    """The product path has no fallback: without the built library the binding refuses to import."""
+    import importlib
+    import sys
+    from paper_2505_10183_b200 import build
+    monkeypatch.setattr(build, "LIB", str(tmp_path / "nope.so"))
+    saved = sys.modules.pop("paper_2505_10183_b200.binding", None)
+    try:
+        with pytest.raises(ImportError):
+            importlib.import_module("paper_2505_10183_b200.binding")
+    finally:
+        sys.modules.pop("paper_2505_10183_b200.binding", None)
+        if saved is not None:
+            sys.modules["paper_2505_10183_b200.binding"] = saved

@@ -1,0 +1,380 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the CPU oracle on the
+same seeded inputs.  Bars: bit-exact for pack / unpack / casts / shares / plan; for the
+reductions the kernels follow the oracle's operation order, so results are compared bit
+for bit as well, and the stated tolerances (1e-6 relative for fp32 sources, 1e-2 for
+bf16-sourced gradients) are checked against an fp64 weighted mean on top."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2505_10183_b200 import workloads as W
+
+import _harness as H
+
+pytestmark = pytest.mark.gpu
+
+F32, BF16 = 0, 1
+
+
+@pytest.fixture(scope="module")
+def kt():
+    if not torch.cuda.is_available():
+        pytest.fail("these tests need a CUDA device")
+    from paper_2505_10183_b200 import binding
+    torch.cuda.set_device(0)
+    return binding
+
+
+def compare_all(kt, oracle, wl, **kw):
+    shares = H.shares_of(wl, kt)
+    host, dev = H.device_gradients(wl, misalign=kw.pop("misalign", 0))
+    out, transport, plan, ctx = H.run_gpu_path(kt, wl, dev, shares, **kw)
+    o_out, o_parts, o_S, o_plan = H.run_oracle_path(
+        oracle, wl, host, shares, scale=kw.get("scale", 1.0),
+        out_dtype=None if kw.get("out_dtype") is None else {torch.float32: F32, torch.bfloat16: BF16}[kw["out_dtype"]])
+    # plan: integers, exact
+    assert plan.n_buckets == o_plan.n_buckets
+    assert plan.tensor_offset == o_plan.tensor_offset.tolist()
+    assert plan.bucket_of == o_plan.bucket_of.tolist()
+    assert plan.bucket_start == o_plan.bucket_start.tolist()
+    assert plan.bucket_numel == o_plan.bucket_numel.tolist()
+    assert plan.transport_numel == o_plan.transport_numel
+    # group partials incl. zero padding, then every output copy
+    for g in range(wl.G):
+        H.assert_bit_equal(transport[g], o_parts[g], "transport[%d]" % g)
+    for c in range(len(out)):
+        for t in range(wl.T):
+            H.assert_bit_equal(out[c][t], o_out[t], "out[%d][%d]" % (c, t))
+    kt.kt_destroy(ctx)
+    return host, out, shares
+
+
+def check_tolerance(oracle, wl, host, out, shares):
+    """Stated tolerance against the fp64 weighted mean, forward-error denominator."""
+    dt = H.ORACLE_DT[wl.dtype]
+    xs = [np.concatenate(h) for h in host]
+    F, absF = oracle.flat_reduce_f64(xs, dt, shares)
+    got = np.concatenate([W.as_numpy(t) for t in out[0]])
+    if got.dtype == np.uint16:
+        got = oracle.bf16_to_f32(got)
+        tol = 1e-2
+    else:
+        tol = 1e-6
+    nz = absF > 0
+    assert np.max(np.abs(got[nz] - F[nz]) / absF[nz]) <= tol
+
+
+# ------------------------------------------------------------------ the named configurations
+def test_tiny(kt, oracle):
+    wl = W.tiny()
+    host, out, shares = compare_all(kt, oracle, wl)
+    check_tolerance(oracle, wl, host, out, shares)
+
+
+def test_schedule_matches_oracle_and_named_values(kt, oracle):
+    assert kt.kt_schedule([1.0, 1.0, 1.6, 1.6], 256) == [79, 79, 49, 49]
+    assert kt.kt_schedule([1.0] * 4 + [1.4] * 2 + [2.1] * 2, 256) == [40, 40, 40, 40, 29, 29, 19, 19]
+    rng = np.random.default_rng(0)
+    for _ in range(500):
+        K = int(rng.integers(1, 17))
+        times = rng.uniform(0.2, 5.0, size=K).tolist()
+        B = int(rng.integers(K, 2048))
+        assert kt.kt_schedule(times, B) == oracle.schedule(times, B).tolist()
+
+
+def test_resnet18_staged_as_benchmarked(kt, oracle):
+    """Full size, bucket by bucket, partials relayed through pinned host memory: the launch
+    configuration the benchmark times."""
+    wl = W.resnet18()
+    host, out, shares = compare_all(kt, oracle, wl, per_bucket=True, staged=True)
+    assert shares == [79, 79, 49, 49]
+    check_tolerance(oracle, wl, host, out, shares)
+
+
+def test_resnet18_single_launch(kt, oracle):
+    compare_all(kt, oracle, W.resnet18())
+
+
+def test_resnet50_bf16(kt, oracle):
+    wl = W.resnet50()
+    host, out, shares = compare_all(kt, oracle, wl, per_bucket=True)
+    check_tolerance(oracle, wl, host, out, shares)
+    # fp32 output of bf16 sources: 1e-6-class accuracy is kept by the fp32 accumulation
+    host, out, shares = compare_all(kt, oracle, wl, out_dtype=torch.float32)
+    dt = H.ORACLE_DT[wl.dtype]
+    F, absF = oracle.flat_reduce_f64([np.concatenate(h) for h in host], dt, shares)
+    got = np.concatenate([W.as_numpy(t) for t in out[0]])
+    assert np.max(np.abs(got - F) / absF) <= 1e-6
+
+
+def test_mobilenet_v2_ragged(kt, oracle):
+    wl = W.mobilenet_v2()
+    host, out, shares = compare_all(kt, oracle, wl)
+    assert shares == [40, 40, 40, 40, 29, 29, 19, 19]
+    check_tolerance(oracle, wl, host, out, shares)
+
+
+@pytest.mark.parametrize("K", [2, 4, 8, 16])
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("nbytes", [4 << 10, 64 << 10, 1 << 20, 16 << 20])
+def test_sweep_small_points(kt, oracle, K, dtype, nbytes):
+    if nbytes == 16 << 20 and K == 16 and dtype == "bf16":
+        pytest.skip("covered by the fp32 point of the same size")
+    compare_all(kt, oracle, W.sweep_point(K, nbytes, dtype))
+
+
+def test_sweep_large_point_sampled_windows(kt, oracle):
+    """1 GiB per rank, K = 4: device-generated values; 2^20-element windows are copied to
+    the host and checked element by element (the path is element-wise, so a window's
+    result depends on that window's inputs only)."""
+    wl = W.sweep_point(4, 1 << 30, "f32")
+    shares = wl.shares
+    n = wl.N
+    dev = [[W.rank_gradients(wl, r, "cuda")] for r in range(wl.K)]
+    ctx = kt.kt_groups_init(wl.group_of, shares, wl.G)
+    kt.kt_bucket_pack(ctx, dev, wl.bucket_cap_bytes)
+    plan = kt.kt_plan_query(ctx)
+    assert plan.transport_numel == n and plan.n_buckets == 1
+    transport = [torch.empty(n, device="cuda") for _ in range(wl.G)]
+    out = [[torch.empty(n, device="cuda")]]
+    kt.kt_hier_reduce(ctx, kt.KT_INTRA, transport)
+    kt.kt_unpack_scale(ctx, transport, out)
+    torch.cuda.synchronize()
+    win = 1 << 20
+    rng = np.random.default_rng(5)
+    starts = [0, n - win] + (rng.integers(0, n // win - 1, size=6) * win + 12345).tolist()
+    for s in starts:
+        s = int(min(max(s, 0), n - win))
+        hx = [[W.as_numpy(dev[r][0][s:s + win])] for r in range(wl.K)]
+        o_out, o_parts, _, _ = oracle.sync_step(hx, [win], F32, wl.group_of, shares, wl.G, 1 << 62)
+        for g in range(wl.G):
+            H.assert_bit_equal(transport[g][s:s + win], o_parts[g], "window %d transport[%d]" % (s, g))
+        H.assert_bit_equal(out[0][0][s:s + win], o_out[0], "window %d out" % s)
+    kt.kt_destroy(ctx)
+
+
+# ------------------------------------------------------------------ variants and edge cases
+def test_misaligned_sources_take_the_element_path(kt, oracle):
+    for wl in (W.tiny(), W.sweep_point(4, 1 << 20, "bf16"), W.sweep_point(2, 1 << 20, "f32")):
+        compare_all(kt, oracle, wl, misalign=1)
+        compare_all(kt, oracle, wl, misalign=3)
+
+
+def test_broadcast_copies_and_scale(kt, oracle):
+    wl = W.tiny()
+    compare_all(kt, oracle, wl, R=wl.K, scale=0.125)
+    wl = W.mobilenet_v2()
+    compare_all(kt, oracle, wl, R=3, scale=1.0 / 3.0)
+
+
+def test_combined_buffer_route(kt, oracle):
+    compare_all(kt, oracle, W.tiny(), use_combined=True)
+    compare_all(kt, oracle, W.resnet18(), use_combined=True, per_bucket=True)
+
+
+def test_bf16_out_from_f32_sources_and_back(kt, oracle):
+    compare_all(kt, oracle, W.tiny(), out_dtype=torch.bfloat16)
+    compare_all(kt, oracle, W.sweep_point(4, 1 << 20, "bf16"), out_dtype=torch.float32)
+
+
+def test_empty_and_odd_tensors(kt, oracle):
+    wl = W.Workload("odd", 7, [(0,), (1,), (7,), (2049,), (0,), (4096,), (13,)], "f32",
+                    [0, 1, 1, 2, 0], [3, 5, 7, 11, 13], bucket_cap_bytes=5000 * 4)
+    compare_all(kt, oracle, wl)
+    compare_all(kt, oracle, wl, per_bucket=True, R=2)
+    wl.dtype = "bf16"
+    compare_all(kt, oracle, wl)
+
+
+def test_single_rank_and_singleton_groups(kt, oracle):
+    wl = W.Workload("one", 8, [(5000,)], "f32", [0], [7])
+    host, out, _ = compare_all(kt, oracle, wl)
+    assert np.array_equal(W.as_numpy(out[0][0]), host[0][0])          # K = 1: identity
+    wl = W.Workload("singletons", 9, [(3000,), (17,)], "f32", [0, 1, 2, 3, 4], [5, 9, 17, 3, 30])
+    compare_all(kt, oracle, wl)
+
+
+def test_identical_ranks_and_equal_shares(kt, oracle):
+    wl = W.tiny()
+    flat = W.rank_gradients(wl, 0, "cpu")
+    dev = [[t.cuda() for t in W.split_tensors(flat, wl.numel)] for _ in range(4)]
+    out, *_ = H.run_gpu_path(kt, wl, dev, [64, 64, 64, 64])
+    for t, ref in zip(out[0], W.split_tensors(flat, wl.numel)):
+        assert torch.equal(t.cpu(), ref)                               # exact: all weights are powers of two
+    # equal shares: arithmetic mean
+    host, dev = H.device_gradients(wl)
+    out, *_ = H.run_gpu_path(kt, wl, dev, [32] * 4)
+    stack = np.stack([np.concatenate(h).astype(np.float64) for h in host])
+    got = np.concatenate([W.as_numpy(t) for t in out[0]])
+    assert np.max(np.abs(got - stack.mean(0)) / np.abs(stack).mean(0)) < 1e-6
+
+
+def test_sum_then_divide_coefficients(kt, oracle):
+    """Plain sums across the hierarchy with one final division (weights a_r = b_r, W_g = 1,
+    scale 1/B) through kt_set_coefficients; oracle fed the same coefficients."""
+    wl = W.tiny()
+    shares = wl.shares
+    host, dev = H.device_gradients(wl)
+    ctx = kt.kt_groups_init(wl.group_of, shares, wl.G)
+    kt.kt_set_coefficients(ctx, [float(b) for b in shares], [1.0] * wl.G)
+    a, Wg = kt.kt_get_coefficients(ctx)
+    assert a == [float(b) for b in shares] and Wg == [1.0] * wl.G
+    kt.kt_bucket_pack(ctx, dev, wl.bucket_cap_bytes)
+    plan = kt.kt_plan_query(ctx)
+    tr = [torch.empty(plan.transport_numel, device="cuda") for _ in range(wl.G)]
+    out = [[torch.empty(m, device="cuda") for m in wl.numel]]
+    kt.kt_hier_reduce(ctx, kt.KT_INTRA, tr)
+    kt.kt_unpack_scale(ctx, tr, out, scale=1.0 / sum(shares))
+    torch.cuda.synchronize()
+    oplan = oracle.bucket_plan(wl.numel, wl.bucket_cap_bytes)
+    parts = oracle.intra_reduce(host, oplan, F32, wl.group_of, np.array(shares, np.float32), wl.G)
+    S = oracle.combine(parts, np.ones(wl.G, np.float32))
+    want = oracle.unpack_scale(S, oplan, np.float32(1.0 / sum(shares)), F32)
+    for t in range(wl.T):
+        H.assert_bit_equal(out[0][t], want[t])
+    # and switching back to share-derived weights
+    kt.kt_set_shares(ctx, shares)
+    a, Wg = kt.kt_get_coefficients(ctx)
+    oa, oW, _ = oracle.coefficients(wl.group_of, shares, wl.G)
+    assert a == oa.tolist() and Wg == oW.tolist()
+    kt.kt_destroy(ctx)
+
+
+def test_standalone_pack(kt, oracle):
+    for wl in (W.tiny(), W.mobilenet_v2()):
+        for dtype in ("f32", "bf16"):
+            wl.dtype = dtype
+            host, dev = H.device_gradients(wl)
+            ctx = kt.kt_groups_init(wl.group_of, H.shares_of(wl, kt), wl.G)
+            n = kt.kt_plan_buckets(wl.numel, wl.bucket_cap_bytes).transport_numel
+            flat = [torch.full((n,), 1.0, dtype=H.TORCH_DT[dtype], device="cuda") for _ in range(wl.K)]
+            kt.kt_bucket_pack(ctx, dev, wl.bucket_cap_bytes, flat_out=flat)
+            torch.cuda.synchronize()
+            oplan = oracle.bucket_plan(wl.numel, wl.bucket_cap_bytes)
+            for r in range(wl.K):
+                H.assert_bit_equal(flat[r], oracle.pack(host[r], oplan, H.ORACLE_DT[dtype]), "flat[%d]" % r)
+            kt.kt_destroy(ctx)
+
+
+def test_cast_kernels_exhaustive(kt, oracle):
+    # bf16 -> fp32: all 65 536 patterns
+    h = torch.arange(65536, dtype=torch.int32).to(torch.int16).view(torch.bfloat16).cuda()
+    f = torch.empty(65536, device="cuda")
+    kt.kt_cast(h, f)
+    want = oracle.bf16_to_f32(np.arange(65536, dtype=np.uint16))
+    got = f.cpu().numpy()
+    assert np.array_equal(got.view(np.uint32), want.view(np.uint32))
+    # fp32 -> bf16: all 2^32 patterns, 2^26 at a time
+    chunk = 1 << 26
+    base = torch.arange(chunk, dtype=torch.int64, device="cuda")
+    out = torch.empty(chunk, dtype=torch.bfloat16, device="cuda")
+    from concurrent.futures import ThreadPoolExecutor
+    pool = ThreadPoolExecutor(8)
+    for c in range(64):
+        bits = (base + c * chunk).to(torch.int32).contiguous()      # wraps to the signed pattern
+        kt.kt_cast(bits.view(torch.float32), out)
+        got = out.view(torch.int16).cpu().numpy().view(np.uint16)
+        fb = bits.cpu().numpy().view(np.float32)
+        parts = list(pool.map(oracle.f32_to_bf16, np.array_split(fb, 8)))
+        want = np.concatenate(parts)
+        nan = np.isnan(fb)
+        assert np.array_equal(got[~nan], want[~nan]), "chunk %d" % c
+        if nan.any():
+            assert np.all(np.isnan(oracle.bf16_to_f32(got[nan])))
+    pool.shutdown()
+
+
+# ------------------------------------------------------------------ staging
+def test_staging_bytes_and_ordering(kt, oracle):
+    """Host bytes equal the device partials; the copy never starts before the reduce that
+    feeds it has finished (the transport is poisoned right before the reduce is queued)."""
+    wl = W.resnet18()
+    shares = H.shares_of(wl, kt)
+    host_g, dev = H.device_gradients(wl)
+    ctx = kt.kt_groups_init(wl.group_of, shares, wl.G)
+    kt.kt_bucket_pack(ctx, dev, wl.bucket_cap_bytes)
+    plan = kt.kt_plan_query(ctx)
+    n = plan.transport_numel
+    tr = [torch.empty(n, device="cuda") for _ in range(wl.G)]
+    pinned = [torch.zeros(n).pin_memory() for _ in range(wl.G)]
+    side = torch.cuda.Stream()
+    poison = float(np.float32(-7.25e33))
+    for _ in range(3):
+        for t in tr:
+            t.fill_(poison)
+        kt.kt_hier_reduce(ctx, kt.KT_INTRA, tr)
+        kt.kt_stage_to_host(ctx, kt.KT_D2H, tr, pinned, side_stream=side)
+        kt.kt_stage_wait(ctx, kt.KT_D2H, timeout_ms=20000)
+        for g in range(wl.G):
+            assert not (pinned[g] == poison).any()
+            assert torch.equal(pinned[g], tr[g].cpu())
+    _, o_parts, _, _ = H.run_oracle_path(oracle, wl, host_g, shares)
+    for g in range(wl.G):
+        H.assert_bit_equal(pinned[g], o_parts[g])
+    kt.kt_destroy(ctx)
+
+
+# ------------------------------------------------------------------ error paths
+def test_error_codes(kt):
+    E = kt.KtError
+    with pytest.raises(E) as e:
+        kt.kt_groups_init([0, 2], [1, 1], 3)
+    assert e.value.status == kt.KT_ERR_INVALID
+    with pytest.raises(E):
+        kt.kt_groups_init([0, 1], [1, 0])
+    ctx = kt.kt_groups_init([0, 0, 1], [1, 2, 3])
+    tr = [torch.empty(64, device="cuda") for _ in range(2)]
+    with pytest.raises(E) as e:
+        kt.kt_hier_reduce(ctx, kt.KT_INTRA, tr)
+    assert e.value.status == kt.KT_ERR_STATE
+    g = [[torch.zeros(100, device="cuda")] for _ in range(3)]
+    kt.kt_bucket_pack(ctx, g, 1 << 20)
+    plan = kt.kt_plan_query(ctx)
+    assert plan.transport_numel == 128
+    tr = [torch.empty(128, device="cuda") for _ in range(2)]
+    with pytest.raises(E) as e:
+        kt.kt_hier_reduce(ctx, kt.KT_INTRA, tr, bucket=1)
+    assert e.value.status == kt.KT_ERR_SHAPE
+    with pytest.raises(E) as e:
+        kt.kt_hier_reduce(ctx, kt.KT_INTER, tr, None)
+    assert e.value.status == kt.KT_ERR_INVALID
+    with pytest.raises(E) as e:
+        kt.kt_hier_reduce(ctx, 7, tr)
+    assert e.value.status == kt.KT_ERR_INVALID
+    odd = torch.empty(132, device="cuda")[1:129]
+    with pytest.raises(E) as e:
+        kt.kt_hier_reduce(ctx, kt.KT_INTRA, [odd, tr[1]])
+    assert e.value.status == kt.KT_ERR_ALIGN
+    with pytest.raises(E) as e:
+        kt.kt_stage_wait(ctx, kt.KT_D2H)
+    assert e.value.status == kt.KT_ERR_STATE
+    with pytest.raises(E) as e:
+        kt.kt_unpack_scale(ctx, tr, [[torch.empty(100, device="cuda")] for _ in range(4)])
+    assert e.value.status == kt.KT_ERR_SHAPE
+    assert "R = 4" in kt.kt_last_error()
+    # the context stays usable after errors
+    kt.kt_hier_reduce(ctx, kt.KT_INTRA, tr)
+    torch.cuda.synchronize()
+    assert kt.kt_launch_count(ctx) == 1
+    kt.kt_destroy(ctx)
+    kt.kt_destroy(ctx)      # idempotent
+
+
+def test_stage_wait_deadline_returns_timeout_status(kt):
+    """A wait whose deadline passes returns KT_ERR_TIMEOUT to the host and leaves the
+    context usable; nothing on the device is interrupted."""
+    n = 1 << 28                                   # 1 GiB per buffer: tens of milliseconds on the host link
+    ctx = kt.kt_groups_init([0, 1], [1, 1])
+    g = [[torch.zeros(n, device="cuda")] for _ in range(2)]
+    kt.kt_bucket_pack(ctx, g, 1 << 62)
+    tr = [torch.ones(n, device="cuda") for _ in range(2)]
+    pinned = [torch.zeros(n).pin_memory() for _ in range(2)]
+    side = torch.cuda.Stream()
+    torch.cuda.synchronize()
+    kt.kt_stage_to_host(ctx, kt.KT_D2H, tr, pinned, side_stream=side)
+    with pytest.raises(kt.KtError) as e:
+        kt.kt_stage_wait(ctx, kt.KT_D2H, timeout_ms=0)
+    assert e.value.status == kt.KT_ERR_TIMEOUT
+    kt.kt_stage_wait(ctx, kt.KT_D2H, timeout_ms=60000)    # now it completes
+    assert float(pinned[1][-1]) == 1.0
+    kt.kt_destroy(ctx)
