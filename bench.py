@@ -1,0 +1,461 @@
+#!/usr/bin/env python
+"""Benchmark of the hierarchical, load-weighted gradient synchronisation step.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload resnet18] [--impl ours|reference]
+    python bench.py --sweep            # bucket-size sweep of the fused reduce, one JSON line per point
+
+One step = one pass of the whole path over one batch of synthetic gradients that already
+sit in device memory: per bucket the fused pack+widen+weighted intra-group reduce, the relay
+of the fp32 group partials through pinned host memory (when the workload says so), then the
+inter-group combine + scale + unpack into per-parameter gradients.  Prints ONE JSON line.
+
+The default workload is ResNet-18 (10-class head), fp32, K = 4 ranks in 2 groups, shares
+from kt_schedule(1, 1, 1.6, 1.6; 256), 25 MiB buckets, partials staged through pinned host
+memory.  With N > 1 every GPU runs an independent replica of the same problem (the path
+has no exchange between GPUs); the value is the sum over replicas divided by the slowest.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import torch  # noqa: E402
+
+from paper_2505_10183_b200 import workloads as W  # noqa: E402
+
+METRIC = "hierarchical weighted grad-reduce throughput"
+UNIT = "GB/s"
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+
+
+# ----------------------------------------------------------------------------- helpers
+def algorithmic_bytes(wl) -> dict:
+    """Bytes the method must move per step (N = gradient elements per rank)."""
+    N, K, G, s = wl.N, wl.K, wl.G, wl.elem_size
+    k1 = K * N * s + G * N * 4          # read every gradient once, write G fp32 partials
+    k2 = G * N * 4 + N * s              # read G partials, write the result once
+    return {"k1": k1, "k2": k2, "step": k1 + k2, "stage_each_way": G * N * 4 if wl.staged else 0}
+
+
+def measured_peak() -> tuple:
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.proc = None
+        self.file = None
+
+    def start(self):
+        try:
+            self.file = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.FIELDS,
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=self.file, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self) -> dict:
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        self.file.flush()
+        self.file.seek(0)
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.file.read().splitlines():
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                mx.append(float(parts[1]))
+            except ValueError:
+                continue
+            for name, val in zip(names, parts[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        self.file.close()
+        os.unlink(self.file.name)
+        if sm:
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), reasons=sorted(reasons),
+                       samples=len(sm))
+        return out
+
+
+# ----------------------------------------------------------------------------- our arm
+class Problem:
+    """Device state of one replica: gradients, context, transport / receive / pinned buffers."""
+
+    def __init__(self, wl, kt, device_values: bool = True):
+        self.wl, self.kt = wl, kt
+        self.shares = list(wl.shares) if wl.shares is not None else kt.kt_schedule(wl.step_times, wl.global_batch)
+        dt = torch.float32 if wl.dtype == "f32" else torch.bfloat16
+        self.grads = []
+        for r in range(wl.K):
+            flat = W.rank_gradients(wl, r, "cuda" if device_values else "cpu")
+            self.grads.append([t.cuda() for t in W.split_tensors(flat, wl.numel)])
+            del flat
+        self.ctx = kt.kt_groups_init(wl.group_of, self.shares, wl.G)
+        kt.kt_bucket_pack(self.ctx, self.grads, wl.bucket_cap_bytes)
+        self.plan = kt.kt_plan_query(self.ctx)
+        n = self.plan.transport_numel
+        self.transport = kt.kt_ptrs([torch.zeros(n, device="cuda") for _ in range(wl.G)])
+        self.out = [[torch.zeros(m, dtype=dt, device="cuda") for m in wl.numel]]
+        self.out_ptrs = kt.kt_ptrs([t for c in self.out for t in c])
+        self.out_dtype = kt.KT_F32 if wl.dtype == "f32" else kt.KT_BF16
+        self.main = torch.cuda.Stream()
+        if wl.staged:
+            self.recv = kt.kt_ptrs([torch.zeros(n, device="cuda") for _ in range(wl.G)])
+            self.pinned = kt.kt_ptrs([torch.zeros(n).pin_memory() for _ in range(wl.G)])
+            self.side_d2h = torch.cuda.Stream()
+            self.side_h2d = torch.cuda.Stream()
+        self.k1_events = []
+
+    def step(self, time_k1: bool = False):
+        kt, ctx, wl = self.kt, self.ctx, self.wl
+        nb = self.plan.n_buckets
+        for b in range(nb):
+            if time_k1:
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record(self.main)
+            kt.kt_hier_reduce(ctx, kt.KT_INTRA, self.transport, bucket=b, stream=self.main)
+            if time_k1:
+                e1.record(self.main)
+                self.k1_events.append((e0, e1))
+            if wl.staged:
+                kt.kt_stage_to_host(ctx, kt.KT_D2H, self.transport, self.pinned, bucket=b,
+                                    main_stream=self.main, side_stream=self.side_d2h)
+                kt.kt_stage_to_host(ctx, kt.KT_H2D, self.recv, self.pinned, bucket=b,
+                                    main_stream=self.main, side_stream=self.side_h2d)
+        src = self.recv if wl.staged else self.transport
+        for b in range(nb):
+            if wl.staged:
+                kt.kt_stage_wait(ctx, kt.KT_H2D, bucket=b, main_stream=self.main)
+            kt.kt_unpack_scale(ctx, src, self.out_ptrs, scale=1.0, bucket=b, out_dtype=self.out_dtype,
+                               R=1, stream=self.main)
+
+    def k1_seconds(self) -> float:
+        return sum(a.elapsed_time(b) for a, b in self.k1_events) * 1e-3
+
+
+def host_link_bandwidth(nbytes: int = 256 << 20, reps: int = 10) -> dict:
+    """Pinned cudaMemcpyAsync both ways, best of `reps` (GB/s)."""
+    dev = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+    host = torch.empty(nbytes, dtype=torch.uint8).pin_memory()
+    best = {"d2h": 0.0, "h2d": 0.0}
+    for _ in range(reps):
+        for name, (dst, src) in (("d2h", (host, dev)), ("h2d", (dev, host))):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            dst.copy_(src, non_blocking=True)
+            b.record()
+            b.synchronize()
+            best[name] = max(best[name], nbytes / (a.elapsed_time(b) * 1e-3) / 1e9)
+    return best
+
+
+def run_ours(args) -> dict:
+    from paper_2505_10183_b200 import binding as kt
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+
+    wl = W.by_name(args.workload)
+    prob = Problem(wl, kt)
+    nbytes = algorithmic_bytes(wl)
+    link = host_link_bandwidth() if wl.staged else None
+
+    def barrier():
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    with torch.cuda.stream(prob.main):
+        for _ in range(args.warmup):
+            prob.step()
+        barrier()
+        sampler = ClockSampler(local)
+        if rank == 0:
+            sampler.start()
+        launches0 = kt.kt_launch_count(prob.ctx)
+        t_start, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        marks = []
+        t_start.record(prob.main)
+        for _ in range(args.steps):
+            prob.step(time_k1=True)
+            m = torch.cuda.Event(enable_timing=True)
+            m.record(prob.main)
+            marks.append(m)
+        t_end.record(prob.main)
+        barrier()
+        clocks = sampler.stop() if rank == 0 else None
+        launches = kt.kt_launch_count(prob.ctx) - launches0
+        total_s = t_start.elapsed_time(t_end) * 1e-3
+        per_step = [a.elapsed_time(b) for a, b in zip([t_start] + marks[:-1], marks)]
+        k1_s = prob.k1_seconds()
+
+        # end to end: gradients start in pinned host memory, the result ends there
+        e2e = run_e2e(prob, kt, args, barrier)
+
+    if dist is not None:
+        t = torch.tensor([total_s, e2e["seconds"]], device="cuda", dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_s, e2e["seconds"] = float(t[0]), float(t[1])
+
+    peak, peak_kind = measured_peak()
+    k1_launch_bytes = nbytes["k1"] / prob.plan.n_buckets          # average per launch
+    k1_launch_s = k1_s / (args.steps * prob.plan.n_buckets)
+    achieved = k1_launch_bytes / k1_launch_s / 1e9
+    value = world * nbytes["step"] * args.steps / total_s / 1e9
+    result = {
+        "metric": METRIC, "value": round(value, 2), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": round(total_s / args.steps * 1e3, 4),
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": wl.dtype,
+        "data": "synthetic",
+        "config": {
+            "workload": "%s: %d tensors, %d elements per rank, K=%d ranks in %d groups, shares %s, "
+                        "%d buckets of <= 25 MiB%s" % (wl.name, wl.T, wl.N, wl.K, wl.G, prob.shares,
+                                                      prob.plan.n_buckets,
+                                                      ", fp32 partials relayed through pinned host memory"
+                                                      if wl.staged else ""),
+            "bytes_per_step": nbytes["step"],
+            "bytes_counted": "algorithmic HBM bytes of the two kernels (K*N*s + 4*G*N read/written by the "
+                             "fused reduce, 4*G*N + N*s by combine+unpack); staging copies add time, not bytes",
+            "staging_bytes_each_way": nbytes["stage_each_way"],
+            "l2": "inputs (%.0f MB) exceed the 126 MB L2 and every step streams all buffers through it"
+                  % (wl.K * wl.N * wl.elem_size / 1e6),
+            "multi_gpu": "independent replicas, no collective",
+            "latency_ms": {"p50": round(statistics.median(per_step), 4),
+                           "p95": round(sorted(per_step)[int(0.95 * (len(per_step) - 1))], 4)},
+        },
+        "roofline": {"bound": "hbm", "kernel": "k1_intra_reduce", "achieved": round(achieved, 1),
+                     "peak": peak, "unit": "GB/s", "frac": round(achieved / peak, 4),
+                     "peak_kind": peak_kind, "frac_of_nominal_8TBs": round(achieved / NOMINAL_HBM_GBS, 4),
+                     "bytes_per_launch": int(k1_launch_bytes), "us_per_launch": round(k1_launch_s * 1e6, 2),
+                     "traffic": TRAFFIC_K1.get(wl.name)},
+        "e2e": {"value": round(world * nbytes["step"] * args.steps / e2e["seconds"] / 1e9, 2), "unit": UNIT,
+                "h2d_bytes_per_step": e2e["h2d"], "d2h_bytes_per_step": e2e["d2h"],
+                "ms_per_step": round(e2e["seconds"] / args.steps * 1e3, 4)},
+        "gpu_launches": int(launches),
+        "clocks": clocks,
+    }
+    if link is not None:
+        result["host_link"] = {"d2h_GBps": round(link["d2h"], 1), "h2d_GBps": round(link["h2d"], 1),
+                               "how": "pinned copy of 256 MiB, best of 10"}
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        result["cpu_baseline"] = cpu_baseline(wl, prob.shares, budget_s=args.cpu_seconds)
+    if dist is not None:
+        dist.destroy_process_group()
+    return result if rank == 0 else None
+
+
+# ncu dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel; null
+# until captured for the kernel as it stands (see profiles/).
+TRAFFIC_K1 = {}
+
+
+def run_e2e(prob, kt, args, barrier) -> dict:
+    """Same step, but every step first copies all ranks' gradients from pinned host memory
+    to the device and ends with the reduced gradients copied back to pinned host memory."""
+    wl = prob.wl
+    host_in = [[t.cpu().pin_memory() for t in row] for row in prob.grads]
+    host_out = [torch.empty(t.shape, dtype=t.dtype).pin_memory() for t in prob.out[0]]
+    dst = kt.kt_ptrs([t for row in prob.grads for t in row])
+    src = kt.kt_ptrs([t for row in host_in for t in row])
+    import ctypes
+    sizes = [t.numel() * t.element_size() for row in prob.grads for t in row]
+    sizes_c = (ctypes.c_int64 * len(sizes))(*sizes)
+    o_dst = kt.kt_ptrs(host_out)
+    o_src = kt.kt_ptrs(prob.out[0])
+    o_sizes = [t.numel() * t.element_size() for t in prob.out[0]]
+    o_sizes_c = (ctypes.c_int64 * len(o_sizes))(*o_sizes)
+
+    def one():
+        kt.kt_copy_tensors(dst, src, sizes_c, kt.KT_H2D, stream=prob.main)
+        prob.step()
+        kt.kt_copy_tensors(o_dst, o_src, o_sizes_c, kt.KT_D2H, stream=prob.main)
+
+    for _ in range(max(1, min(args.warmup, 3))):
+        one()
+    barrier()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record(prob.main)
+    for _ in range(args.steps):
+        one()
+    b.record(prob.main)
+    barrier()
+    return {"seconds": a.elapsed_time(b) * 1e-3, "h2d": sum(sizes), "d2h": sum(o_sizes)}
+
+
+# ----------------------------------------------------------------------------- the oracle as CPU baseline
+def oracle_inputs(wl):
+    host = []
+    for r in range(wl.K):
+        flat = W.rank_gradients(wl, r, "cpu")
+        host.append([W.as_numpy(t) for t in W.split_tensors(flat, wl.numel)])
+    return host
+
+
+def cpu_baseline(wl, shares, budget_s: float = 12.0) -> dict:
+    """The oracle as it stands, one thread, on the full workload, repeated for about
+    budget_s seconds; GB/s over the same algorithmic bytes as the GPU path."""
+    from oracle import kt_oracle as oracle
+    host = oracle_inputs(wl)
+    dt = 0 if wl.dtype == "f32" else 1
+    nbytes = algorithmic_bytes(wl)["step"]
+    oracle.sync_step(host, wl.numel, dt, wl.group_of, shares, wl.G, wl.bucket_cap_bytes)   # warm
+    times = []
+    t_all = time.perf_counter()
+    while time.perf_counter() - t_all < budget_s or len(times) < 2:
+        t0 = time.perf_counter()
+        oracle.sync_step(host, wl.numel, dt, wl.group_of, shares, wl.G, wl.bucket_cap_bytes)
+        times.append(time.perf_counter() - t0)
+    best = statistics.median(times)
+    return {"value": round(nbytes / best / 1e9, 3), "unit": UNIT, "cores": 1, "kind": "oracle",
+            "sample": "full %s step (all %d elements x %d ranks), %d repetitions, median" %
+                      (wl.name, wl.N, wl.K, len(times)),
+            "ms_per_step": round(best * 1e3, 2), "host_cores_available": os.cpu_count()}
+
+
+def run_reference(args) -> dict:
+    """The reference arm: the CPU oracle, unmodified, on the machine's host cores."""
+    if int(os.environ.get("RANK", "0")) != 0:
+        return None
+    from oracle import kt_oracle as oracle
+    wl = W.by_name(args.workload)
+    shares = list(wl.shares) if wl.shares is not None else oracle.schedule(wl.step_times, wl.global_batch).tolist()
+    host = oracle_inputs(wl)
+    dt = 0 if wl.dtype == "f32" else 1
+    nbytes = algorithmic_bytes(wl)["step"]
+    for _ in range(args.warmup):
+        oracle.sync_step(host, wl.numel, dt, wl.group_of, shares, wl.G, wl.bucket_cap_bytes)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle.sync_step(host, wl.numel, dt, wl.group_of, shares, wl.G, wl.bucket_cap_bytes)
+    total = time.perf_counter() - t0
+    value = round(nbytes * args.steps / total / 1e9, 3)
+    sample = "full %s step on one host thread, host-resident inputs" % wl.name
+    return {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT,
+        "n_gpus": int(os.environ.get("WORLD_SIZE", "1")), "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": round(total / args.steps * 1e3, 3), "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": wl.dtype, "data": "synthetic",
+        "config": {"workload": "%s: %d tensors, %d elements per rank, K=%d ranks in %d groups, shares %s"
+                               % (wl.name, wl.T, wl.N, wl.K, wl.G, shares), "bytes_per_step": nbytes},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+
+
+# ----------------------------------------------------------------------------- bucket sweep
+def run_sweep(args) -> None:
+    """Fused reduce (K1) and combine+unpack (K2) alone on flat buffers, 4 KB .. 1 GB per rank.
+    Buffers that fit the L2 are rotated over enough copies to exceed it."""
+    from paper_2505_10183_b200 import binding as kt
+    torch.cuda.set_device(0)
+    peak, peak_kind = measured_peak()
+    l2 = 126 << 20
+    sizes = [4 << 10 << (2 * i) for i in range(10)]
+    for dtype in ("f32", "bf16"):
+        for K in (2, 4, 8, 16):
+            for nb in sizes:
+                if args.sweep_max_bytes and nb > args.sweep_max_bytes:
+                    continue
+                wl = W.sweep_point(K, nb, dtype)
+                by = algorithmic_bytes(wl)
+                foot = by["k1"] + wl.N * wl.elem_size
+                copies = max(1, min(64, -(-2 * l2 // foot)))
+                probs = [Problem(wl, kt) for _ in range(copies)]
+                main = torch.cuda.Stream()
+                reps = max(5, min(200, int(2e9 // max(by["k1"], 1))))
+                res = {}
+                with torch.cuda.stream(main):
+                    for name in ("k1", "k2"):
+                        def launch(p):
+                            if name == "k1":
+                                kt.kt_hier_reduce(p.ctx, kt.KT_INTRA, p.transport, stream=main)
+                            else:
+                                kt.kt_unpack_scale(p.ctx, p.transport, p.out_ptrs, out_dtype=p.out_dtype, R=1,
+                                                   stream=main)
+                        for i in range(3 * copies):
+                            launch(probs[i % copies])
+                        torch.cuda.synchronize()
+                        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                        a.record(main)
+                        for i in range(reps):
+                            launch(probs[i % copies])
+                        b.record(main)
+                        torch.cuda.synchronize()
+                        us = a.elapsed_time(b) * 1e3 / reps
+                        res[name] = {"us": round(us, 2), "GBps": round(by[name] / us / 1e3, 1),
+                                     "frac": round(by[name] / us / 1e3 / peak, 4)}
+                print(json.dumps({"sweep": wl.name, "K": K, "dtype": dtype, "bytes_per_rank": nb,
+                                  "shares": wl.shares, "rotated_copies": copies, "peak": peak,
+                                  "peak_kind": peak_kind, **res}), flush=True)
+                for p in probs:
+                    kt.kt_destroy(p.ctx)
+                del probs
+                torch.cuda.empty_cache()
+
+
+def main() -> None:
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="resnet18", choices=["tiny", "resnet18", "resnet50", "mobilenet_v2"])
+    ap.add_argument("--sweep", action="store_true")
+    ap.add_argument("--sweep-max-bytes", type=int, default=0)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--cpu-seconds", type=float, default=12.0)
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.sweep:
+        run_sweep(args)
+        return
+    out = run_reference(args) if args.impl == "reference" else run_ours(args)
+    if out is not None:
+        print(json.dumps(out), flush=True)
+
+
+if __name__ == "__main__":
+    main()

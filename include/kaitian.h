@@ -179,6 +179,14 @@ int kt_unpack_scale(kt_ctx *ctx, const float *const *src, int from_combined,
  * Errors: KT_ERR_INVALID, KT_ERR_CUDA. */
 int kt_cast(const void *in, int in_dtype, void *out, int out_dtype, int64_t n, void *stream);
 
+/* Host <-> device movement of a tensor list (the accelerator <-> host RAM copies of
+ * Section III-A applied to per-parameter tensors): n asynchronous copies dst[i] <- src[i] of
+ * bytes[i] bytes on `stream`, one copy per tensor.
+ * dst, src, bytes: host arrays.  dir KT_H2D: src host (pinned for true asynchrony), dst
+ * device; KT_D2H: the reverse.  Errors: KT_ERR_INVALID, KT_ERR_CUDA. */
+int kt_copy_tensors(void *const *dst, const void *const *src, const int64_t *bytes, int n, int dir,
+                    void *stream);
+
 /* Number of kernels this context has launched so far (for launch accounting). */
 int64_t kt_launch_count(const kt_ctx *ctx);
 

@@ -25,7 +25,7 @@ KT_MAX_RANKS, KT_MAX_GROUPS = 64, 16
 
 EXPORTS = ["kt_schedule", "kt_groups_init", "kt_set_shares", "kt_set_coefficients",
            "kt_get_coefficients", "kt_bucket_pack", "kt_plan_buckets", "kt_plan_query", "kt_hier_reduce",
-           "kt_stage_to_host", "kt_stage_wait", "kt_unpack_scale", "kt_cast", "kt_launch_count",
+           "kt_stage_to_host", "kt_stage_wait", "kt_unpack_scale", "kt_cast", "kt_copy_tensors", "kt_launch_count",
            "kt_last_error", "kt_destroy"]
 
 _DTYPES = {torch.float32: KT_F32, torch.bfloat16: KT_BF16}
@@ -60,6 +60,7 @@ def _load() -> C.CDLL:
         "kt_stage_wait": ([vp, C.c_int, C.c_int, vp, C.c_int], C.c_int),
         "kt_unpack_scale": ([vp, vpp, C.c_int, vpp, C.c_int, C.c_int, C.c_float, C.c_int, vp], C.c_int),
         "kt_cast": ([vp, C.c_int, vp, C.c_int, C.c_int64, vp], C.c_int),
+        "kt_copy_tensors": ([vpp, vpp, i64p, C.c_int, C.c_int, vp], C.c_int),
         "kt_launch_count": ([vp], C.c_int64),
         "kt_last_error": ([vp], C.c_char_p),
         "kt_destroy": ([vp], None),
@@ -279,6 +280,14 @@ def kt_cast(inp: torch.Tensor, out: torch.Tensor, stream=None) -> None:
         raise KtError(KT_ERR_SHAPE, "kt_cast: size or dtype mismatch")
     _check(_lib.kt_cast(C.c_void_p(inp.data_ptr()), _DTYPES[inp.dtype], C.c_void_p(out.data_ptr()),
                         _DTYPES[out.dtype], inp.numel(), _stream(stream)))
+
+
+def kt_copy_tensors(dst: Ptrs, src: Ptrs, nbytes: Sequence[int], direction: int, stream=None) -> None:
+    d, s = kt_ptrs(dst), kt_ptrs(src)
+    if d.n != s.n or d.n != len(nbytes):
+        raise KtError(KT_ERR_SHAPE, "kt_copy_tensors: list lengths differ")
+    sizes = nbytes if isinstance(nbytes, C.Array) else (C.c_int64 * max(d.n, 1))(*[int(b) for b in nbytes])
+    _check(_lib.kt_copy_tensors(d.array, s.array, sizes, d.n, int(direction), _stream(stream)))
 
 
 def kt_launch_count(ctx: Ctx) -> int:

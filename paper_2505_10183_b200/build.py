@@ -11,6 +11,7 @@ import sys
 _PKG = os.path.dirname(os.path.abspath(__file__))
 _ROOT = os.path.dirname(_PKG)
 SOURCES = [os.path.join(_PKG, "csrc", "kaitian.cu")]
+DEPENDS = [os.path.join(_PKG, "csrc", "kt_kernels.cuh")]
 HEADERS = [os.path.join(_ROOT, "include", "kaitian.h")]
 LIB = os.path.join(_PKG, "libkaitian_b200.so")
 
@@ -29,7 +30,7 @@ def is_stale() -> bool:
     if not os.path.exists(LIB):
         return True
     built = os.path.getmtime(LIB)
-    return any(os.path.getmtime(p) > built for p in SOURCES + HEADERS)
+    return any(os.path.getmtime(p) > built for p in SOURCES + DEPENDS + HEADERS)
 
 
 def build(force: bool = False, verbose: bool = False) -> str:

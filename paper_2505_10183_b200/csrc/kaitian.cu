@@ -1,6 +1,7 @@
-// kaitian.cu -- sm_100a kernels and C ABI for KAITIAN's hierarchical, load-weighted
-// gradient synchronisation (paper Sections III-A and III-C).  See include/kaitian.h for
-// the contract of every entry point.
+// kaitian.cu -- host side of the C ABI for KAITIAN's hierarchical, load-weighted gradient
+// synchronisation (paper Sections III-A and III-C): scheduler, weights, bucket plan, device
+// tables, launches, pinned-host staging.  The kernels are in kt_kernels.cuh; the contract of
+// every entry point is in include/kaitian.h.
 //
 // Data layout in device memory
 //   gradients   K*T caller-owned tensors (fp32 or bf16), read in place through a pointer
@@ -10,18 +11,12 @@
 //               multiples of 64, zero padding in the gaps
 //   tensor table  one 32-byte record per tensor (transport offset, numel, numel + padding,
 //               flags) and a prefix sum of TILE-sized work units per tensor
-// Work decomposition: the transport is cut into tiles of TILE elements that never cross a
-// tensor boundary.  A CTA walks tiles in a grid-stride loop, finds the tensor of a tile by
-// binary search in the prefix (shared memory), and streams the K rank buffers of that tile
-// with 128-bit loads.  Interior tiles of 16-byte aligned tensors take a branch-free vector
-// path; ragged tails, padding and misaligned tensors take an element-wise path.
-//
-// Arithmetic order is fixed: first member of a group acc = a*x (one rounded multiply),
-// later members acc = fma(a, x, acc); the same across groups with W_g.
 
 #include "../../include/kaitian.h"
 
 #include <cuda_runtime.h>
+
+#include "kt_kernels.cuh"
 
 #include <chrono>
 #include <cmath>
@@ -34,10 +29,6 @@
 #include <vector>
 
 namespace {
-
-constexpr int NT = 256;          // threads per CTA
-constexpr int TILE = 2048;       // transport elements per work unit
-constexpr int FLAG_ALIGNED = 1;  // all K sources of the tensor are 16-byte aligned
 
 // ------------------------------------------------------------------ error reporting
 thread_local char g_err[512] = "";
@@ -56,352 +47,6 @@ int fail(int code, const char *fmt, ...) {
         if (e_ != cudaSuccess)                                                              \
             return fail(KT_ERR_CUDA, "%s: %s", #call, cudaGetErrorString(e_));              \
     } while (0)
-
-// ------------------------------------------------------------------ device tables
-struct TInfo {            // one per tensor, transport order
-    long long dst_off;    // element offset in the transport
-    long long numel;      // gradient elements
-    long long ext;        // numel + zero padding up to the next tensor (multiple of 8 apart)
-    int flags;
-    int pad_;
-};
-
-struct RankTab {          // ranks in group-major order (ascending rank inside a group)
-    float coef[KT_MAX_RANKS];
-    signed char gid[KT_MAX_RANKS];
-    unsigned char first[KT_MAX_RANKS];   // first member of its group
-    unsigned char last[KT_MAX_RANKS];    // last member of its group
-    int K;
-};
-
-struct GroupTab {
-    float W[KT_MAX_GROUPS];
-    int G;
-};
-
-struct TilePlan {         // which tiles a launch covers and how to decode them
-    const int *prefix;    // [T+1] tiles before tensor u
-    const TInfo *info;    // [T]
-    int T;
-    int u_lo, u_hi;       // tensors [u_lo, u_hi) take part
-    int tile_lo;          // prefix[u_lo]
-    int n_tiles;          // prefix[u_hi] - prefix[u_lo]
-    int prefix_in_smem;   // stage prefix[u_lo .. u_hi] in shared memory
-};
-
-struct K1Params {
-    TilePlan tp;
-    const void *const *ptrs;           // [K][T] device pointer table
-    float *transport[KT_MAX_GROUPS];
-    RankTab rt;
-};
-
-struct K2Params {
-    TilePlan tp;
-    const float *src[KT_MAX_GROUPS];   // partials (or one combined buffer)
-    GroupTab gt;
-    void *const *out_ptrs;             // [R][T] device pointer table
-    const unsigned char *out_aligned;  // [T] all R destinations 16-byte aligned
-    int R;
-    float scale;
-};
-
-struct PackParams {
-    TilePlan tp;
-    const void *const *ptrs;           // [K][T], group-major rank order
-    void *flat[KT_MAX_RANKS];          // same rank order
-    int K;
-};
-
-// ------------------------------------------------------------------ device helpers
-__device__ __forceinline__ uint4 ld_stream(const void *p) {
-    // read-once data: keep it out of L1
-    uint4 v;
-    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
-                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
-                 : "l"(p));
-    return v;
-}
-
-template <typename P>
-__device__ __forceinline__ P *ldg_ptr(P *const *slot) {
-    // pointer tables are read-only for the lifetime of a launch
-    return reinterpret_cast<P *>(__ldg(reinterpret_cast<const unsigned long long *>(slot)));
-}
-
-__device__ __forceinline__ unsigned pack_bf16x2(float lo, float hi) {
-    unsigned d;   // round-to-nearest-even narrowing of two floats; hi lands in the upper half
-    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
-    return d;
-}
-
-template <typename T> struct Elem;
-template <> struct Elem<float> {
-    static constexpr int VEC = 4;
-    __device__ static __forceinline__ float widen(float v) { return v; }
-    __device__ static __forceinline__ void unpack(const uint4 &v, float (&x)[4]) {
-        x[0] = __uint_as_float(v.x); x[1] = __uint_as_float(v.y);
-        x[2] = __uint_as_float(v.z); x[3] = __uint_as_float(v.w);
-    }
-};
-template <> struct Elem<unsigned short> {
-    static constexpr int VEC = 8;
-    __device__ static __forceinline__ float widen(unsigned short v) {
-        return __uint_as_float(static_cast<unsigned>(v) << 16);
-    }
-    __device__ static __forceinline__ void unpack(const uint4 &v, float (&x)[8]) {
-        x[0] = __uint_as_float(v.x << 16); x[1] = __uint_as_float(v.x & 0xFFFF0000u);
-        x[2] = __uint_as_float(v.y << 16); x[3] = __uint_as_float(v.y & 0xFFFF0000u);
-        x[4] = __uint_as_float(v.z << 16); x[5] = __uint_as_float(v.z & 0xFFFF0000u);
-        x[6] = __uint_as_float(v.w << 16); x[7] = __uint_as_float(v.w & 0xFFFF0000u);
-    }
-};
-
-// Stage the tile prefix of the participating tensors in shared memory (or leave it global).
-__device__ __forceinline__ const int *stage_prefix(const TilePlan &tp, int *smem) {
-    if (!tp.prefix_in_smem) return tp.prefix + tp.u_lo;
-    const int n = tp.u_hi - tp.u_lo + 1;
-    for (int i = threadIdx.x; i < n; i += NT) smem[i] = tp.prefix[tp.u_lo + i];
-    __syncthreads();
-    return smem;
-}
-
-// Largest u in [0, n) with pre[u] <= tile (pre is non-decreasing, pre[n] > tile).
-__device__ __forceinline__ int find_tensor(const int *pre, int n, int tile) {
-    int lo = 0, hi = n;
-    while (hi - lo > 1) {
-        const int mid = (lo + hi) >> 1;
-        if (pre[mid] <= tile) lo = mid; else hi = mid;
-    }
-    return lo;
-}
-
-// ------------------------------------------------------------------ K1: fused pack + widen + weighted intra-group reduce
-// P_g[off_u + e] = sum_{r in g} a_r * f32(x_r^(u)[e]), zero in the padding.
-template <typename Tin, int KB>
-__global__ void __launch_bounds__(NT) k1_intra_reduce(const __grid_constant__ K1Params p) {
-    constexpr int VEC = Elem<Tin>::VEC;
-    constexpr int ITERS = TILE / (NT * VEC);
-    extern __shared__ int smem_prefix[];
-    const int *pre = stage_prefix(p.tp, smem_prefix);
-    const int nu = p.tp.u_hi - p.tp.u_lo;
-    const int K = p.rt.K;
-    const int T = p.tp.T;
-
-    for (int tile = blockIdx.x; tile < p.tp.n_tiles; tile += gridDim.x) {
-        const int gt = tile + p.tp.tile_lo;
-        const int ul = find_tensor(pre, nu, gt);
-        const int u = ul + p.tp.u_lo;
-        const TInfo ti = p.tp.info[u];
-        const long long e0 = static_cast<long long>(gt - pre[ul]) * TILE;
-
-        if ((ti.flags & FLAG_ALIGNED) && e0 + TILE <= ti.numel) {
-            // ---- interior tile, every source 16-byte aligned: branch-free vector path
-            const long long v0 = (e0 / VEC) + threadIdx.x;       // 16-byte vector index
-            float acc[ITERS][VEC];
-            for (int kb = 0; kb < K; kb += KB) {
-                uint4 raw[KB][ITERS];
-#pragma unroll
-                for (int j = 0; j < KB; ++j) {
-                    if (kb + j < K) {
-                        const uint4 *s = static_cast<const uint4 *>(
-                            ldg_ptr(&p.ptrs[static_cast<size_t>(kb + j) * T + u])) + v0;
-#pragma unroll
-                        for (int it = 0; it < ITERS; ++it) raw[j][it] = ld_stream(s + it * NT);
-                    }
-                }
-#pragma unroll
-                for (int j = 0; j < KB; ++j) {
-                    if (kb + j < K) {
-                        const float a = p.rt.coef[kb + j];
-                        const bool first = p.rt.first[kb + j];
-#pragma unroll
-                        for (int it = 0; it < ITERS; ++it) {
-                            float x[VEC];
-                            Elem<Tin>::unpack(raw[j][it], x);
-#pragma unroll
-                            for (int c = 0; c < VEC; ++c)
-                                acc[it][c] = first ? __fmul_rn(a, x[c]) : __fmaf_rn(a, x[c], acc[it][c]);
-                        }
-                        if (p.rt.last[kb + j]) {
-                            float *d = p.transport[p.rt.gid[kb + j]] + ti.dst_off + e0;
-#pragma unroll
-                            for (int it = 0; it < ITERS; ++it) {
-                                float4 *dv = reinterpret_cast<float4 *>(d + (it * NT + threadIdx.x) * VEC);
-#pragma unroll
-                                for (int q = 0; q < VEC / 4; ++q)
-                                    dv[q] = make_float4(acc[it][4 * q], acc[it][4 * q + 1],
-                                                        acc[it][4 * q + 2], acc[it][4 * q + 3]);
-                            }
-                        }
-                    }
-                }
-            }
-        } else {
-            // ---- ragged tail, padding or misaligned tensor: groups of 4 elements, element loads
-            for (long long e = e0 + 4 * threadIdx.x; e < e0 + TILE && e < ti.ext; e += 4 * NT) {
-                float acc[4] = {0.f, 0.f, 0.f, 0.f};
-                for (int k = 0; k < K; ++k) {
-                    const Tin *s = static_cast<const Tin *>(ldg_ptr(&p.ptrs[static_cast<size_t>(k) * T + u]));
-                    const float a = p.rt.coef[k];
-                    const bool first = p.rt.first[k];
-#pragma unroll
-                    for (int c = 0; c < 4; ++c) {
-                        if (e + c < ti.numel) {
-                            const float x = Elem<Tin>::widen(s[e + c]);
-                            acc[c] = first ? __fmul_rn(a, x) : __fmaf_rn(a, x, acc[c]);
-                        } else {
-                            acc[c] = 0.f;
-                        }
-                    }
-                    if (p.rt.last[k])
-                        *reinterpret_cast<float4 *>(p.transport[p.rt.gid[k]] + ti.dst_off + e) =
-                            make_float4(acc[0], acc[1], acc[2], acc[3]);
-                }
-            }
-        }
-    }
-}
-
-// ------------------------------------------------------------------ K2: inter-group combine + scale + cast + unpack
-// out_c^(u)[e] = cast(scale * sum_g W_g P_g[off_u + e]) for every copy c < R.
-template <typename Tout>
-__global__ void __launch_bounds__(NT) k2_combine_unpack(const __grid_constant__ K2Params p) {
-    constexpr int VEC = Elem<Tout>::VEC;
-    constexpr int ITERS = TILE / (NT * VEC);
-    extern __shared__ int smem_prefix[];
-    const int *pre = stage_prefix(p.tp, smem_prefix);
-    const int nu = p.tp.u_hi - p.tp.u_lo;
-    const int G = p.gt.G;
-    const int T = p.tp.T;
-
-    for (int tile = blockIdx.x; tile < p.tp.n_tiles; tile += gridDim.x) {
-        const int gt = tile + p.tp.tile_lo;
-        const int ul = find_tensor(pre, nu, gt);
-        const int u = ul + p.tp.u_lo;
-        const TInfo ti = p.tp.info[u];
-        const long long e0 = static_cast<long long>(gt - pre[ul]) * TILE;
-
-        if (p.out_aligned[u] && e0 + TILE <= ti.numel) {
-            float acc[ITERS][VEC];
-#pragma unroll
-            for (int it = 0; it < ITERS; ++it) {
-                const long long e = e0 + (it * NT + threadIdx.x) * VEC;
-                for (int g = 0; g < G; ++g) {
-                    const float4 *s = reinterpret_cast<const float4 *>(p.src[g] + ti.dst_off + e);
-                    const float w = p.gt.W[g];
-#pragma unroll
-                    for (int q = 0; q < VEC / 4; ++q) {
-                        const float4 v = s[q];
-                        if (g == 0) {
-                            acc[it][4 * q] = __fmul_rn(w, v.x); acc[it][4 * q + 1] = __fmul_rn(w, v.y);
-                            acc[it][4 * q + 2] = __fmul_rn(w, v.z); acc[it][4 * q + 3] = __fmul_rn(w, v.w);
-                        } else {
-                            acc[it][4 * q] = __fmaf_rn(w, v.x, acc[it][4 * q]);
-                            acc[it][4 * q + 1] = __fmaf_rn(w, v.y, acc[it][4 * q + 1]);
-                            acc[it][4 * q + 2] = __fmaf_rn(w, v.z, acc[it][4 * q + 2]);
-                            acc[it][4 * q + 3] = __fmaf_rn(w, v.w, acc[it][4 * q + 3]);
-                        }
-                    }
-                }
-            }
-#pragma unroll
-            for (int it = 0; it < ITERS; ++it) {
-                uint4 o;
-                float y[VEC];
-#pragma unroll
-                for (int c = 0; c < VEC; ++c) y[c] = __fmul_rn(acc[it][c], p.scale);
-                if constexpr (VEC == 4) {
-                    o = make_uint4(__float_as_uint(y[0]), __float_as_uint(y[1]), __float_as_uint(y[2]),
-                                   __float_as_uint(y[3]));
-                } else {
-                    o = make_uint4(pack_bf16x2(y[0], y[1]), pack_bf16x2(y[2], y[3]),
-                                   pack_bf16x2(y[4], y[5]), pack_bf16x2(y[6], y[7]));
-                }
-                const long long vi = e0 / VEC + it * NT + threadIdx.x;
-                for (int c = 0; c < p.R; ++c)
-                    static_cast<uint4 *>(ldg_ptr(&p.out_ptrs[static_cast<size_t>(c) * T + u]))[vi] = o;
-            }
-        } else {
-            for (long long e = e0 + threadIdx.x; e < e0 + TILE && e < ti.numel; e += NT) {
-                float acc = __fmul_rn(p.gt.W[0], p.src[0][ti.dst_off + e]);
-                for (int g = 1; g < G; ++g) acc = __fmaf_rn(p.gt.W[g], p.src[g][ti.dst_off + e], acc);
-                const float y = __fmul_rn(acc, p.scale);
-                for (int c = 0; c < p.R; ++c) {
-                    void *d = ldg_ptr(&p.out_ptrs[static_cast<size_t>(c) * T + u]);
-                    if (VEC == 4) static_cast<float *>(d)[e] = y;
-                    else static_cast<unsigned short *>(d)[e] = static_cast<unsigned short>(pack_bf16x2(y, 0.f) & 0xFFFFu);
-                }
-            }
-        }
-    }
-}
-
-// ------------------------------------------------------------------ flat inter-group combine into a combined buffer
-__global__ void __launch_bounds__(NT) k_combine_flat(const __grid_constant__ K2Params p, float *combined,
-                                                     long long lo, long long n4) {
-    const int G = p.gt.G;
-    for (long long i = blockIdx.x * static_cast<long long>(NT) + threadIdx.x; i < n4;
-         i += static_cast<long long>(gridDim.x) * NT) {
-        const long long e = lo + 4 * i;
-        float4 v = *reinterpret_cast<const float4 *>(p.src[0] + e);
-        const float w0 = p.gt.W[0];
-        float4 acc = make_float4(__fmul_rn(w0, v.x), __fmul_rn(w0, v.y), __fmul_rn(w0, v.z), __fmul_rn(w0, v.w));
-        for (int g = 1; g < G; ++g) {
-            v = *reinterpret_cast<const float4 *>(p.src[g] + e);
-            const float w = p.gt.W[g];
-            acc.x = __fmaf_rn(w, v.x, acc.x); acc.y = __fmaf_rn(w, v.y, acc.y);
-            acc.z = __fmaf_rn(w, v.z, acc.z); acc.w = __fmaf_rn(w, v.w, acc.w);
-        }
-        *reinterpret_cast<float4 *>(combined + e) = acc;
-    }
-}
-
-// ------------------------------------------------------------------ standalone pack (bit copy of every rank's tensors into its flat buffer)
-template <typename Tin>
-__global__ void __launch_bounds__(NT) k_pack(const __grid_constant__ PackParams p) {
-    constexpr int VEC = Elem<Tin>::VEC;
-    constexpr int ITERS = TILE / (NT * VEC);
-    extern __shared__ int smem_prefix[];
-    const int *pre = stage_prefix(p.tp, smem_prefix);
-    const int nu = p.tp.u_hi - p.tp.u_lo;
-    const int T = p.tp.T;
-    const int k = blockIdx.y;
-    Tin *flat = static_cast<Tin *>(p.flat[k]);
-
-    for (int tile = blockIdx.x; tile < p.tp.n_tiles; tile += gridDim.x) {
-        const int gt = tile + p.tp.tile_lo;
-        const int ul = find_tensor(pre, nu, gt);
-        const int u = ul + p.tp.u_lo;
-        const TInfo ti = p.tp.info[u];
-        const long long e0 = static_cast<long long>(gt - pre[ul]) * TILE;
-        const Tin *s = static_cast<const Tin *>(ldg_ptr(&p.ptrs[static_cast<size_t>(k) * T + u]));
-        if ((ti.flags & FLAG_ALIGNED) && e0 + TILE <= ti.numel) {
-            const uint4 *sv = reinterpret_cast<const uint4 *>(s + e0) + threadIdx.x;
-            uint4 *dv = reinterpret_cast<uint4 *>(flat + ti.dst_off + e0) + threadIdx.x;
-            uint4 raw[ITERS];
-#pragma unroll
-            for (int it = 0; it < ITERS; ++it) raw[it] = ld_stream(sv + it * NT);
-#pragma unroll
-            for (int it = 0; it < ITERS; ++it) dv[it * NT] = raw[it];
-        } else {
-            for (long long e = e0 + threadIdx.x; e < e0 + TILE && e < ti.ext; e += NT)
-                flat[ti.dst_off + e] = e < ti.numel ? s[e] : Tin(0);
-        }
-    }
-}
-
-// ------------------------------------------------------------------ standalone casts
-__global__ void __launch_bounds__(NT) k_cast_bf16_to_f32(const unsigned short *in, float *out, long long n) {
-    for (long long i = blockIdx.x * static_cast<long long>(NT) + threadIdx.x; i < n;
-         i += static_cast<long long>(gridDim.x) * NT)
-        out[i] = __uint_as_float(static_cast<unsigned>(in[i]) << 16);
-}
-__global__ void __launch_bounds__(NT) k_cast_f32_to_bf16(const float *in, unsigned short *out, long long n) {
-    for (long long i = blockIdx.x * static_cast<long long>(NT) + threadIdx.x; i < n;
-         i += static_cast<long long>(gridDim.x) * NT)
-        out[i] = static_cast<unsigned short>(pack_bf16x2(in[i], 0.f) & 0xFFFFu);
-}
 
 // ------------------------------------------------------------------ host-side state
 struct StageSlot {
@@ -558,12 +203,7 @@ int make_tile_plan(const kt_ctx *c, int bucket, TilePlan *tp) {
     tp->u_hi = bucket < 0 ? c->T : c->bucket_u_hi[bucket];
     tp->tile_lo = c->prefix[tp->u_lo];
     tp->n_tiles = c->prefix[tp->u_hi] - tp->tile_lo;
-    tp->prefix_in_smem = (tp->u_hi - tp->u_lo + 1) * sizeof(int) <= 32 * 1024;
     return KT_OK;
-}
-
-size_t prefix_smem(const TilePlan &tp) {
-    return tp.prefix_in_smem ? (tp.u_hi - tp.u_lo + 1) * sizeof(int) : 0;
 }
 
 void bucket_range(const kt_ctx *c, int bucket, int64_t *lo, int64_t *n) {
@@ -594,11 +234,11 @@ int check_buffers(const kt_ctx *c, const float *const *bufs, int n, const char *
 
 template <typename Tin>
 int launch_k1(kt_ctx *c, const K1Params &p, cudaStream_t s) {
-    const size_t sm = prefix_smem(p.tp);
+    // one CTA per tile
     if (c->K <= 4)
-        k1_intra_reduce<Tin, 4><<<grid_for(c, k1_intra_reduce<Tin, 4>, sm, p.tp.n_tiles), NT, sm, s>>>(p);
+        k1_intra_reduce<Tin, 4><<<p.tp.n_tiles, NT, 0, s>>>(p);
     else
-        k1_intra_reduce<Tin, 8><<<grid_for(c, k1_intra_reduce<Tin, 8>, sm, p.tp.n_tiles), NT, sm, s>>>(p);
+        k1_intra_reduce<Tin, 8><<<p.tp.n_tiles, NT, 0, s>>>(p);
     c->launches += 1;
     KT_CUDA(cudaGetLastError());
     return KT_OK;
@@ -835,12 +475,11 @@ int kt_bucket_pack(kt_ctx *c, const void *const *grads, const int64_t *numel, in
         p.K = c->K;
         for (int k = 0; k < c->K; ++k) p.flat[k] = flat_out[c->order[k]];
         if (p.tp.n_tiles > 0) {
-            const size_t sm = prefix_smem(p.tp);
             cudaStream_t s = static_cast<cudaStream_t>(stream);
             if (in_dtype == KT_F32)
-                k_pack<float><<<dim3(grid_for(c, k_pack<float>, sm, p.tp.n_tiles), c->K), NT, sm, s>>>(p);
+                k_pack<float><<<dim3(p.tp.n_tiles, c->K), NT, 0, s>>>(p);
             else
-                k_pack<unsigned short><<<dim3(grid_for(c, k_pack<unsigned short>, sm, p.tp.n_tiles), c->K), NT, sm, s>>>(p);
+                k_pack<unsigned short><<<dim3(p.tp.n_tiles, c->K), NT, 0, s>>>(p);
             c->launches += 1;
             KT_CUDA(cudaGetLastError());
         }
@@ -1047,11 +686,10 @@ int kt_unpack_scale(kt_ctx *c, const float *const *src, int from_combined, void 
     p.out_aligned = static_cast<const unsigned char *>(c->d_out) + sz_ptrs;
     p.R = R;
     p.scale = scale;
-    const size_t sm = prefix_smem(tp);
     if (out_dtype == KT_F32)
-        k2_combine_unpack<float><<<grid_for(c, k2_combine_unpack<float>, sm, tp.n_tiles), NT, sm, s>>>(p);
+        k2_combine_unpack<float><<<tp.n_tiles, NT, 0, s>>>(p);
     else
-        k2_combine_unpack<unsigned short><<<grid_for(c, k2_combine_unpack<unsigned short>, sm, tp.n_tiles), NT, sm, s>>>(p);
+        k2_combine_unpack<unsigned short><<<tp.n_tiles, NT, 0, s>>>(p);
     c->launches += 1;
     KT_CUDA(cudaGetLastError());
     return KT_OK;
@@ -1079,6 +717,24 @@ int kt_cast(const void *in, int in_dtype, void *out, int out_dtype, int64_t n, v
     else
         k_cast_f32_to_bf16<<<grid, NT, 0, s>>>(static_cast<const float *>(in), static_cast<unsigned short *>(out), n);
     KT_CUDA(cudaGetLastError());
+    return KT_OK;
+}
+
+int kt_copy_tensors(void *const *dst, const void *const *src, const int64_t *bytes, int n, int dir, void *stream) {
+    if (n < 0) return fail(KT_ERR_INVALID, "n is negative");
+    if (n == 0) return KT_OK;
+    if (!dst || !src || !bytes) return fail(KT_ERR_INVALID, "NULL argument");
+    if (dir != KT_D2H && dir != KT_H2D) return fail(KT_ERR_INVALID, "unknown direction %d", dir);
+    const cudaMemcpyKind kind = dir == KT_D2H ? cudaMemcpyDeviceToHost : cudaMemcpyHostToDevice;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    for (int i = 0; i < n; ++i) {
+        if (bytes[i] < 0) return fail(KT_ERR_INVALID, "bytes[%d] is negative", i);
+        if (bytes[i] > 0 && (!dst[i] || !src[i])) return fail(KT_ERR_INVALID, "pointer %d is NULL", i);
+    }
+    // one copy per tensor: neighbouring tensors may belong to different host registrations,
+    // which a single copy must not span
+    for (int i = 0; i < n; ++i)
+        if (bytes[i] > 0) KT_CUDA(cudaMemcpyAsync(dst[i], src[i], static_cast<size_t>(bytes[i]), kind, s));
     return KT_OK;
 }
 

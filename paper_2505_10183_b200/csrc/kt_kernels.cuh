@@ -1,0 +1,380 @@
+// kt_kernels.cuh -- device tables and sm_100a kernels of the hierarchical, load-weighted
+// gradient synchronisation (paper Section III-A: intra-group reduce, fp32 transport,
+// inter-group combine; Section III-C supplies the weights).
+//
+// Work decomposition.  The fp32 transport is cut into tiles of TILE elements that never
+// cross a tensor boundary; one CTA handles one tile (the grid is the tile count, so the
+// hardware scheduler balances ragged tensor lists and partial waves by itself).  A CTA
+// finds its tensor by binary search in the per-tensor tile prefix, then streams the K rank
+// buffers of that tile with 128-bit loads, all loads of a batch of ranks issued before the
+// first multiply.  Interior tiles of 16-byte aligned tensors run without predicates; tiles
+// that hold a tensor's tail, zero padding, or a misaligned tensor use the same code with
+// per-vector predicates and element loads only where a vector would cross the end.
+//
+// Arithmetic order is fixed: first member of a group acc = a*x (one rounded multiply),
+// later members acc = fma(a, x, acc); the same across groups with W_g.
+#pragma once
+
+#include <cuda_runtime.h>
+
+#include "../../include/kaitian.h"
+
+namespace {
+
+constexpr int NT = 256;          // threads per CTA
+constexpr int TILE = 2048;       // transport elements per work unit
+constexpr int FLAG_ALIGNED = 1;  // all K sources of the tensor are 16-byte aligned
+
+// ------------------------------------------------------------------ device tables
+struct TInfo {            // one per tensor, transport order
+    long long dst_off;    // element offset in the transport
+    long long numel;      // gradient elements
+    long long ext;        // numel + zero padding up to the next tensor (a multiple of 8)
+    int flags;
+    int pad_;
+};
+
+struct RankTab {          // ranks in group-major order (ascending rank inside a group)
+    float coef[KT_MAX_RANKS];
+    signed char gid[KT_MAX_RANKS];
+    unsigned char first[KT_MAX_RANKS];   // first member of its group
+    unsigned char last[KT_MAX_RANKS];    // last member of its group
+    int K;
+};
+
+struct GroupTab {
+    float W[KT_MAX_GROUPS];
+    int G;
+};
+
+struct TilePlan {         // which tiles a launch covers and how to decode them
+    const int *prefix;    // [T+1] tiles before tensor u
+    const TInfo *info;    // [T]
+    int T;
+    int u_lo, u_hi;       // tensors [u_lo, u_hi) take part
+    int tile_lo;          // prefix[u_lo]
+    int n_tiles;          // prefix[u_hi] - prefix[u_lo]
+};
+
+struct K1Params {
+    TilePlan tp;
+    const void *const *ptrs;           // [K][T] device pointer table
+    float *transport[KT_MAX_GROUPS];
+    RankTab rt;
+};
+
+struct K2Params {
+    TilePlan tp;
+    const float *src[KT_MAX_GROUPS];   // partials (or one combined buffer)
+    GroupTab gt;
+    void *const *out_ptrs;             // [R][T] device pointer table
+    const unsigned char *out_aligned;  // [T] all R destinations 16-byte aligned
+    int R;
+    float scale;
+};
+
+struct PackParams {
+    TilePlan tp;
+    const void *const *ptrs;           // [K][T], group-major rank order
+    void *flat[KT_MAX_RANKS];          // same rank order
+    int K;
+};
+
+// ------------------------------------------------------------------ device helpers
+__device__ __forceinline__ uint4 ld_stream(const void *p) {
+    // read-once data: keep it out of L1
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                 : "l"(p));
+    return v;
+}
+
+template <typename P>
+__device__ __forceinline__ P *ldg_ptr(P *const *slot) {
+    // pointer tables are read-only for the lifetime of a launch
+    return reinterpret_cast<P *>(__ldg(reinterpret_cast<const unsigned long long *>(slot)));
+}
+
+__device__ __forceinline__ unsigned pack_bf16x2(float lo, float hi) {
+    unsigned d;   // round-to-nearest-even narrowing of two floats; hi lands in the upper half
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
+    return d;
+}
+
+template <typename T> struct Elem;
+template <> struct Elem<float> {
+    static constexpr int VEC = 4;   // elements per 16-byte vector
+    __device__ static __forceinline__ void unpack(const uint4 &v, float (&x)[4]) {
+        x[0] = __uint_as_float(v.x); x[1] = __uint_as_float(v.y);
+        x[2] = __uint_as_float(v.z); x[3] = __uint_as_float(v.w);
+    }
+    // elements [e, e + 4) of s that lie below n, zero elsewhere
+    __device__ static __forceinline__ uint4 gather(const float *s, long long e, long long n) {
+        unsigned w[4];
+#pragma unroll
+        for (int c = 0; c < 4; ++c) w[c] = (e + c < n) ? __float_as_uint(s[e + c]) : 0u;
+        return make_uint4(w[0], w[1], w[2], w[3]);
+    }
+    __device__ static __forceinline__ uint4 narrow(const float (&y)[4]) {
+        return make_uint4(__float_as_uint(y[0]), __float_as_uint(y[1]), __float_as_uint(y[2]),
+                          __float_as_uint(y[3]));
+    }
+    __device__ static __forceinline__ float narrow_one(float y) { return y; }
+};
+template <> struct Elem<unsigned short> {
+    static constexpr int VEC = 8;
+    __device__ static __forceinline__ void unpack(const uint4 &v, float (&x)[8]) {
+        // bf16 is the upper half of a binary32: widening is a shift
+        x[0] = __uint_as_float(v.x << 16); x[1] = __uint_as_float(v.x & 0xFFFF0000u);
+        x[2] = __uint_as_float(v.y << 16); x[3] = __uint_as_float(v.y & 0xFFFF0000u);
+        x[4] = __uint_as_float(v.z << 16); x[5] = __uint_as_float(v.z & 0xFFFF0000u);
+        x[6] = __uint_as_float(v.w << 16); x[7] = __uint_as_float(v.w & 0xFFFF0000u);
+    }
+    __device__ static __forceinline__ uint4 gather(const unsigned short *s, long long e, long long n) {
+        unsigned w[4];
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+            const unsigned lo = (e + 2 * c < n) ? s[e + 2 * c] : 0u;
+            const unsigned hi = (e + 2 * c + 1 < n) ? s[e + 2 * c + 1] : 0u;
+            w[c] = lo | (hi << 16);
+        }
+        return make_uint4(w[0], w[1], w[2], w[3]);
+    }
+    __device__ static __forceinline__ uint4 narrow(const float (&y)[8]) {
+        return make_uint4(pack_bf16x2(y[0], y[1]), pack_bf16x2(y[2], y[3]), pack_bf16x2(y[4], y[5]),
+                          pack_bf16x2(y[6], y[7]));
+    }
+    __device__ static __forceinline__ unsigned short narrow_one(float y) {
+        return static_cast<unsigned short>(pack_bf16x2(y, 0.f) & 0xFFFFu);
+    }
+};
+
+// What a CTA works on: tensor u (transport order), its record, first element of the tile.
+struct TileRef {
+    int u;
+    TInfo ti;
+    long long e0;
+};
+
+// Tile -> tensor: largest u with prefix[u] <= tile (prefix is non-decreasing, its last entry
+// exceeds every tile of the launch).  Uniform across the CTA; the few words it reads stay in L1.
+__device__ __forceinline__ TileRef locate_tile(const TilePlan &tp) {
+    const int tile = blockIdx.x + tp.tile_lo;
+    int lo = tp.u_lo, hi = tp.u_hi;
+    while (hi - lo > 1) {
+        const int mid = (lo + hi) >> 1;
+        if (__ldg(tp.prefix + mid) <= tile) lo = mid; else hi = mid;
+    }
+    TileRef r;
+    r.u = lo;
+    const int4 *rec = reinterpret_cast<const int4 *>(tp.info + lo);
+    const int4 a = __ldg(rec), b = __ldg(rec + 1);
+    r.ti.dst_off = (static_cast<long long>(a.y) << 32) | static_cast<unsigned>(a.x);
+    r.ti.numel = (static_cast<long long>(a.w) << 32) | static_cast<unsigned>(a.z);
+    r.ti.ext = (static_cast<long long>(b.y) << 32) | static_cast<unsigned>(b.x);
+    r.ti.flags = b.z;
+    r.ti.pad_ = 0;
+    r.e0 = static_cast<long long>(tile - __ldg(tp.prefix + lo)) * TILE;
+    return r;
+}
+
+// ------------------------------------------------------------------ K1: fused pack + widen + weighted intra-group reduce
+// P_g[off_u + e] = sum_{r in g} a_r * f32(x_r^(u)[e]), zero in the padding.
+template <typename Tin, int KB, bool EDGE>
+__device__ __forceinline__ void k1_tile(const K1Params &p, const TileRef &t) {
+    constexpr int VEC = Elem<Tin>::VEC;
+    constexpr int ITERS = TILE / (NT * VEC);
+    const int K = p.rt.K;
+    const int T = p.tp.T;
+    const bool aligned = t.ti.flags & FLAG_ALIGNED;
+    long long e[ITERS];
+#pragma unroll
+    for (int it = 0; it < ITERS; ++it) e[it] = t.e0 + (it * NT + threadIdx.x) * VEC;
+
+    float acc[ITERS][VEC];
+    for (int kb = 0; kb < K; kb += KB) {
+        uint4 raw[KB][ITERS];
+#pragma unroll
+        for (int j = 0; j < KB; ++j) {
+            if (kb + j < K) {
+                const Tin *s = static_cast<const Tin *>(ldg_ptr(&p.ptrs[static_cast<size_t>(kb + j) * T + t.u]));
+#pragma unroll
+                for (int it = 0; it < ITERS; ++it) {
+                    if (!EDGE || (aligned && e[it] + VEC <= t.ti.numel))
+                        raw[j][it] = ld_stream(s + e[it]);
+                    else
+                        raw[j][it] = Elem<Tin>::gather(s, e[it], t.ti.numel);
+                }
+            }
+        }
+#pragma unroll
+        for (int j = 0; j < KB; ++j) {
+            if (kb + j < K) {
+                const float a = p.rt.coef[kb + j];
+                const bool first = p.rt.first[kb + j];
+#pragma unroll
+                for (int it = 0; it < ITERS; ++it) {
+                    float x[VEC];
+                    Elem<Tin>::unpack(raw[j][it], x);
+#pragma unroll
+                    for (int c = 0; c < VEC; ++c)
+                        acc[it][c] = first ? __fmul_rn(a, x[c]) : __fmaf_rn(a, x[c], acc[it][c]);
+                }
+                if (p.rt.last[kb + j]) {
+                    float *d = p.transport[p.rt.gid[kb + j]] + t.ti.dst_off;
+#pragma unroll
+                    for (int it = 0; it < ITERS; ++it) {
+                        if (EDGE) {
+                            if (e[it] >= t.ti.ext) continue;
+#pragma unroll
+                            for (int c = 0; c < VEC; ++c)   // padding is +0 whatever the weights
+                                if (e[it] + c >= t.ti.numel) acc[it][c] = 0.f;
+                        }
+                        float4 *dv = reinterpret_cast<float4 *>(d + e[it]);
+#pragma unroll
+                        for (int q = 0; q < VEC / 4; ++q)
+                            dv[q] = make_float4(acc[it][4 * q], acc[it][4 * q + 1], acc[it][4 * q + 2],
+                                                acc[it][4 * q + 3]);
+                    }
+                }
+            }
+        }
+    }
+}
+
+template <typename Tin, int KB>
+__global__ void __launch_bounds__(NT) k1_intra_reduce(const __grid_constant__ K1Params p) {
+    const TileRef t = locate_tile(p.tp);
+    if ((t.ti.flags & FLAG_ALIGNED) && t.e0 + TILE <= t.ti.numel)
+        k1_tile<Tin, KB, false>(p, t);
+    else
+        k1_tile<Tin, KB, true>(p, t);
+}
+
+// ------------------------------------------------------------------ K2: inter-group combine + scale + cast + unpack
+// out_c^(u)[e] = cast(scale * sum_g W_g P_g[off_u + e]) for every copy c < R.
+template <typename Tout, bool EDGE>
+__device__ __forceinline__ void k2_tile(const K2Params &p, const TileRef &t) {
+    constexpr int VEC = Elem<Tout>::VEC;
+    constexpr int ITERS = TILE / (NT * VEC);
+    constexpr int Q = VEC / 4;
+    const int G = p.gt.G;
+    const int T = p.tp.T;
+    const bool aligned = p.out_aligned[t.u];
+    long long e[ITERS];
+#pragma unroll
+    for (int it = 0; it < ITERS; ++it) e[it] = t.e0 + (it * NT + threadIdx.x) * VEC;
+
+    float acc[ITERS][VEC];
+    for (int g = 0; g < G; ++g) {
+        const float *s = p.src[g] + t.ti.dst_off;
+        const float w = p.gt.W[g];
+        float4 v[ITERS][Q];
+#pragma unroll
+        for (int it = 0; it < ITERS; ++it) {
+#pragma unroll
+            for (int q = 0; q < Q; ++q) {
+                // the transport holds ext elements per tensor, so a vector below ext is readable
+                if (!EDGE || e[it] < t.ti.ext) v[it][q] = __ldcs(reinterpret_cast<const float4 *>(s + e[it]) + q);
+                else v[it][q] = make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+        }
+#pragma unroll
+        for (int it = 0; it < ITERS; ++it) {
+#pragma unroll
+            for (int q = 0; q < Q; ++q) {
+                const float x[4] = {v[it][q].x, v[it][q].y, v[it][q].z, v[it][q].w};
+#pragma unroll
+                for (int c = 0; c < 4; ++c)
+                    acc[it][4 * q + c] = g == 0 ? __fmul_rn(w, x[c]) : __fmaf_rn(w, x[c], acc[it][4 * q + c]);
+            }
+        }
+    }
+#pragma unroll
+    for (int it = 0; it < ITERS; ++it) {
+        float y[VEC];
+#pragma unroll
+        for (int c = 0; c < VEC; ++c) y[c] = __fmul_rn(acc[it][c], p.scale);
+        if (!EDGE || (aligned && e[it] + VEC <= t.ti.numel)) {
+            const uint4 o = Elem<Tout>::narrow(y);
+            for (int c = 0; c < p.R; ++c)
+                *reinterpret_cast<uint4 *>(static_cast<Tout *>(ldg_ptr(&p.out_ptrs[static_cast<size_t>(c) * T + t.u])) + e[it]) = o;
+        } else if (e[it] < t.ti.numel) {
+            for (int c = 0; c < p.R; ++c) {
+                Tout *d = static_cast<Tout *>(ldg_ptr(&p.out_ptrs[static_cast<size_t>(c) * T + t.u]));
+#pragma unroll
+                for (int k = 0; k < VEC; ++k)
+                    if (e[it] + k < t.ti.numel) d[e[it] + k] = Elem<Tout>::narrow_one(y[k]);
+            }
+        }
+    }
+}
+
+template <typename Tout>
+__global__ void __launch_bounds__(NT) k2_combine_unpack(const __grid_constant__ K2Params p) {
+    const TileRef t = locate_tile(p.tp);
+    if (p.out_aligned[t.u] && t.e0 + TILE <= t.ti.numel)
+        k2_tile<Tout, false>(p, t);
+    else
+        k2_tile<Tout, true>(p, t);
+}
+
+// ------------------------------------------------------------------ flat inter-group combine into a combined buffer
+__global__ void __launch_bounds__(NT) k_combine_flat(const __grid_constant__ K2Params p, float *combined,
+                                                     long long lo, long long n4) {
+    const int G = p.gt.G;
+    for (long long i = blockIdx.x * static_cast<long long>(NT) + threadIdx.x; i < n4;
+         i += static_cast<long long>(gridDim.x) * NT) {
+        const long long e = lo + 4 * i;
+        float4 v = *reinterpret_cast<const float4 *>(p.src[0] + e);
+        const float w0 = p.gt.W[0];
+        float4 acc = make_float4(__fmul_rn(w0, v.x), __fmul_rn(w0, v.y), __fmul_rn(w0, v.z), __fmul_rn(w0, v.w));
+        for (int g = 1; g < G; ++g) {
+            v = *reinterpret_cast<const float4 *>(p.src[g] + e);
+            const float w = p.gt.W[g];
+            acc.x = __fmaf_rn(w, v.x, acc.x); acc.y = __fmaf_rn(w, v.y, acc.y);
+            acc.z = __fmaf_rn(w, v.z, acc.z); acc.w = __fmaf_rn(w, v.w, acc.w);
+        }
+        *reinterpret_cast<float4 *>(combined + e) = acc;
+    }
+}
+
+// ------------------------------------------------------------------ standalone pack (bit copy of every rank's tensors into its flat buffer)
+template <typename Tin>
+__global__ void __launch_bounds__(NT) k_pack(const __grid_constant__ PackParams p) {
+    constexpr int VEC = Elem<Tin>::VEC;
+    constexpr int ITERS = TILE / (NT * VEC);
+    const TileRef t = locate_tile(p.tp);
+    const int k = blockIdx.y;
+    const Tin *s = static_cast<const Tin *>(ldg_ptr(&p.ptrs[static_cast<size_t>(k) * p.tp.T + t.u]));
+    Tin *flat = static_cast<Tin *>(p.flat[k]) + t.ti.dst_off;
+    const bool aligned = t.ti.flags & FLAG_ALIGNED;
+    uint4 raw[ITERS];
+#pragma unroll
+    for (int it = 0; it < ITERS; ++it) {
+        const long long e = t.e0 + (it * NT + threadIdx.x) * VEC;
+        if (aligned && e + VEC <= t.ti.numel) raw[it] = ld_stream(s + e);
+        else raw[it] = Elem<Tin>::gather(s, e, t.ti.numel);
+    }
+#pragma unroll
+    for (int it = 0; it < ITERS; ++it) {
+        const long long e = t.e0 + (it * NT + threadIdx.x) * VEC;
+        // ext is a multiple of 8 elements, so a vector that starts below ext ends inside it
+        if (e < t.ti.ext) *reinterpret_cast<uint4 *>(flat + e) = raw[it];
+    }
+}
+
+// ------------------------------------------------------------------ standalone casts
+__global__ void __launch_bounds__(NT) k_cast_bf16_to_f32(const unsigned short *in, float *out, long long n) {
+    for (long long i = blockIdx.x * static_cast<long long>(NT) + threadIdx.x; i < n;
+         i += static_cast<long long>(gridDim.x) * NT)
+        out[i] = __uint_as_float(static_cast<unsigned>(in[i]) << 16);
+}
+__global__ void __launch_bounds__(NT) k_cast_f32_to_bf16(const float *in, unsigned short *out, long long n) {
+    for (long long i = blockIdx.x * static_cast<long long>(NT) + threadIdx.x; i < n;
+         i += static_cast<long long>(gridDim.x) * NT)
+        out[i] = static_cast<unsigned short>(pack_bf16x2(in[i], 0.f) & 0xFFFFu);
+}
+
+}  // namespace

@@ -1,0 +1,59 @@
+"""Runs a few launches of the two hot kernels on one small flat case, for profilers.
+
+    python -m paper_2505_10183_b200.profile_case --K 4 --bytes 67108864 --dtype f32 --launches 3
+
+One flat gradient buffer per rank (ranks 0..K/2-1 in group 0, the rest in group 1), the
+fused intra-group reduce and the combine+unpack kernel launched `launches` times each,
+after one warm-up launch of each.  Prints the CUDA-event time of every launch.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+
+import torch
+
+from . import binding as kt
+from . import workloads as W
+
+
+def main() -> None:
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--K", type=int, default=4)
+    ap.add_argument("--bytes", type=int, default=64 << 20, help="bytes per rank")
+    ap.add_argument("--dtype", default="f32", choices=["f32", "bf16"])
+    ap.add_argument("--launches", type=int, default=3)
+    ap.add_argument("--workload", default=None, help="a named workload instead of a flat case")
+    args = ap.parse_args()
+
+    torch.cuda.set_device(0)
+    wl = W.by_name(args.workload) if args.workload else W.sweep_point(args.K, args.bytes, args.dtype)
+    shares = list(wl.shares) if wl.shares is not None else kt.kt_schedule(wl.step_times, wl.global_batch)
+    dt = torch.float32 if wl.dtype == "f32" else torch.bfloat16
+    grads = [[t.cuda() for t in W.split_tensors(W.rank_gradients(wl, r, "cuda"), wl.numel)] for r in range(wl.K)]
+    ctx = kt.kt_groups_init(wl.group_of, shares, wl.G)
+    kt.kt_bucket_pack(ctx, grads, 1 << 62)
+    n = kt.kt_plan_query(ctx).transport_numel
+    transport = kt.kt_ptrs([torch.zeros(n, device="cuda") for _ in range(wl.G)])
+    out = kt.kt_ptrs([torch.zeros(m, dtype=dt, device="cuda") for m in wl.numel])
+    odt = kt.KT_F32 if wl.dtype == "f32" else kt.KT_BF16
+    times = {"k1_us": [], "k2_us": []}
+    for i in range(args.launches + 1):
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+        ev[0].record()
+        kt.kt_hier_reduce(ctx, kt.KT_INTRA, transport)
+        ev[1].record()
+        kt.kt_unpack_scale(ctx, transport, out, out_dtype=odt, R=1)
+        ev[2].record()
+        torch.cuda.synchronize()
+        if i:
+            times["k1_us"].append(round(ev[0].elapsed_time(ev[1]) * 1e3, 2))
+            times["k2_us"].append(round(ev[1].elapsed_time(ev[2]) * 1e3, 2))
+    k1_bytes = wl.K * wl.N * wl.elem_size + wl.G * wl.N * 4
+    k2_bytes = wl.G * wl.N * 4 + wl.N * wl.elem_size
+    print(json.dumps({"case": wl.name, "k1_bytes": k1_bytes, "k2_bytes": k2_bytes, **times}))
+    kt.kt_destroy(ctx)
+
+
+if __name__ == "__main__":
+    main()
