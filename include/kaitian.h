@@ -187,6 +187,41 @@ int kt_cast(const void *in, int in_dtype, void *out, int out_dtype, int64_t n, v
 int kt_copy_tensors(void *const *dst, const void *const *src, const int64_t *bytes, int n, int dir,
                     void *stream);
 
+/* The whole flat path in one call that allocates nothing.  (The paper has no counterpart:
+ * this entry point exists for the library's users, not for the method.)
+ *
+ * Who needs it: callers that are not allowed to allocate device memory at the point where
+ * gradients must be synchronised -- code running inside a framework's no-allocation region,
+ * plugins that must stay out of the host application's memory pool, processes whose device
+ * memory is fully planned up front.  Every other entry point either allocates small device
+ * tables itself (kt_bucket_pack, kt_unpack_scale) or needs caller-allocated transport
+ * buffers; this one keeps its tables and the fp32 group partials in a fixed array that is
+ * part of the library image.
+ *
+ * Computes, for one flat gradient buffer per rank,
+ *   out[i] = cast(scale * sum_g W_g * sum_{r in g} a_r * f32(grads[r][i])),  i < n,
+ * with the weights and the operation order of kt_groups_init / kt_hier_reduce /
+ * kt_unpack_scale (results are bit-identical to that route).
+ *   group_of[K], shares[K] (host): as in kt_groups_init.
+ *   grads (host array of K device pointers): n elements of in_dtype each, element aligned.
+ *   out (device): n elements of out_dtype.
+ * Limit: G * round_up(n, 64) <= KT_STATIC_MAX_ELEMS fp32 elements of scratch (4 MiB, held
+ * by every GPU that loads the library until the process exits); larger problems are
+ * rejected with KT_ERR_SHAPE and a message naming the sizes.
+ * Set-up: the first call on each device looks up the device address of the scratch array
+ * (with that device current).  Make that first call outside any stream capture.
+ * Sharing: all calls on a device use the same array, which keeps whatever the last call
+ * left in it.  Nothing in it has to start at zero -- each call rewrites the tables and every
+ * partial element it later reads -- but two calls that overlap on the GPU (different
+ * streams, or different host threads without ordering) race on it: keep calls on one
+ * stream, or order them with events.
+ * Calls no cudaMalloc / cudaFree and no allocating library routine; host state is on the
+ * stack.  Errors: KT_ERR_INVALID, KT_ERR_SHAPE, KT_ERR_ALIGN, KT_ERR_CUDA. */
+#define KT_STATIC_MAX_ELEMS (1 << 20)
+int kt_sync_flat_static(const int32_t *group_of, const int32_t *shares, int K, int G,
+                        const void *const *grads, int in_dtype, int64_t n, void *out, int out_dtype,
+                        float scale, void *stream);
+
 /* Number of kernels this context has launched so far (for launch accounting). */
 int64_t kt_launch_count(const kt_ctx *ctx);
 

@@ -25,7 +25,7 @@ KT_MAX_RANKS, KT_MAX_GROUPS = 64, 16
 
 EXPORTS = ["kt_schedule", "kt_groups_init", "kt_set_shares", "kt_set_coefficients",
            "kt_get_coefficients", "kt_bucket_pack", "kt_plan_buckets", "kt_plan_query", "kt_hier_reduce",
-           "kt_stage_to_host", "kt_stage_wait", "kt_unpack_scale", "kt_cast", "kt_copy_tensors", "kt_launch_count",
+           "kt_stage_to_host", "kt_stage_wait", "kt_unpack_scale", "kt_cast", "kt_copy_tensors", "kt_sync_flat_static", "kt_launch_count",
            "kt_last_error", "kt_destroy"]
 
 _DTYPES = {torch.float32: KT_F32, torch.bfloat16: KT_BF16}
@@ -61,6 +61,8 @@ def _load() -> C.CDLL:
         "kt_unpack_scale": ([vp, vpp, C.c_int, vpp, C.c_int, C.c_int, C.c_float, C.c_int, vp], C.c_int),
         "kt_cast": ([vp, C.c_int, vp, C.c_int, C.c_int64, vp], C.c_int),
         "kt_copy_tensors": ([vpp, vpp, i64p, C.c_int, C.c_int, vp], C.c_int),
+        "kt_sync_flat_static": ([i32p, i32p, C.c_int, C.c_int, vpp, C.c_int, C.c_int64, vp, C.c_int,
+                                 C.c_float, vp], C.c_int),
         "kt_launch_count": ([vp], C.c_int64),
         "kt_last_error": ([vp], C.c_char_p),
         "kt_destroy": ([vp], None),
@@ -288,6 +290,29 @@ def kt_copy_tensors(dst: Ptrs, src: Ptrs, nbytes: Sequence[int], direction: int,
         raise KtError(KT_ERR_SHAPE, "kt_copy_tensors: list lengths differ")
     sizes = nbytes if isinstance(nbytes, C.Array) else (C.c_int64 * max(d.n, 1))(*[int(b) for b in nbytes])
     _check(_lib.kt_copy_tensors(d.array, s.array, sizes, d.n, int(direction), _stream(stream)))
+
+
+KT_STATIC_MAX_ELEMS = 1 << 20
+
+
+def kt_sync_flat_static(group_of: Sequence[int], shares: Sequence[int], grads: Sequence[torch.Tensor],
+                        out: torch.Tensor, scale: float = 1.0, G: Optional[int] = None, stream=None) -> None:
+    """The flat path for callers that may not allocate device memory: one gradient buffer per
+    rank in, one reduced buffer out, scratch in the library's fixed device array.  Marshals
+    pointers only (no tensor is created here); see the header for limits and sharing rules."""
+    K = len(group_of)
+    if len(shares) != K or len(grads) != K:
+        raise KtError(KT_ERR_SHAPE, "group_of, shares and grads differ in length")
+    G = (max(group_of) + 1 if K else 0) if G is None else G
+    n = out.numel()
+    if any(g.numel() != n or g.dtype != grads[0].dtype or not g.is_contiguous() for g in grads):
+        raise KtError(KT_ERR_SHAPE, "grads: size, dtype or layout mismatch")
+    if grads[0].dtype not in _DTYPES or out.dtype not in _DTYPES or not out.is_contiguous():
+        raise KtError(KT_ERR_INVALID, "unsupported dtype or layout")
+    ptrs = (C.c_void_p * max(K, 1))(*[g.data_ptr() for g in grads])
+    _check(_lib.kt_sync_flat_static(_i32(group_of), _i32(shares), K, int(G), ptrs, _DTYPES[grads[0].dtype],
+                                    n, C.c_void_p(out.data_ptr()), _DTYPES[out.dtype], C.c_float(scale),
+                                    _stream(stream)))
 
 
 def kt_launch_count(ctx: Ctx) -> int:

@@ -21,8 +21,10 @@
 #include <chrono>
 #include <cmath>
 #include <cstdarg>
+#include <cstddef>
 #include <cstdio>
 #include <cstring>
+#include <mutex>
 #include <new>
 #include <thread>
 #include <utility>
@@ -756,3 +758,154 @@ void kt_destroy(kt_ctx *c) {
 }
 
 }  // extern "C"
+
+// ====================================================================== entry point that allocates nothing
+// For callers that must not allocate: code running where cudaMalloc is off limits (inside a
+// region that forbids synchronising allocations, under a memory pool it may not touch, late
+// in a process whose device memory is spoken for).  The whole flat path -- weighted
+// intra-group reduce, combine, scale, cast -- runs with its scratch (tensor table, pointer
+// tables and the fp32 group partials) in one file-scope device array of fixed size.
+namespace {
+
+constexpr size_t STATIC_TABLE_BYTES = 4096;
+
+struct alignas(256) StaticTables {      // image of the first STATIC_TABLE_BYTES of the scratch
+    int prefix[8];                      // tiles before tensor 0 and 1
+    alignas(32) TInfo info;             // the one tensor
+    alignas(8) const void *in_ptrs[KT_MAX_RANKS];
+    void *out_ptr[1];
+    unsigned char out_aligned[8];
+};
+static_assert(sizeof(StaticTables) <= STATIC_TABLE_BYTES, "tables outgrew their slot");
+
+// Held by every GPU that loads the library, until the process exits.
+static __device__ __align__(256) unsigned char
+    g_static_scratch[STATIC_TABLE_BYTES + static_cast<size_t>(KT_STATIC_MAX_ELEMS) * sizeof(float)];
+
+constexpr int STATIC_MAX_DEVICES = 64;
+std::mutex g_static_mutex;
+unsigned char *g_static_addr[STATIC_MAX_DEVICES] = {};   // device address of the array, per device
+
+}  // namespace
+
+extern "C" int kt_sync_flat_static(const int32_t *group_of, const int32_t *shares, int K, int G,
+                                   const void *const *grads, int in_dtype, int64_t n, void *out,
+                                   int out_dtype, float scale, void *stream) {
+    if (!group_of || !grads || !out) return fail(KT_ERR_INVALID, "NULL argument");
+    if (K < 1 || K > KT_MAX_RANKS) return fail(KT_ERR_INVALID, "K = %d outside [1, %d]", K, KT_MAX_RANKS);
+    if (G < 1 || G > KT_MAX_GROUPS || G > K) return fail(KT_ERR_INVALID, "G = %d outside [1, min(K, %d)]", G, KT_MAX_GROUPS);
+    if (int rc = check_shares(shares, K)) return rc;
+    if ((in_dtype != KT_F32 && in_dtype != KT_BF16) || (out_dtype != KT_F32 && out_dtype != KT_BF16))
+        return fail(KT_ERR_INVALID, "unknown dtype");
+    if (n < 1) return fail(KT_ERR_INVALID, "n = %lld must be >= 1", static_cast<long long>(n));
+    const int64_t stride = round_up(n, 64);          // elements of one group's partial
+    if (stride * G > KT_STATIC_MAX_ELEMS)
+        return fail(KT_ERR_SHAPE,
+                    "n = %lld with G = %d needs %lld fp32 scratch elements; the static scratch holds %d "
+                    "(use kt_hier_reduce with caller-allocated transport buffers for larger problems)",
+                    static_cast<long long>(n), G, static_cast<long long>(stride * G), KT_STATIC_MAX_ELEMS);
+    const size_t es_in = in_dtype == KT_F32 ? 4 : 2, es_out = out_dtype == KT_F32 ? 4 : 2;
+    if (reinterpret_cast<uintptr_t>(out) % es_out) return fail(KT_ERR_ALIGN, "out is not element aligned");
+
+    // weights, in group-major rank order; everything on the stack
+    int64_t Bg[KT_MAX_GROUPS] = {};
+    int64_t B = 0;
+    for (int r = 0; r < K; ++r) {
+        if (group_of[r] < 0 || group_of[r] >= G) return fail(KT_ERR_INVALID, "group_of[%d] = %d outside [0, %d)", r, group_of[r], G);
+        if (!grads[r]) return fail(KT_ERR_INVALID, "grads[%d] is NULL", r);
+        if (reinterpret_cast<uintptr_t>(grads[r]) % es_in) return fail(KT_ERR_ALIGN, "grads[%d] is not element aligned", r);
+        Bg[group_of[r]] += shares[r];
+        B += shares[r];
+    }
+    for (int g = 0; g < G; ++g)
+        if (!Bg[g]) return fail(KT_ERR_INVALID, "group %d has no rank", g);
+
+    StaticTables tab;
+    std::memset(&tab, 0, sizeof(tab));
+    K1Params p1{};
+    K2Params p2{};
+    p1.rt.K = K;
+    p2.gt.G = G;
+    bool all_aligned = true;
+    int k = 0;
+    for (int g = 0; g < G; ++g) {
+        bool first = true;
+        for (int r = 0; r < K; ++r) {
+            if (group_of[r] != g) continue;
+            p1.rt.coef[k] = static_cast<float>(static_cast<double>(shares[r]) / static_cast<double>(Bg[g]));
+            p1.rt.gid[k] = static_cast<signed char>(g);
+            p1.rt.first[k] = first;
+            p1.rt.last[k] = 0;
+            tab.in_ptrs[k] = grads[r];
+            all_aligned = all_aligned && aligned16(grads[r]);
+            first = false;
+            ++k;
+        }
+        p1.rt.last[k - 1] = 1;
+        p2.gt.W[g] = static_cast<float>(static_cast<double>(Bg[g]) / static_cast<double>(B));
+    }
+    const int n_tiles = static_cast<int>((stride + TILE - 1) / TILE);
+    tab.prefix[0] = 0;
+    tab.prefix[1] = n_tiles;
+    tab.info.dst_off = 0;
+    tab.info.numel = n;
+    tab.info.ext = stride;
+    tab.info.flags = all_aligned ? FLAG_ALIGNED : 0;
+    tab.out_ptr[0] = out;
+    tab.out_aligned[0] = aligned16(out) ? 1 : 0;
+
+    // set-up, once per device: the array's name is only a host-side stand-in; kernels need
+    // the device address the runtime reports for it on the current device
+    int dev = 0;
+    KT_CUDA(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= STATIC_MAX_DEVICES) return fail(KT_ERR_INVALID, "device ordinal %d not supported", dev);
+    unsigned char *scratch = nullptr;
+    {
+        std::lock_guard<std::mutex> lock(g_static_mutex);
+        if (!g_static_addr[dev]) {
+            void *sym = nullptr;
+            KT_CUDA(cudaGetSymbolAddress(&sym, g_static_scratch));
+            g_static_addr[dev] = static_cast<unsigned char *>(sym);
+        }
+        scratch = g_static_addr[dev];
+    }
+
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    // tables: the source is ordinary stack memory, which the runtime stages before returning
+    KT_CUDA(cudaMemcpyAsync(scratch, &tab, sizeof(tab), cudaMemcpyHostToDevice, s));
+
+    TilePlan tp{};
+    tp.prefix = reinterpret_cast<const int *>(scratch + offsetof(StaticTables, prefix));
+    tp.info = reinterpret_cast<const TInfo *>(scratch + offsetof(StaticTables, info));
+    tp.T = 1;
+    tp.u_lo = 0;
+    tp.u_hi = 1;
+    tp.tile_lo = 0;
+    tp.n_tiles = n_tiles;
+    float *partials = reinterpret_cast<float *>(scratch + STATIC_TABLE_BYTES);
+    p1.tp = tp;
+    p1.ptrs = reinterpret_cast<const void *const *>(scratch + offsetof(StaticTables, in_ptrs));
+    p2.tp = tp;
+    p2.out_ptrs = reinterpret_cast<void *const *>(scratch + offsetof(StaticTables, out_ptr));
+    p2.out_aligned = scratch + offsetof(StaticTables, out_aligned);
+    p2.R = 1;
+    p2.scale = scale;
+    for (int g = 0; g < G; ++g) {
+        p1.transport[g] = partials + g * stride;
+        p2.src[g] = partials + g * stride;
+    }
+    // the reduce writes every element of the partials it uses, padding included, so nothing
+    // left over from an earlier call is ever read
+    if (in_dtype == KT_F32) {
+        if (K <= 4) k1_intra_reduce<float, 4><<<n_tiles, NT, 0, s>>>(p1);
+        else k1_intra_reduce<float, 8><<<n_tiles, NT, 0, s>>>(p1);
+    } else {
+        if (K <= 4) k1_intra_reduce<unsigned short, 4><<<n_tiles, NT, 0, s>>>(p1);
+        else k1_intra_reduce<unsigned short, 8><<<n_tiles, NT, 0, s>>>(p1);
+    }
+    KT_CUDA(cudaGetLastError());
+    if (out_dtype == KT_F32) k2_combine_unpack<float><<<n_tiles, NT, 0, s>>>(p2);
+    else k2_combine_unpack<unsigned short><<<n_tiles, NT, 0, s>>>(p2);
+    KT_CUDA(cudaGetLastError());
+    return KT_OK;
+}
