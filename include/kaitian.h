@@ -155,6 +155,19 @@ int kt_hier_reduce(kt_ctx *ctx, int phase, int bucket, float *const *transport, 
 int kt_stage_to_host(kt_ctx *ctx, int dir, int bucket, float *const *transport,
                      float *const *host_pinned, void *main_stream, void *side_stream);
 
+/* The relay of Section III-A as one pipelined call (device -> host RAM -> device): the
+ * bucket's range is cut into chunks of about chunk_bytes; chunk k of every send[g] is copied
+ * to host_pinned[g] on d2h_stream and, as soon as that copy is done, from host_pinned[g] to
+ * recv[g] on h2d_stream, so the two directions of the host link work at the same time.  Both
+ * copy streams first wait for the work queued so far on main_stream.  Completion of the way
+ * down / up is what kt_stage_wait(KT_D2H / KT_H2D, bucket) waits for.
+ * send, host_pinned, recv: host arrays of G pointers (device fp32, pinned host, device fp32),
+ * same element offsets in all three.  chunk_bytes >= 256; the two copy streams must differ.
+ * Errors: KT_ERR_STATE, KT_ERR_SHAPE, KT_ERR_INVALID, KT_ERR_CUDA. */
+int kt_relay_through_host(kt_ctx *ctx, int bucket, float *const *send, float *const *host_pinned,
+                          float *const *recv, int64_t chunk_bytes, void *main_stream,
+                          void *d2h_stream, void *h2d_stream);
+
 /* Makes main_stream wait for the last kt_stage_to_host(dir, bucket).  timeout_ms < 0:
  * returns at once (stream-side wait only).  timeout_ms >= 0: additionally polls the
  * event on the host until it completes or the deadline passes (KT_ERR_TIMEOUT; the copy

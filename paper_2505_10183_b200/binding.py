@@ -25,7 +25,7 @@ KT_MAX_RANKS, KT_MAX_GROUPS = 64, 16
 
 EXPORTS = ["kt_schedule", "kt_groups_init", "kt_set_shares", "kt_set_coefficients",
            "kt_get_coefficients", "kt_bucket_pack", "kt_plan_buckets", "kt_plan_query", "kt_hier_reduce",
-           "kt_stage_to_host", "kt_stage_wait", "kt_unpack_scale", "kt_cast", "kt_copy_tensors", "kt_sync_flat_static", "kt_launch_count",
+           "kt_stage_to_host", "kt_relay_through_host", "kt_stage_wait", "kt_unpack_scale", "kt_cast", "kt_copy_tensors", "kt_sync_flat_static", "kt_launch_count",
            "kt_last_error", "kt_destroy"]
 
 _DTYPES = {torch.float32: KT_F32, torch.bfloat16: KT_BF16}
@@ -57,6 +57,7 @@ def _load() -> C.CDLL:
         "kt_plan_query": ([vp, i32p, i64p, i64p, i64p, i32p, i64p], C.c_int),
         "kt_hier_reduce": ([vp, C.c_int, C.c_int, vpp, vp, vp], C.c_int),
         "kt_stage_to_host": ([vp, C.c_int, C.c_int, vpp, vpp, vp, vp], C.c_int),
+        "kt_relay_through_host": ([vp, C.c_int, vpp, vpp, vpp, C.c_int64, vp, vp, vp], C.c_int),
         "kt_stage_wait": ([vp, C.c_int, C.c_int, vp, C.c_int], C.c_int),
         "kt_unpack_scale": ([vp, vpp, C.c_int, vpp, C.c_int, C.c_int, C.c_float, C.c_int, vp], C.c_int),
         "kt_cast": ([vp, C.c_int, vp, C.c_int, C.c_int64, vp], C.c_int),
@@ -242,6 +243,15 @@ def kt_stage_to_host(ctx: Ctx, direction: int, transport: Ptrs, host_pinned: Ptr
         raise KtError(KT_ERR_SHAPE, "expected %d device and %d host buffers" % (ctx.G, ctx.G))
     _check(_lib.kt_stage_to_host(ctx.handle, int(direction), int(bucket), tr.array, hp.array,
                                  _stream(main_stream), _stream(side_stream)))
+
+
+def kt_relay_through_host(ctx: Ctx, send: Ptrs, host_pinned: Ptrs, recv: Ptrs, d2h_stream, h2d_stream,
+                          bucket: int = -1, chunk_bytes: int = 4 << 20, main_stream=None) -> None:
+    sd, hp, rv = kt_ptrs(send), kt_ptrs(host_pinned), kt_ptrs(recv)
+    if sd.n != ctx.G or hp.n != ctx.G or rv.n != ctx.G:
+        raise KtError(KT_ERR_SHAPE, "expected %d buffers in every list" % ctx.G)
+    _check(_lib.kt_relay_through_host(ctx.handle, int(bucket), sd.array, hp.array, rv.array, int(chunk_bytes),
+                                      _stream(main_stream), _stream(d2h_stream), _stream(h2d_stream)))
 
 
 def kt_stage_wait(ctx: Ctx, direction: int, bucket: int = -1, main_stream=None, timeout_ms: int = -1) -> None:

@@ -71,6 +71,7 @@ struct kt_ctx {
     bool planned = false;
     int T = 0;
     int in_dtype = KT_F32;
+    int tile = TILE_F32;                             // elements per work unit (by gradient dtype)
     std::vector<int64_t> numel, tensor_offset;       // user tensor order
     std::vector<int32_t> bucket_of;
     std::vector<int64_t> bucket_start, bucket_numel;
@@ -91,6 +92,7 @@ struct kt_ctx {
 
     cudaEvent_t ev_main = nullptr;
     std::vector<StageSlot> slots[2]; // per direction: index 0 = all buckets, 1 + b = bucket b
+    std::vector<cudaEvent_t> chunk_events;   // chunk k went down: its way up may start
     int64_t launches = 0;
     std::vector<std::pair<const void *, int>> occupancy;   // resident CTAs per SM, per kernel
 };
@@ -205,6 +207,7 @@ int make_tile_plan(const kt_ctx *c, int bucket, TilePlan *tp) {
     tp->u_hi = bucket < 0 ? c->T : c->bucket_u_hi[bucket];
     tp->tile_lo = c->prefix[tp->u_lo];
     tp->n_tiles = c->prefix[tp->u_hi] - tp->tile_lo;
+    tp->tile = c->tile;
     return KT_OK;
 }
 
@@ -244,6 +247,16 @@ int launch_k1(kt_ctx *c, const K1Params &p, cudaStream_t s) {
     c->launches += 1;
     KT_CUDA(cudaGetLastError());
     return KT_OK;
+}
+
+// combine + unpack: the tile size is the plan's (fixed by the gradient dtype), the vector
+// width follows the output dtype
+template <typename Tout>
+void launch_k2(int tile, int n_tiles, cudaStream_t s, const K2Params &p) {
+    if (tile == TILE_F32)
+        k2_combine_unpack<Tout, TILE_F32><<<n_tiles, NT, 0, s>>>(p);
+    else
+        k2_combine_unpack<Tout, TILE_BF16><<<n_tiles, NT, 0, s>>>(p);
 }
 
 }  // namespace
@@ -399,6 +412,7 @@ int kt_bucket_pack(kt_ctx *c, const void *const *grads, const int64_t *numel, in
     const int nb = static_cast<int>(bstart.size());
 
     // ---- tile tables in transport order
+    const int tile = in_dtype == KT_F32 ? TILE_F32 : TILE_BF16;
     std::vector<int> prefix(T + 1, 0);
     std::vector<TInfo> info(T);
     for (int u = 0; u < T; ++u) {
@@ -412,7 +426,7 @@ int kt_bucket_pack(kt_ctx *c, const void *const *grads, const int64_t *numel, in
         ti.pad_ = 0;
         for (int r = 0; r < c->K; ++r)
             if (!aligned16(grads[static_cast<size_t>(r) * T + t])) ti.flags = 0;
-        const int64_t tiles = (ti.ext + TILE - 1) / TILE;
+        const int64_t tiles = (ti.ext + tile - 1) / tile;
         if (prefix[u] + tiles > 0x7FFFFFF0LL) return fail(KT_ERR_SHAPE, "too many elements for one plan");
         prefix[u + 1] = prefix[u] + static_cast<int>(tiles);
     }
@@ -448,6 +462,7 @@ int kt_bucket_pack(kt_ctx *c, const void *const *grads, const int64_t *numel, in
 
     c->T = T;
     c->in_dtype = in_dtype;
+    c->tile = tile;
     c->numel.assign(numel, numel + T);
     c->tensor_offset = offset;
     c->bucket_of = bof;
@@ -595,6 +610,50 @@ int kt_stage_to_host(kt_ctx *c, int dir, int bucket, float *const *transport, fl
     return KT_OK;
 }
 
+int kt_relay_through_host(kt_ctx *c, int bucket, float *const *send, float *const *host_pinned,
+                          float *const *recv, int64_t chunk_bytes, void *main_stream, void *d2h_stream,
+                          void *h2d_stream) {
+    if (int rc = check_ctx(c, true)) return rc;
+    if (!send || !host_pinned || !recv) return fail(KT_ERR_INVALID, "NULL argument");
+    if (bucket < -1 || bucket >= static_cast<int>(c->bucket_start.size()))
+        return fail(KT_ERR_SHAPE, "bucket %d out of range", bucket);
+    if (chunk_bytes < 256) return fail(KT_ERR_INVALID, "chunk_bytes must be >= 256");
+    if (d2h_stream == h2d_stream) return fail(KT_ERR_INVALID, "the two copy streams must differ");
+    for (int g = 0; g < c->G; ++g)
+        if (!send[g] || !host_pinned[g] || !recv[g]) return fail(KT_ERR_INVALID, "buffer %d is NULL", g);
+    int64_t lo, n;
+    bucket_range(c, bucket, &lo, &n);
+    const int64_t chunk = chunk_bytes / 256 * 64;                 // elements, a multiple of 64
+    const int64_t n_chunks = (n + chunk - 1) / chunk;
+    KT_CUDA(cudaSetDevice(c->device));
+    while (static_cast<int64_t>(c->chunk_events.size()) < n_chunks) {
+        cudaEvent_t e;
+        KT_CUDA(cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
+        c->chunk_events.push_back(e);
+    }
+    cudaStream_t ms = static_cast<cudaStream_t>(main_stream);
+    cudaStream_t ds = static_cast<cudaStream_t>(d2h_stream), hs = static_cast<cudaStream_t>(h2d_stream);
+    KT_CUDA(cudaEventRecord(c->ev_main, ms));
+    KT_CUDA(cudaStreamWaitEvent(ds, c->ev_main, 0));
+    KT_CUDA(cudaStreamWaitEvent(hs, c->ev_main, 0));
+    for (int64_t k = 0; k < n_chunks; ++k) {
+        const int64_t at = lo + k * chunk;
+        const size_t len = static_cast<size_t>((k + 1 < n_chunks ? chunk : n - k * chunk)) * sizeof(float);
+        for (int g = 0; g < c->G; ++g)
+            KT_CUDA(cudaMemcpyAsync(host_pinned[g] + at, send[g] + at, len, cudaMemcpyDeviceToHost, ds));
+        KT_CUDA(cudaEventRecord(c->chunk_events[k], ds));
+        KT_CUDA(cudaStreamWaitEvent(hs, c->chunk_events[k], 0));
+        for (int g = 0; g < c->G; ++g)
+            KT_CUDA(cudaMemcpyAsync(recv[g] + at, host_pinned[g] + at, len, cudaMemcpyHostToDevice, hs));
+    }
+    StageSlot &down = c->slots[KT_D2H][bucket + 1], &up = c->slots[KT_H2D][bucket + 1];
+    KT_CUDA(cudaEventRecord(down.done, ds));
+    down.recorded = true;
+    KT_CUDA(cudaEventRecord(up.done, hs));
+    up.recorded = true;
+    return KT_OK;
+}
+
 int kt_stage_wait(kt_ctx *c, int dir, int bucket, void *main_stream, int timeout_ms) {
     if (int rc = check_ctx(c, true)) return rc;
     if (dir != KT_D2H && dir != KT_H2D) return fail(KT_ERR_INVALID, "unknown direction %d", dir);
@@ -689,9 +748,9 @@ int kt_unpack_scale(kt_ctx *c, const float *const *src, int from_combined, void 
     p.R = R;
     p.scale = scale;
     if (out_dtype == KT_F32)
-        k2_combine_unpack<float><<<tp.n_tiles, NT, 0, s>>>(p);
+        launch_k2<float>(tp.tile, tp.n_tiles, s, p);
     else
-        k2_combine_unpack<unsigned short><<<tp.n_tiles, NT, 0, s>>>(p);
+        launch_k2<unsigned short>(tp.tile, tp.n_tiles, s, p);
     c->launches += 1;
     KT_CUDA(cudaGetLastError());
     return KT_OK;
@@ -754,6 +813,7 @@ void kt_destroy(kt_ctx *c) {
     for (int dir = 0; dir < 2; ++dir)
         for (auto &s : c->slots[dir])
             if (s.done) cudaEventDestroy(s.done);
+    for (cudaEvent_t e : c->chunk_events) cudaEventDestroy(e);
     delete c;
 }
 
@@ -844,7 +904,8 @@ extern "C" int kt_sync_flat_static(const int32_t *group_of, const int32_t *share
         p1.rt.last[k - 1] = 1;
         p2.gt.W[g] = static_cast<float>(static_cast<double>(Bg[g]) / static_cast<double>(B));
     }
-    const int n_tiles = static_cast<int>((stride + TILE - 1) / TILE);
+    const int tile = in_dtype == KT_F32 ? TILE_F32 : TILE_BF16;
+    const int n_tiles = static_cast<int>((stride + tile - 1) / tile);
     tab.prefix[0] = 0;
     tab.prefix[1] = n_tiles;
     tab.info.dst_off = 0;
@@ -882,6 +943,7 @@ extern "C" int kt_sync_flat_static(const int32_t *group_of, const int32_t *share
     tp.u_hi = 1;
     tp.tile_lo = 0;
     tp.n_tiles = n_tiles;
+    tp.tile = tile;
     float *partials = reinterpret_cast<float *>(scratch + STATIC_TABLE_BYTES);
     p1.tp = tp;
     p1.ptrs = reinterpret_cast<const void *const *>(scratch + offsetof(StaticTables, in_ptrs));
@@ -904,8 +966,8 @@ extern "C" int kt_sync_flat_static(const int32_t *group_of, const int32_t *share
         else k1_intra_reduce<unsigned short, 8><<<n_tiles, NT, 0, s>>>(p1);
     }
     KT_CUDA(cudaGetLastError());
-    if (out_dtype == KT_F32) k2_combine_unpack<float><<<n_tiles, NT, 0, s>>>(p2);
-    else k2_combine_unpack<unsigned short><<<n_tiles, NT, 0, s>>>(p2);
+    if (out_dtype == KT_F32) launch_k2<float>(tile, n_tiles, s, p2);
+    else launch_k2<unsigned short>(tile, n_tiles, s, p2);
     KT_CUDA(cudaGetLastError());
     return KT_OK;
 }

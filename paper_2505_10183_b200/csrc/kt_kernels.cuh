@@ -22,7 +22,10 @@
 namespace {
 
 constexpr int NT = 256;          // threads per CTA
-constexpr int TILE = 2048;       // transport elements per work unit
+// transport elements per work unit (one CTA each): chosen by the gradient dtype so that every
+// thread has two 16-byte loads per rank in flight
+constexpr int TILE_F32 = 2048;
+constexpr int TILE_BF16 = 4096;
 constexpr int FLAG_ALIGNED = 1;  // all K sources of the tensor are 16-byte aligned
 
 // ------------------------------------------------------------------ device tables
@@ -54,6 +57,7 @@ struct TilePlan {         // which tiles a launch covers and how to decode them
     int u_lo, u_hi;       // tensors [u_lo, u_hi) take part
     int tile_lo;          // prefix[u_lo]
     int n_tiles;          // prefix[u_hi] - prefix[u_lo]
+    int tile;             // elements per tile the prefix was built for
 };
 
 struct K1Params {
@@ -105,6 +109,7 @@ __device__ __forceinline__ unsigned pack_bf16x2(float lo, float hi) {
 template <typename T> struct Elem;
 template <> struct Elem<float> {
     static constexpr int VEC = 4;   // elements per 16-byte vector
+    static constexpr int TILE = TILE_F32;
     __device__ static __forceinline__ void unpack(const uint4 &v, float (&x)[4]) {
         x[0] = __uint_as_float(v.x); x[1] = __uint_as_float(v.y);
         x[2] = __uint_as_float(v.z); x[3] = __uint_as_float(v.w);
@@ -124,6 +129,7 @@ template <> struct Elem<float> {
 };
 template <> struct Elem<unsigned short> {
     static constexpr int VEC = 8;
+    static constexpr int TILE = TILE_BF16;
     __device__ static __forceinline__ void unpack(const uint4 &v, float (&x)[8]) {
         // bf16 is the upper half of a binary32: widening is a shift
         x[0] = __uint_as_float(v.x << 16); x[1] = __uint_as_float(v.x & 0xFFFF0000u);
@@ -175,7 +181,7 @@ __device__ __forceinline__ TileRef locate_tile(const TilePlan &tp) {
     r.ti.ext = (static_cast<long long>(b.y) << 32) | static_cast<unsigned>(b.x);
     r.ti.flags = b.z;
     r.ti.pad_ = 0;
-    r.e0 = static_cast<long long>(tile - __ldg(tp.prefix + lo)) * TILE;
+    r.e0 = static_cast<long long>(tile - __ldg(tp.prefix + lo)) * tp.tile;
     return r;
 }
 
@@ -184,6 +190,7 @@ __device__ __forceinline__ TileRef locate_tile(const TilePlan &tp) {
 template <typename Tin, int KB, bool EDGE>
 __device__ __forceinline__ void k1_tile(const K1Params &p, const TileRef &t) {
     constexpr int VEC = Elem<Tin>::VEC;
+    constexpr int TILE = Elem<Tin>::TILE;
     constexpr int ITERS = TILE / (NT * VEC);
     const int K = p.rt.K;
     const int T = p.tp.T;
@@ -246,7 +253,7 @@ __device__ __forceinline__ void k1_tile(const K1Params &p, const TileRef &t) {
 template <typename Tin, int KB>
 __global__ void __launch_bounds__(NT) k1_intra_reduce(const __grid_constant__ K1Params p) {
     const TileRef t = locate_tile(p.tp);
-    if ((t.ti.flags & FLAG_ALIGNED) && t.e0 + TILE <= t.ti.numel)
+    if ((t.ti.flags & FLAG_ALIGNED) && t.e0 + Elem<Tin>::TILE <= t.ti.numel)
         k1_tile<Tin, KB, false>(p, t);
     else
         k1_tile<Tin, KB, true>(p, t);
@@ -254,7 +261,7 @@ __global__ void __launch_bounds__(NT) k1_intra_reduce(const __grid_constant__ K1
 
 // ------------------------------------------------------------------ K2: inter-group combine + scale + cast + unpack
 // out_c^(u)[e] = cast(scale * sum_g W_g P_g[off_u + e]) for every copy c < R.
-template <typename Tout, bool EDGE>
+template <typename Tout, int TILE, bool EDGE>
 __device__ __forceinline__ void k2_tile(const K2Params &p, const TileRef &t) {
     constexpr int VEC = Elem<Tout>::VEC;
     constexpr int ITERS = TILE / (NT * VEC);
@@ -311,13 +318,13 @@ __device__ __forceinline__ void k2_tile(const K2Params &p, const TileRef &t) {
     }
 }
 
-template <typename Tout>
+template <typename Tout, int TILE>
 __global__ void __launch_bounds__(NT) k2_combine_unpack(const __grid_constant__ K2Params p) {
     const TileRef t = locate_tile(p.tp);
     if (p.out_aligned[t.u] && t.e0 + TILE <= t.ti.numel)
-        k2_tile<Tout, false>(p, t);
+        k2_tile<Tout, TILE, false>(p, t);
     else
-        k2_tile<Tout, true>(p, t);
+        k2_tile<Tout, TILE, true>(p, t);
 }
 
 // ------------------------------------------------------------------ flat inter-group combine into a combined buffer
@@ -344,6 +351,7 @@ __global__ void __launch_bounds__(NT) k_combine_flat(const __grid_constant__ K2P
 template <typename Tin>
 __global__ void __launch_bounds__(NT) k_pack(const __grid_constant__ PackParams p) {
     constexpr int VEC = Elem<Tin>::VEC;
+    constexpr int TILE = Elem<Tin>::TILE;
     constexpr int ITERS = TILE / (NT * VEC);
     const TileRef t = locate_tile(p.tp);
     const int k = blockIdx.y;
