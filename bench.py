@@ -307,9 +307,10 @@ def run_ours(args) -> dict:
     return result if rank == 0 else None
 
 
-# ncu dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel; null
-# until captured for the kernel as it stands (see profiles/).
-TRAFFIC_K1 = {}
+# ncu dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, captured
+# for the kernel as it stands (profiles/k1_k2_resnet18.md); a workload without a capture
+# reports null.
+TRAFFIC_K1 = {"resnet18": 216822784}
 
 
 def run_e2e(prob, kt, args, barrier) -> dict:

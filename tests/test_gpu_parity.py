@@ -83,12 +83,23 @@ def test_schedule_matches_oracle_and_named_values(kt, oracle):
 
 
 def test_resnet18_staged_as_benchmarked(kt, oracle):
-    """Full size, bucket by bucket, partials relayed through pinned host memory: the launch
-    configuration the benchmark times."""
+    """Full size, in the launch configuration the benchmark times: one fused-reduce launch,
+    the partials relayed bucket by bucket through pinned host memory as a chunk pipeline, one
+    combine/unpack launch.  Every element is compared."""
     wl = W.resnet18()
-    host, out, shares = compare_all(kt, oracle, wl, per_bucket=True, staged=True)
+    host, out, shares = compare_all(kt, oracle, wl, staged="relay")
     assert shares == [79, 79, 49, 49]
     check_tolerance(oracle, wl, host, out, shares)
+    # odd chunk sizes: ragged last chunk, chunk larger than a bucket
+    compare_all(kt, oracle, wl, staged="relay", relay_chunk=(1 << 20) + 256)
+    compare_all(kt, oracle, wl, staged="relay", relay_chunk=1 << 30)
+
+
+def test_resnet18_staged_bucket_by_bucket(kt, oracle):
+    """The per-bucket route: reduce, copy down, copy up and unpack one bucket at a time."""
+    wl = W.resnet18()
+    compare_all(kt, oracle, wl, per_bucket=True, staged=True)
+    compare_all(kt, oracle, W.tiny(), staged="relay", relay_chunk=256)
 
 
 def test_resnet18_single_launch(kt, oracle):
