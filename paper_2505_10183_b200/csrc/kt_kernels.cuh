@@ -21,11 +21,23 @@
 
 namespace {
 
-constexpr int NT = 256;          // threads per CTA
+#ifndef KT_NT
+#define KT_NT 256
+#endif
+#ifndef KT_ITERS
+#define KT_ITERS 2
+#endif
+#ifndef KT_KB
+#define KT_KB 4                  /* ranks whose loads are issued together */
+#endif
+#ifndef KT_WARM_CTAS
+#define KT_WARM_CTAS 1184        /* about two waves: CTAs that prefetch the tables into L2 */
+#endif
+constexpr int NT = KT_NT;        // threads per CTA
 // transport elements per work unit (one CTA each): chosen by the gradient dtype so that every
-// thread has two 16-byte loads per rank in flight
-constexpr int TILE_F32 = 2048;
-constexpr int TILE_BF16 = 4096;
+// thread has KT_ITERS 16-byte loads per rank in flight
+constexpr int TILE_F32 = NT * 4 * KT_ITERS;
+constexpr int TILE_BF16 = NT * 8 * KT_ITERS;
 constexpr int FLAG_ALIGNED = 1;  // all K sources of the tensor are 16-byte aligned
 
 // ------------------------------------------------------------------ device tables
@@ -58,6 +70,8 @@ struct TilePlan {         // which tiles a launch covers and how to decode them
     int tile_lo;          // prefix[u_lo]
     int n_tiles;          // prefix[u_hi] - prefix[u_lo]
     int tile;             // elements per tile the prefix was built for
+    const void *tables;   // start of the table allocation (prefix, records, pointers) ...
+    int table_bytes;      // ... and how much of it is worth prefetching (0: nothing)
 };
 
 struct K1Params {
@@ -65,6 +79,7 @@ struct K1Params {
     const void *const *ptrs;           // [K][T] device pointer table
     float *transport[KT_MAX_GROUPS];
     RankTab rt;
+    int wide;                          // every transport base is 32-byte aligned
 };
 
 struct K2Params {
@@ -75,6 +90,7 @@ struct K2Params {
     const unsigned char *out_aligned;  // [T] all R destinations 16-byte aligned
     int R;
     float scale;
+    int wide;                          // every source base is 32-byte aligned
 };
 
 struct PackParams {
@@ -104,6 +120,35 @@ __device__ __forceinline__ unsigned pack_bf16x2(float lo, float hi) {
     unsigned d;   // round-to-nearest-even narrowing of two floats; hi lands in the upper half
     asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
     return d;
+}
+
+// VEC consecutive floats to / from the transport.  Eight floats go as one 256-bit access when
+// the buffers allow it (32-byte aligned bases), so that every access covers whole 32-byte
+// sectors; otherwise as two 128-bit accesses.
+template <int VEC>
+__device__ __forceinline__ void store_vec(float *d, const float (&a)[VEC], bool wide) {
+    if (VEC == 8 && wide) {
+        asm volatile("st.global.v8.f32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(d), "f"(a[0]), "f"(a[1]),
+                     "f"(a[2]), "f"(a[3]), "f"(a[4 % VEC]), "f"(a[5 % VEC]), "f"(a[6 % VEC]), "f"(a[7 % VEC])
+                     : "memory");
+    } else {
+#pragma unroll
+        for (int q = 0; q < VEC / 4; ++q)
+            reinterpret_cast<float4 *>(d)[q] = make_float4(a[4 * q], a[4 * q + 1], a[4 * q + 2], a[4 * q + 3]);
+    }
+}
+
+template <int Q>
+__device__ __forceinline__ void load_vec(const float *s, float4 (&v)[Q], bool wide) {
+    if (Q == 2 && wide) {
+        asm volatile("ld.global.nc.L1::no_allocate.v8.f32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                     : "=f"(v[0].x), "=f"(v[0].y), "=f"(v[0].z), "=f"(v[0].w), "=f"(v[Q - 1].x), "=f"(v[Q - 1].y),
+                       "=f"(v[Q - 1].z), "=f"(v[Q - 1].w)
+                     : "l"(s));
+    } else {
+#pragma unroll
+        for (int q = 0; q < Q; ++q) v[q] = __ldcs(reinterpret_cast<const float4 *>(s) + q);
+    }
 }
 
 template <typename T> struct Elem;
@@ -163,15 +208,25 @@ struct TileRef {
     long long e0;
 };
 
-// Tile -> tensor: largest u with prefix[u] <= tile (prefix is non-decreasing, its last entry
-// exceeds every tile of the launch).  Uniform across the CTA; the few words it reads stay in L1.
+// Tile -> tensor: the u with prefix[u] <= tile < prefix[u + 1] (prefix is non-decreasing, so
+// empty tensors never match).  One memory round trip: thread i tests tensor u_lo + i (in
+// strides of the CTA when there are more tensors than threads), the one that matches
+// publishes it through shared memory.  The first CTAs of a launch also pull the small tables
+// into L2 up front, so that the dependent look-ups that follow (record, pointers) do not
+// each wait for DRAM while the machine is still empty.
 __device__ __forceinline__ TileRef locate_tile(const TilePlan &tp) {
+    __shared__ int s_u;
     const int tile = blockIdx.x + tp.tile_lo;
-    int lo = tp.u_lo, hi = tp.u_hi;
-    while (hi - lo > 1) {
-        const int mid = (lo + hi) >> 1;
-        if (__ldg(tp.prefix + mid) <= tile) lo = mid; else hi = mid;
+    if (blockIdx.x < KT_WARM_CTAS) {
+        const char *line = static_cast<const char *>(tp.tables) + 128 * threadIdx.x;
+        if (128 * threadIdx.x < tp.table_bytes) asm volatile("prefetch.global.L2 [%0];" ::"l"(line));
     }
+    for (int u = tp.u_lo + threadIdx.x; u < tp.u_hi; u += NT) {
+        const int a = __ldg(tp.prefix + u), b = __ldg(tp.prefix + u + 1);
+        if (a <= tile && tile < b) s_u = u;
+    }
+    __syncthreads();
+    const int lo = s_u;
     TileRef r;
     r.u = lo;
     const int4 *rec = reinterpret_cast<const int4 *>(tp.info + lo);
@@ -238,11 +293,7 @@ __device__ __forceinline__ void k1_tile(const K1Params &p, const TileRef &t) {
                             for (int c = 0; c < VEC; ++c)   // padding is +0 whatever the weights
                                 if (e[it] + c >= t.ti.numel) acc[it][c] = 0.f;
                         }
-                        float4 *dv = reinterpret_cast<float4 *>(d + e[it]);
-#pragma unroll
-                        for (int q = 0; q < VEC / 4; ++q)
-                            dv[q] = make_float4(acc[it][4 * q], acc[it][4 * q + 1], acc[it][4 * q + 2],
-                                                acc[it][4 * q + 3]);
+                        store_vec<VEC>(d + e[it], acc[it], p.wide);
                     }
                 }
             }
@@ -280,11 +331,12 @@ __device__ __forceinline__ void k2_tile(const K2Params &p, const TileRef &t) {
         float4 v[ITERS][Q];
 #pragma unroll
         for (int it = 0; it < ITERS; ++it) {
+            // the transport holds ext elements per tensor, so a vector below ext is readable
+            if (!EDGE || e[it] < t.ti.ext) {
+                load_vec<Q>(s + e[it], v[it], p.wide);
+            } else {
 #pragma unroll
-            for (int q = 0; q < Q; ++q) {
-                // the transport holds ext elements per tensor, so a vector below ext is readable
-                if (!EDGE || e[it] < t.ti.ext) v[it][q] = __ldcs(reinterpret_cast<const float4 *>(s + e[it]) + q);
-                else v[it][q] = make_float4(0.f, 0.f, 0.f, 0.f);
+                for (int q = 0; q < Q; ++q) v[it][q] = make_float4(0.f, 0.f, 0.f, 0.f);
             }
         }
 #pragma unroll
