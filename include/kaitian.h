@@ -156,7 +156,8 @@ int kt_stage_to_host(kt_ctx *ctx, int dir, int bucket, float *const *transport,
                      float *const *host_pinned, void *main_stream, void *side_stream);
 
 /* The relay of Section III-A as one pipelined call (device -> host RAM -> device): the
- * bucket's range is cut into chunks of about chunk_bytes; chunk k of every send[g] is copied
+ * bucket's range is cut into chunks of chunk_bytes (a few MiB works best; very small chunks
+ * use the host link badly); chunk k of every send[g] is copied
  * to host_pinned[g] on d2h_stream and, as soon as that copy is done, from host_pinned[g] to
  * recv[g] on h2d_stream, so the two directions of the host link work at the same time.  Both
  * copy streams first wait for the work queued so far on main_stream.  Completion of the way

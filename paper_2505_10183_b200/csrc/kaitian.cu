@@ -635,8 +635,12 @@ int kt_relay_through_host(kt_ctx *c, int bucket, float *const *send, float *cons
         if (!send[g] || !host_pinned[g] || !recv[g]) return fail(KT_ERR_INVALID, "buffer %d is NULL", g);
     int64_t lo, n;
     bucket_range(c, bucket, &lo, &n);
-    const int64_t chunk = chunk_bytes / 256 * 64;                 // elements, a multiple of 64
-    const int64_t n_chunks = (n + chunk - 1) / chunk;
+    // Uniform chunks (elements, a multiple of 64).  Shorter chunks at the two ends of the
+    // pipeline were tried and measured slower: small copies use the host link badly.
+    const int64_t chunk = chunk_bytes / 256 * 64;
+    std::vector<int64_t> sizes;
+    for (int64_t left = n; left > 0; left -= sizes.back()) sizes.push_back(left < chunk ? left : chunk);
+    const int64_t n_chunks = static_cast<int64_t>(sizes.size());
     KT_CUDA(cudaSetDevice(c->device));
     while (static_cast<int64_t>(c->chunk_events.size()) < n_chunks) {
         cudaEvent_t e;
@@ -648,9 +652,9 @@ int kt_relay_through_host(kt_ctx *c, int bucket, float *const *send, float *cons
     KT_CUDA(cudaEventRecord(c->ev_main, ms));
     KT_CUDA(cudaStreamWaitEvent(ds, c->ev_main, 0));
     KT_CUDA(cudaStreamWaitEvent(hs, c->ev_main, 0));
-    for (int64_t k = 0; k < n_chunks; ++k) {
-        const int64_t at = lo + k * chunk;
-        const size_t len = static_cast<size_t>((k + 1 < n_chunks ? chunk : n - k * chunk)) * sizeof(float);
+    int64_t at = lo;
+    for (int64_t k = 0; k < n_chunks; at += sizes[k], ++k) {
+        const size_t len = static_cast<size_t>(sizes[k]) * sizeof(float);
         for (int g = 0; g < c->G; ++g)
             KT_CUDA(cudaMemcpyAsync(host_pinned[g] + at, send[g] + at, len, cudaMemcpyDeviceToHost, ds));
         KT_CUDA(cudaEventRecord(c->chunk_events[k], ds));

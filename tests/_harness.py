@@ -56,14 +56,15 @@ def run_gpu_path(kt, wl, dev_grads, shares, out_dtype=None, R=1, scale=1.0, per_
         recv = [torch.full((n,), float("nan"), device="cuda") for _ in range(wl.G)]
         side = torch.cuda.Stream()
         src = recv
-    if staged == "relay":
+    if staged in ("relay", "relay_all"):
         # the benchmark's launch configuration: one fused-reduce launch over all buckets, the
         # relay bucket by bucket as a chunk pipeline on two copy streams, one combine/unpack launch
         side2 = torch.cuda.Stream()
         kt.kt_hier_reduce(ctx, kt.KT_INTRA, transport, bucket=-1)
-        for b in range(plan.n_buckets):
+        relay_buckets = [-1] if staged == "relay_all" else list(range(plan.n_buckets))
+        for b in relay_buckets:
             kt.kt_relay_through_host(ctx, transport, host, recv, side, side2, bucket=b, chunk_bytes=relay_chunk)
-        for b in range(plan.n_buckets):
+        for b in relay_buckets:
             kt.kt_stage_wait(ctx, kt.KT_H2D, bucket=b)
         kt.kt_unpack_scale(ctx, recv, out, scale=scale, bucket=-1)
         torch.cuda.synchronize()

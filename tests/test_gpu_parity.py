@@ -87,11 +87,12 @@ def test_resnet18_staged_as_benchmarked(kt, oracle):
     the partials relayed bucket by bucket through pinned host memory as a chunk pipeline, one
     combine/unpack launch.  Every element is compared."""
     wl = W.resnet18()
-    host, out, shares = compare_all(kt, oracle, wl, staged="relay")
+    host, out, shares = compare_all(kt, oracle, wl, staged="relay_all", relay_chunk=4 << 20)
     assert shares == [79, 79, 49, 49]
     check_tolerance(oracle, wl, host, out, shares)
-    # odd chunk sizes: ragged last chunk, chunk larger than a bucket
-    compare_all(kt, oracle, wl, staged="relay", relay_chunk=(1 << 20) + 256)
+    # the relay bucket by bucket, and odd chunk sizes: ragged last chunk, chunk larger than a bucket
+    compare_all(kt, oracle, wl, staged="relay")
+    compare_all(kt, oracle, wl, staged="relay_all", relay_chunk=(1 << 20) + 256)
     compare_all(kt, oracle, wl, staged="relay", relay_chunk=1 << 30)
 
 

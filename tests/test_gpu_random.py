@@ -68,7 +68,7 @@ def run_case(kt, oracle, rnd):
     elif route == "combined":
         kw.update(use_combined=True, per_bucket=rnd.random() < 0.5)
     elif route == "relay":
-        kw.update(staged="relay", relay_chunk=rnd.choice([256, 1024, 65536, 1 << 22]))
+        kw.update(staged=rnd.choice(["relay", "relay_all"]), relay_chunk=rnd.choice([256, 1024, 65536, 1 << 19, 1 << 22]))
     elif route == "staged_buckets":
         kw.update(staged=True, per_bucket=True)
     out, transport, plan, ctx = H.run_gpu_path(kt, wl, dev, wl.shares, **kw)
