@@ -116,22 +116,48 @@ class ClockSampler:
 class Problem:
     """Device state of one replica: gradients, context, transport / receive / pinned buffers."""
 
-    def __init__(self, wl, kt, device_values: bool = True, chunk_bytes: int = 4 << 20):
+    def __init__(self, wl, kt, device_values: bool = True, chunk_bytes: int = 4 << 20, arena: bool = False):
+        """arena=False: every gradient and output tensor is its own allocation (as per-parameter
+        gradients are).  arena=True: the tensors of one rank are views into one buffer, each at
+        a multiple of 64 elements, so that a whole rank moves between host and device in one
+        copy (the end-to-end arm)."""
         self.wl, self.kt = wl, kt
         self.chunk_bytes = chunk_bytes
         self.shares = list(wl.shares) if wl.shares is not None else kt.kt_schedule(wl.step_times, wl.global_batch)
         dt = torch.float32 if wl.dtype == "f32" else torch.bfloat16
         self.grads = []
+        starts, pos = [], 0
+        for m in wl.numel:
+            starts.append(pos)
+            pos += -(-m // 64) * 64
+        self.arena_numel = pos
+
+        def views(buf):
+            return [buf[s:s + m] for s, m in zip(starts, wl.numel)]
+
+        self.grad_arenas = []
         for r in range(wl.K):
             flat = W.rank_gradients(wl, r, "cuda" if device_values else "cpu")
-            self.grads.append([t.cuda() for t in W.split_tensors(flat, wl.numel)])
+            if arena:
+                buf = torch.zeros(self.arena_numel, dtype=dt, device="cuda")
+                row = views(buf)
+                for dst, src in zip(row, W.split_tensors(flat, wl.numel)):
+                    dst.copy_(src)
+                self.grad_arenas.append(buf)
+                self.grads.append(row)
+            else:
+                self.grads.append([t.cuda() for t in W.split_tensors(flat, wl.numel)])
             del flat
         self.ctx = kt.kt_groups_init(wl.group_of, self.shares, wl.G)
         kt.kt_bucket_pack(self.ctx, self.grads, wl.bucket_cap_bytes)
         self.plan = kt.kt_plan_query(self.ctx)
         n = self.plan.transport_numel
         self.transport = kt.kt_ptrs([torch.zeros(n, device="cuda") for _ in range(wl.G)])
-        self.out = [[torch.zeros(m, dtype=dt, device="cuda") for m in wl.numel]]
+        if arena:
+            self.out_arena = torch.zeros(self.arena_numel, dtype=dt, device="cuda")
+            self.out = [views(self.out_arena)]
+        else:
+            self.out = [[torch.zeros(m, dtype=dt, device="cuda") for m in wl.numel]]
         self.out_ptrs = kt.kt_ptrs([t for c in self.out for t in c])
         self.out_dtype = kt.KT_F32 if wl.dtype == "f32" else kt.KT_BF16
         self.main = torch.cuda.Stream()
@@ -222,7 +248,7 @@ def run_ours(args) -> dict:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
 
     wl = W.by_name(args.workload)
-    prob = Problem(wl, kt)
+    prob = Problem(wl, kt, chunk_bytes=args_chunk(args))
     nbytes = algorithmic_bytes(wl)
     link = host_link_bandwidth() if wl.staged else None
 
@@ -302,7 +328,9 @@ def run_ours(args) -> dict:
                      "traffic": TRAFFIC_K1.get(wl.name)},
         "e2e": {"value": round(job_throughput(nbytes["step"], args.steps, world, e2e["seconds"]), 2), "unit": UNIT,
                 "h2d_bytes_per_step": e2e["h2d"], "d2h_bytes_per_step": e2e["d2h"],
-                "ms_per_step": round(e2e["seconds"] / args.steps * 1e3, 4)},
+                "ms_per_step": round(e2e["seconds"] / args.steps * 1e3, 4),
+                "layout": "one pinned host buffer and one device buffer per rank, tensors at multiples of "
+                          "64 elements (views): K copies in, 1 copy out, through kt_copy_tensors"},
         "gpu_launches": int(launches),
         "clocks": clocks,
     }
@@ -322,20 +350,28 @@ def run_ours(args) -> dict:
 TRAFFIC_K1 = {"resnet18": 217354496}
 
 
+def args_chunk(args) -> int:
+    return int(getattr(args, "relay_chunk_mib", 4)) << 20
+
+
 def run_e2e(prob, kt, args, barrier) -> dict:
     """Same step, but every step first copies all ranks' gradients from pinned host memory
     to the device and ends with the reduced gradients copied back to pinned host memory."""
-    wl = prob.wl
-    host_in = [[t.cpu().pin_memory() for t in row] for row in prob.grads]
-    host_out = [torch.empty(t.shape, dtype=t.dtype).pin_memory() for t in prob.out[0]]
-    dst = kt.kt_ptrs([t for row in prob.grads for t in row])
-    src = kt.kt_ptrs([t for row in host_in for t in row])
+    # Host side: one pinned buffer per rank holding that rank's tensors, each at a multiple of
+    # 64 elements; device side: the same layout, the per-parameter tensors being views.  A rank
+    # then crosses the host link in one copy instead of one per tensor (with hundreds of small
+    # tensors the per-copy cost would otherwise dominate).
     import ctypes
-    sizes = [t.numel() * t.element_size() for row in prob.grads for t in row]
+    wl = prob.wl
+    del prob
+    prob = Problem(wl, kt, chunk_bytes=args_chunk(args), arena=True)
+    host_in = [a.cpu().pin_memory() for a in prob.grad_arenas]
+    host_out = [torch.empty_like(prob.out_arena, device="cpu").pin_memory()]
+    dst, src = kt.kt_ptrs(prob.grad_arenas), kt.kt_ptrs(host_in)
+    sizes = [a.numel() * a.element_size() for a in prob.grad_arenas]
     sizes_c = (ctypes.c_int64 * len(sizes))(*sizes)
-    o_dst = kt.kt_ptrs(host_out)
-    o_src = kt.kt_ptrs(prob.out[0])
-    o_sizes = [t.numel() * t.element_size() for t in prob.out[0]]
+    o_dst, o_src = kt.kt_ptrs(host_out), kt.kt_ptrs([prob.out_arena])
+    o_sizes = [prob.out_arena.numel() * prob.out_arena.element_size()]
     o_sizes_c = (ctypes.c_int64 * len(o_sizes))(*o_sizes)
 
     def one():
@@ -352,6 +388,9 @@ def run_e2e(prob, kt, args, barrier) -> dict:
         one()
     b.record(prob.main)
     barrier()
+    if not bool(host_out[0].any()):
+        raise RuntimeError("end-to-end arm: the result buffer on the host is all zero")
+    kt.kt_destroy(prob.ctx)
     return {"seconds": a.elapsed_time(b) * 1e-3, "h2d": sum(sizes), "d2h": sum(o_sizes)}
 
 
@@ -478,6 +517,7 @@ def main() -> None:
     ap.add_argument("--sweep-max-bytes", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--cpu-seconds", type=float, default=12.0)
+    ap.add_argument("--relay-chunk-mib", type=int, default=4)
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.sweep:
