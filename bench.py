@@ -198,6 +198,12 @@ class Problem:
             e3.record(self.main)
             self.k2_events.append((e2, e3))
 
+    def direct(self):
+        """The one-pass route (no transport, no relay): what a collective that needs no host
+        relay costs."""
+        self.kt.kt_sync_direct(self.ctx, self.out_ptrs, scale=1.0, bucket=-1, out_dtype=self.out_dtype,
+                               R=1, stream=self.main)
+
     def k1_seconds(self) -> float:
         return sum(a.elapsed_time(b) for a, b in self.k1_events) * 1e-3
 
@@ -206,10 +212,15 @@ class Problem:
 
 
 def host_link_bandwidth(nbytes: int = 256 << 20, reps: int = 10) -> dict:
-    """Pinned cudaMemcpyAsync both ways, best of `reps` (GB/s)."""
+    """Pinned cudaMemcpyAsync, best of `reps` (GB/s): each direction alone, and both
+    directions at the same time on two streams (per direction; what a relay whose way down
+    and way up overlap can reach at most)."""
     dev = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
     host = torch.empty(nbytes, dtype=torch.uint8).pin_memory()
-    best = {"d2h": 0.0, "h2d": 0.0}
+    dev2 = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
+    host2 = torch.empty(nbytes, dtype=torch.uint8).pin_memory()
+    best = {"d2h": 0.0, "h2d": 0.0, "both": 0.0}
+    s1, s2 = torch.cuda.Stream(), torch.cuda.Stream()
     for _ in range(reps):
         for name, (dst, src) in (("d2h", (host, dev)), ("h2d", (dev, host))):
             a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -218,7 +229,61 @@ def host_link_bandwidth(nbytes: int = 256 << 20, reps: int = 10) -> dict:
             b.record()
             b.synchronize()
             best[name] = max(best[name], nbytes / (a.elapsed_time(b) * 1e-3) / 1e9)
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        s1.wait_event(a)
+        s2.wait_event(a)
+        with torch.cuda.stream(s1):
+            host.copy_(dev, non_blocking=True)
+        with torch.cuda.stream(s2):
+            dev2.copy_(host2, non_blocking=True)
+        torch.cuda.current_stream().wait_stream(s1)
+        torch.cuda.current_stream().wait_stream(s2)
+        b.record()
+        b.synchronize()
+        best["both"] = max(best["both"], nbytes / (a.elapsed_time(b) * 1e-3) / 1e9)
     return best
+
+
+def time_launches(fn, stream, reps: int) -> float:
+    """Average CUDA-event duration (s) of `reps` launches queued back to back on `stream`,
+    each bracketed by its own pair of events."""
+    pairs = []
+    for _ in range(3):
+        fn()
+    torch.cuda.synchronize()
+    for _ in range(reps):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(stream)
+        fn()
+        b.record(stream)
+        pairs.append((a, b))
+    torch.cuda.synchronize()
+    return sum(a.elapsed_time(b) for a, b in pairs) * 1e-3 / reps
+
+
+def large_bucket_roofline(kt, peak: float, K: int = 4, bytes_per_rank: int = 256 << 20) -> dict:
+    """The fused reduce on one flat bucket of 256 MiB per rank (the bucket size the bandwidth
+    target is stated for): algorithmic bytes over the CUDA-event time of a launch."""
+    wl = W.sweep_point(K, bytes_per_rank, "f32")
+    prob = Problem(wl, kt)
+    by = algorithmic_bytes(wl)
+    with torch.cuda.stream(prob.main):
+        k1 = time_launches(lambda: kt.kt_hier_reduce(prob.ctx, kt.KT_INTRA, prob.transport, stream=prob.main),
+                           prob.main, 20)
+        k2 = time_launches(lambda: kt.kt_unpack_scale(prob.ctx, prob.transport, prob.out_ptrs, out_dtype=prob.out_dtype,
+                                                      R=1, stream=prob.main), prob.main, 20)
+        direct = time_launches(prob.direct, prob.main, 20)
+    kt.kt_destroy(prob.ctx)
+    direct_bytes = wl.K * wl.N * wl.elem_size + wl.N * wl.elem_size
+
+    def row(nbytes, sec):
+        return {"us": round(sec * 1e6, 2), "GBps": round(nbytes / sec / 1e9, 1), "frac": round(nbytes / sec / 1e9 / peak, 4),
+                "frac_of_nominal_8TBs": round(nbytes / sec / 1e9 / NOMINAL_HBM_GBS, 4)}
+    return {"workload": "flat fp32 bucket, %d ranks x %d MiB in 2 groups" % (K, bytes_per_rank >> 20),
+            "k1_intra_reduce": row(by["k1"], k1), "k2_combine_unpack": row(by["k2"], k2),
+            "k_direct_sync": row(direct_bytes, direct)}
 
 
 def max_over_ranks(seconds, dist, device) -> list:
@@ -281,6 +346,7 @@ def run_ours(args) -> dict:
         total_s = t_start.elapsed_time(t_end) * 1e-3
         per_step = [a.elapsed_time(b) for a, b in zip([t_start] + marks[:-1], marks)]
         k1_s = prob.k1_seconds()
+        direct_s = time_launches(prob.direct, prob.main, args.steps)
 
         # end to end: gradients start in pinned host memory, the result ends there
         e2e = run_e2e(prob, kt, args, barrier)
@@ -317,7 +383,10 @@ def run_ours(args) -> dict:
             "phases": {"k1_us": round(k1_launch_s * 1e6, 2), "k2_us": round(k2_launch_s * 1e6, 2),
                        "k2_GBps": round(nbytes["k2"] / k2_launch_s / 1e9, 1),
                        "relay_ms": round(relay_s * 1e3, 4) if wl.staged else 0.0,
-                       "relay_GBps_each_way": round(nbytes["stage_each_way"] / relay_s / 1e9, 1) if wl.staged else None},
+                       "relay_GBps_each_way": round(nbytes["stage_each_way"] / relay_s / 1e9, 1) if wl.staged else None,
+                       "direct_us": round(direct_s * 1e6, 2),
+                       "direct_note": "kt_sync_direct: the same arithmetic in one pass without transport or "
+                                      "relay (what a collective inside one vendor group costs); not part of the step"},
             "latency_ms": {"p50": round(statistics.median(per_step), 4),
                            "p95": round(sorted(per_step)[int(0.95 * (len(per_step) - 1))], 4)},
         },
@@ -336,7 +405,12 @@ def run_ours(args) -> dict:
     }
     if link is not None:
         result["host_link"] = {"d2h_GBps": round(link["d2h"], 1), "h2d_GBps": round(link["h2d"], 1),
-                               "how": "pinned copy of 256 MiB, best of 10"}
+                               "both_ways_at_once_GBps_each": round(link["both"], 1),
+                               "relay_frac_of_both_ways": round(nbytes["stage_each_way"] / relay_s / 1e9 / link["both"], 3),
+                               "how": "pinned copy of 256 MiB, best of 10; both ways = one copy down and one "
+                                      "up on two streams at the same time"}
+    if rank == 0 and world == 1 and not args.no_large_bucket:
+        result["roofline_large_bucket"] = large_bucket_roofline(kt, peak)
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         result["cpu_baseline"] = cpu_baseline(wl, prob.shares, budget_s=args.cpu_seconds)
     if dist is not None:
@@ -516,6 +590,7 @@ def main() -> None:
     ap.add_argument("--sweep", action="store_true")
     ap.add_argument("--sweep-max-bytes", type=int, default=0)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-large-bucket", action="store_true")
     ap.add_argument("--cpu-seconds", type=float, default=12.0)
     ap.add_argument("--relay-chunk-mib", type=int, default=4)
     args = ap.parse_args()

@@ -13,6 +13,8 @@
  *   kt_stage_to_host relay of the partials through pinned host RAM  (Section III-A, steps 1-3)
  *   kt_hier_reduce   INTER: S = sum_g W_g P_g
  *   kt_unpack_scale  per-parameter gradients = cast(scale * S)
+ * or, when no host relay is needed (Section III-B, homogeneous dispatch),
+ *   kt_sync_direct   all of the above arithmetic in one pass, no transport
  *
  * Conventions
  *  - Every pointer argument says "host" or "device".  "host array of device pointers"
@@ -187,6 +189,21 @@ int kt_stage_wait(kt_ctx *ctx, int dir, int bucket, void *main_stream, int timeo
 int kt_unpack_scale(kt_ctx *ctx, const float *const *src, int from_combined,
                     void *const *out_grads, int R, int out_dtype, float scale, int bucket,
                     void *stream);
+
+/* The direct path: the whole synchronisation in one pass, without transport buffers.
+ * Section III-B: a collective whose participants need no host relay (one vendor group, or
+ * groups that share a device) is dispatched straight to the device-side reduction; only
+ * collectives that span accelerator types take the staged route above.
+ * Reads every registered gradient element once and writes
+ *   out[t][j] = cast(scale * sum_g W_g * (sum_{r in g} a_r * f32(x_r^(t)[j])))
+ * with the operation order of kt_hier_reduce(KT_INTRA) followed by kt_unpack_scale (group
+ * partials are formed first, in fp32, then combined): results are bit-identical to that
+ * route.  out_grads, R, out_dtype, scale, bucket as in kt_unpack_scale; the gradients are
+ * the ones registered by kt_bucket_pack.  May allocate the destination table like
+ * kt_unpack_scale.
+ * Errors: KT_ERR_STATE, KT_ERR_SHAPE, KT_ERR_INVALID, KT_ERR_ALIGN, KT_ERR_NOMEM, KT_ERR_CUDA. */
+int kt_sync_direct(kt_ctx *ctx, void *const *out_grads, int R, int out_dtype, float scale,
+                   int bucket, void *stream);
 
 /* Standalone cast kernel: n elements from `in` (device, in_dtype) to `out` (device,
  * out_dtype); bf16 -> fp32 exact, fp32 -> bf16 round-to-nearest-even, same type = copy.

@@ -25,7 +25,7 @@ KT_MAX_RANKS, KT_MAX_GROUPS = 64, 16
 
 EXPORTS = ["kt_schedule", "kt_groups_init", "kt_set_shares", "kt_set_coefficients",
            "kt_get_coefficients", "kt_bucket_pack", "kt_plan_buckets", "kt_plan_query", "kt_hier_reduce",
-           "kt_stage_to_host", "kt_relay_through_host", "kt_stage_wait", "kt_unpack_scale", "kt_cast", "kt_copy_tensors", "kt_sync_flat_static", "kt_launch_count",
+           "kt_stage_to_host", "kt_relay_through_host", "kt_stage_wait", "kt_unpack_scale", "kt_sync_direct", "kt_cast", "kt_copy_tensors", "kt_sync_flat_static", "kt_launch_count",
            "kt_last_error", "kt_destroy"]
 
 _DTYPES = {torch.float32: KT_F32, torch.bfloat16: KT_BF16}
@@ -60,6 +60,7 @@ def _load() -> C.CDLL:
         "kt_relay_through_host": ([vp, C.c_int, vpp, vpp, vpp, C.c_int64, vp, vp, vp], C.c_int),
         "kt_stage_wait": ([vp, C.c_int, C.c_int, vp, C.c_int], C.c_int),
         "kt_unpack_scale": ([vp, vpp, C.c_int, vpp, C.c_int, C.c_int, C.c_float, C.c_int, vp], C.c_int),
+        "kt_sync_direct": ([vp, vpp, C.c_int, C.c_int, C.c_float, C.c_int, vp], C.c_int),
         "kt_cast": ([vp, C.c_int, vp, C.c_int, C.c_int64, vp], C.c_int),
         "kt_copy_tensors": ([vpp, vpp, i64p, C.c_int, C.c_int, vp], C.c_int),
         "kt_sync_flat_static": ([i32p, i32p, C.c_int, C.c_int, vpp, C.c_int, C.c_int64, vp, C.c_int,
@@ -258,13 +259,8 @@ def kt_stage_wait(ctx: Ctx, direction: int, bucket: int = -1, main_stream=None, 
     _check(_lib.kt_stage_wait(ctx.handle, int(direction), int(bucket), _stream(main_stream), int(timeout_ms)))
 
 
-def kt_unpack_scale(ctx: Ctx, src: Ptrs, out_grads: Union[PtrArray, Sequence[Sequence[torch.Tensor]]],
-                    scale: float = 1.0, from_combined: bool = False, bucket: int = -1,
-                    out_dtype: Optional[int] = None, R: Optional[int] = None, stream=None) -> None:
-    """out_grads[c][t]: copy c of tensor t (or a PtrArray of R*T pointers with R, out_dtype given)."""
-    sp = kt_ptrs(src)
-    if sp.n != (1 if from_combined else ctx.G):
-        raise KtError(KT_ERR_SHAPE, "wrong number of source buffers")
+def _out_args(ctx: Ctx, out_grads, out_dtype, R):
+    """Marshals out_grads[c][t] (or a ready PtrArray) into (PtrArray, R, out_dtype)."""
     if isinstance(out_grads, PtrArray):
         op = out_grads
         if R is None or out_dtype is None:
@@ -282,8 +278,29 @@ def kt_unpack_scale(ctx: Ctx, src: Ptrs, out_grads: Union[PtrArray, Sequence[Seq
         op = PtrArray(flat)
     if op.n != R * ctx.T:
         raise KtError(KT_ERR_SHAPE, "expected %d output pointers" % (R * ctx.T))
-    _check(_lib.kt_unpack_scale(ctx.handle, sp.array, 1 if from_combined else 0, op.array, int(R),
-                                int(out_dtype), C.c_float(scale), int(bucket), _stream(stream)))
+    return op, int(R), int(out_dtype)
+
+
+def kt_unpack_scale(ctx: Ctx, src: Ptrs, out_grads: Union[PtrArray, Sequence[Sequence[torch.Tensor]]],
+                    scale: float = 1.0, from_combined: bool = False, bucket: int = -1,
+                    out_dtype: Optional[int] = None, R: Optional[int] = None, stream=None) -> None:
+    """out_grads[c][t]: copy c of tensor t (or a PtrArray of R*T pointers with R, out_dtype given)."""
+    sp = kt_ptrs(src)
+    if sp.n != (1 if from_combined else ctx.G):
+        raise KtError(KT_ERR_SHAPE, "wrong number of source buffers")
+    op, R, out_dtype = _out_args(ctx, out_grads, out_dtype, R)
+    _check(_lib.kt_unpack_scale(ctx.handle, sp.array, 1 if from_combined else 0, op.array, R,
+                                out_dtype, C.c_float(scale), int(bucket), _stream(stream)))
+    ctx._keep["out"] = op
+
+
+def kt_sync_direct(ctx: Ctx, out_grads: Union[PtrArray, Sequence[Sequence[torch.Tensor]]],
+                   scale: float = 1.0, bucket: int = -1, out_dtype: Optional[int] = None,
+                   R: Optional[int] = None, stream=None) -> None:
+    """The one-pass route without transport buffers; out_grads as in kt_unpack_scale."""
+    op, R, out_dtype = _out_args(ctx, out_grads, out_dtype, R)
+    _check(_lib.kt_sync_direct(ctx.handle, op.array, R, out_dtype, C.c_float(scale), int(bucket),
+                               _stream(stream)))
     ctx._keep["out"] = op
 
 

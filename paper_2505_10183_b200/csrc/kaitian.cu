@@ -269,6 +269,65 @@ void launch_k2(int tile, int n_tiles, cudaStream_t s, const K2Params &p) {
         k2_combine_unpack<Tout, TILE_BF16><<<n_tiles, NT, 0, s>>>(p);
 }
 
+int check_out_args(const kt_ctx *c, void *const *out_grads, int R, int out_dtype) {
+    if (!out_grads) return fail(KT_ERR_INVALID, "out_grads is NULL");
+    if (R < 1 || R > c->K) return fail(KT_ERR_SHAPE, "R = %d outside [1, K = %d]", R, c->K);
+    if (out_dtype != KT_F32 && out_dtype != KT_BF16) return fail(KT_ERR_INVALID, "unknown out_dtype %d", out_dtype);
+    const size_t es = out_dtype == KT_F32 ? 4 : 2;
+    const int T = c->T;
+    const size_t np = static_cast<size_t>(R) * T;
+    for (size_t i = 0; i < np; ++i) {
+        if (c->numel[i % T] > 0 && !out_grads[i]) return fail(KT_ERR_INVALID, "out_grads[%zu] is NULL", i);
+        if (reinterpret_cast<uintptr_t>(out_grads[i]) % es) return fail(KT_ERR_ALIGN, "out_grads[%zu] is not element aligned", i);
+    }
+    return KT_OK;
+}
+
+// Destination table on the device: R*T pointers in transport tensor order, then one flag per
+// tensor saying that all R destinations are 16-byte aligned.  Uploaded only when it changed.
+// *sz_ptrs receives the byte offset of the flags inside the table.
+int upload_out_table(kt_ctx *c, void *const *out_grads, int R, int out_dtype, cudaStream_t s, size_t *sz_ptrs_out) {
+    const int T = c->T;
+    const size_t np = static_cast<size_t>(R) * T;
+    const bool same = c->out_R == R && c->out_dtype == out_dtype && c->out_cached.size() == np &&
+                      std::memcmp(c->out_cached.data(), out_grads, np * sizeof(void *)) == 0;
+    const size_t sz_ptrs = round_up(np * sizeof(void *), 256);
+    *sz_ptrs_out = sz_ptrs;
+    if (same) return KT_OK;
+    const size_t need = sz_ptrs + round_up(T, 256);
+    if (need > c->d_out_cap) {
+        // the previous table may still be in use by queued kernels: release it once they are done
+        if (c->d_out) {
+            KT_CUDA(cudaDeviceSynchronize());
+            cudaFree(c->d_out);
+            c->d_out = nullptr;
+            c->d_out_cap = 0;
+        }
+        if (cudaMalloc(&c->d_out, need) != cudaSuccess) {
+            cudaGetLastError();
+            return fail(KT_ERR_NOMEM, "device allocation of %zu bytes failed", need);
+        }
+        c->d_out_cap = need;
+    } else {
+        KT_CUDA(cudaStreamSynchronize(s));   // queued kernels may still read the old table
+    }
+    std::vector<char> staging(sz_ptrs + T, 0);
+    for (int cpy = 0; cpy < R; ++cpy)
+        for (int u = 0; u < T; ++u)
+            reinterpret_cast<void **>(staging.data())[static_cast<size_t>(cpy) * T + u] =
+                out_grads[static_cast<size_t>(cpy) * T + (T - 1 - u)];
+    for (int u = 0; u < T; ++u) {
+        bool al = true;
+        for (int cpy = 0; cpy < R; ++cpy) al = al && aligned16(out_grads[static_cast<size_t>(cpy) * T + (T - 1 - u)]);
+        staging[sz_ptrs + u] = al ? 1 : 0;
+    }
+    KT_CUDA(cudaMemcpy(c->d_out, staging.data(), staging.size(), cudaMemcpyHostToDevice));
+    c->out_cached.assign(out_grads, out_grads + np);
+    c->out_R = R;
+    c->out_dtype = out_dtype;
+    return KT_OK;
+}
+
 }  // namespace
 
 // ====================================================================== C ABI
@@ -693,60 +752,15 @@ int kt_stage_wait(kt_ctx *c, int dir, int bucket, void *main_stream, int timeout
 int kt_unpack_scale(kt_ctx *c, const float *const *src, int from_combined, void *const *out_grads, int R,
                     int out_dtype, float scale, int bucket, void *stream) {
     if (int rc = check_ctx(c, true)) return rc;
-    if (!out_grads) return fail(KT_ERR_INVALID, "out_grads is NULL");
-    if (R < 1 || R > c->K) return fail(KT_ERR_SHAPE, "R = %d outside [1, K = %d]", R, c->K);
-    if (out_dtype != KT_F32 && out_dtype != KT_BF16) return fail(KT_ERR_INVALID, "unknown out_dtype %d", out_dtype);
     const int nsrc = from_combined ? 1 : c->G;
+    if (int rc = check_out_args(c, out_grads, R, out_dtype)) return rc;
     if (int rc = check_buffers(c, src, nsrc, "src")) return rc;
-    const size_t es = out_dtype == KT_F32 ? 4 : 2;
-    const int T = c->T;
-    const size_t np = static_cast<size_t>(R) * T;
-    for (size_t i = 0; i < np; ++i) {
-        if (c->numel[i % T] > 0 && !out_grads[i]) return fail(KT_ERR_INVALID, "out_grads[%zu] is NULL", i);
-        if (reinterpret_cast<uintptr_t>(out_grads[i]) % es) return fail(KT_ERR_ALIGN, "out_grads[%zu] is not element aligned", i);
-    }
     TilePlan tp{};
     if (int rc = make_tile_plan(c, bucket, &tp)) return rc;
     KT_CUDA(cudaSetDevice(c->device));
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-
-    // (re)upload the destination table only when it changed
-    const bool same = c->out_R == R && c->out_dtype == out_dtype && c->out_cached.size() == np &&
-                      std::memcmp(c->out_cached.data(), out_grads, np * sizeof(void *)) == 0;
-    const size_t sz_ptrs = round_up(np * sizeof(void *), 256);
-    if (!same) {
-        const size_t need = sz_ptrs + round_up(T, 256);
-        if (need > c->d_out_cap) {
-            // the previous table may still be in use by queued kernels: release it once they are done
-            if (c->d_out) {
-                KT_CUDA(cudaDeviceSynchronize());
-                cudaFree(c->d_out);
-                c->d_out = nullptr;
-                c->d_out_cap = 0;
-            }
-            if (cudaMalloc(&c->d_out, need) != cudaSuccess) {
-                cudaGetLastError();
-                return fail(KT_ERR_NOMEM, "device allocation of %zu bytes failed", need);
-            }
-            c->d_out_cap = need;
-        } else {
-            KT_CUDA(cudaStreamSynchronize(s));   // queued kernels may still read the old table
-        }
-        std::vector<char> staging(sz_ptrs + T, 0);
-        for (int cpy = 0; cpy < R; ++cpy)
-            for (int u = 0; u < T; ++u)
-                reinterpret_cast<void **>(staging.data())[static_cast<size_t>(cpy) * T + u] =
-                    out_grads[static_cast<size_t>(cpy) * T + (T - 1 - u)];
-        for (int u = 0; u < T; ++u) {
-            bool al = true;
-            for (int cpy = 0; cpy < R; ++cpy) al = al && aligned16(out_grads[static_cast<size_t>(cpy) * T + (T - 1 - u)]);
-            staging[sz_ptrs + u] = al ? 1 : 0;
-        }
-        KT_CUDA(cudaMemcpy(c->d_out, staging.data(), staging.size(), cudaMemcpyHostToDevice));
-        c->out_cached.assign(out_grads, out_grads + np);
-        c->out_R = R;
-        c->out_dtype = out_dtype;
-    }
+    size_t sz_ptrs = 0;
+    if (int rc = upload_out_table(c, out_grads, R, out_dtype, s, &sz_ptrs)) return rc;
     if (tp.n_tiles == 0) return KT_OK;
 
     K2Params p{};
@@ -768,6 +782,36 @@ int kt_unpack_scale(kt_ctx *c, const float *const *src, int from_combined, void 
         launch_k2<float>(tp.tile, tp.n_tiles, s, p);
     else
         launch_k2<unsigned short>(tp.tile, tp.n_tiles, s, p);
+    c->launches += 1;
+    KT_CUDA(cudaGetLastError());
+    return KT_OK;
+}
+
+int kt_sync_direct(kt_ctx *c, void *const *out_grads, int R, int out_dtype, float scale, int bucket, void *stream) {
+    if (int rc = check_ctx(c, true)) return rc;
+    if (int rc = check_out_args(c, out_grads, R, out_dtype)) return rc;
+    TilePlan tp{};
+    if (int rc = make_tile_plan(c, bucket, &tp)) return rc;
+    KT_CUDA(cudaSetDevice(c->device));
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    size_t sz_ptrs = 0;
+    if (int rc = upload_out_table(c, out_grads, R, out_dtype, s, &sz_ptrs)) return rc;
+    if (tp.n_tiles == 0) return KT_OK;
+
+    DirectParams p{};
+    p.tp = tp;
+    p.ptrs = c->d_ptrs;
+    p.rt = c->rt;
+    p.gt = c->gt;
+    p.out_ptrs = static_cast<void *const *>(c->d_out);
+    p.out_aligned = static_cast<const unsigned char *>(c->d_out) + sz_ptrs;
+    p.R = R;
+    p.scale = scale;
+    const bool in32 = c->in_dtype == KT_F32, out32 = out_dtype == KT_F32;
+    if (in32 && out32) k_direct_sync<float, float, KT_KB><<<tp.n_tiles, NT, 0, s>>>(p);
+    else if (in32) k_direct_sync<float, unsigned short, KT_KB><<<tp.n_tiles, NT, 0, s>>>(p);
+    else if (out32) k_direct_sync<unsigned short, float, KT_KB_DIRECT_BF16><<<tp.n_tiles, NT, 0, s>>>(p);
+    else k_direct_sync<unsigned short, unsigned short, KT_KB_DIRECT_BF16><<<tp.n_tiles, NT, 0, s>>>(p);
     c->launches += 1;
     KT_CUDA(cudaGetLastError());
     return KT_OK;

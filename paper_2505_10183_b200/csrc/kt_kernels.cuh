@@ -30,6 +30,9 @@ namespace {
 #ifndef KT_KB
 #define KT_KB 4                  /* ranks whose loads are issued together */
 #endif
+#ifndef KT_KB_DIRECT_BF16
+#define KT_KB_DIRECT_BF16 2      /* the same for the direct path on bf16 gradients (keeps it at 4 CTAs per SM) */
+#endif
 #ifndef KT_WARM_CTAS
 #define KT_WARM_CTAS 1184        /* about two waves: CTAs that prefetch the tables into L2 */
 #endif
@@ -91,6 +94,17 @@ struct K2Params {
     int R;
     float scale;
     int wide;                          // every source base is 32-byte aligned
+};
+
+struct DirectParams {
+    TilePlan tp;
+    const void *const *ptrs;           // [K][T] device pointer table
+    RankTab rt;
+    GroupTab gt;
+    void *const *out_ptrs;             // [R][T] device pointer table
+    const unsigned char *out_aligned;  // [T] all R destinations 16-byte aligned
+    int R;
+    float scale;
 };
 
 struct PackParams {
@@ -377,6 +391,107 @@ __global__ void __launch_bounds__(NT) k2_combine_unpack(const __grid_constant__ 
         k2_tile<Tout, TILE, false>(p, t);
     else
         k2_tile<Tout, TILE, true>(p, t);
+}
+
+// ------------------------------------------------------------------ direct path: reduce, combine, scale, cast, unpack in one pass
+// Section III-B: a collective whose participants need no host relay is dispatched straight
+// to the device-side reduction.  Same arithmetic and order as K1 followed by K2, with the
+// group partials kept in registers instead of a transport buffer:
+//   out_c^(u)[e] = cast(scale * sum_g W_g * (sum_{r in g} a_r * f32(x_r^(u)[e]))).
+template <typename Tout, int VEC>
+__device__ __forceinline__ void store_out(Tout *d, const float (&y)[VEC]) {
+    if constexpr (sizeof(Tout) == 4) {
+#pragma unroll
+        for (int q = 0; q < VEC / 4; ++q)
+            reinterpret_cast<float4 *>(d)[q] = make_float4(y[4 * q], y[4 * q + 1], y[4 * q + 2], y[4 * q + 3]);
+    } else if constexpr (VEC == 8) {
+        *reinterpret_cast<uint4 *>(d) = make_uint4(pack_bf16x2(y[0], y[1]), pack_bf16x2(y[2], y[3]),
+                                                   pack_bf16x2(y[4], y[5]), pack_bf16x2(y[6], y[7]));
+    } else {
+        *reinterpret_cast<uint2 *>(d) = make_uint2(pack_bf16x2(y[0], y[1]), pack_bf16x2(y[2], y[3]));
+    }
+}
+
+template <typename Tin, typename Tout, int KB, bool EDGE>
+__device__ __forceinline__ void direct_tile(const DirectParams &p, const TileRef &t) {
+    constexpr int VEC = Elem<Tin>::VEC;
+    constexpr int TILE = Elem<Tin>::TILE;
+    constexpr int ITERS = TILE / (NT * VEC);
+    const int K = p.rt.K;
+    const int T = p.tp.T;
+    const bool aligned = t.ti.flags & FLAG_ALIGNED;
+    long long e[ITERS];
+#pragma unroll
+    for (int it = 0; it < ITERS; ++it) e[it] = t.e0 + (it * NT + threadIdx.x) * VEC;
+
+    float acc[ITERS][VEC], sum[ITERS][VEC];
+    for (int kb = 0; kb < K; kb += KB) {
+        uint4 raw[KB][ITERS];
+#pragma unroll
+        for (int j = 0; j < KB; ++j) {
+            if (kb + j < K) {
+                const Tin *s = static_cast<const Tin *>(ldg_ptr(&p.ptrs[static_cast<size_t>(kb + j) * T + t.u]));
+#pragma unroll
+                for (int it = 0; it < ITERS; ++it) {
+                    if (!EDGE || (aligned && e[it] + VEC <= t.ti.numel))
+                        raw[j][it] = ld_stream(s + e[it]);
+                    else
+                        raw[j][it] = Elem<Tin>::gather(s, e[it], t.ti.numel);
+                }
+            }
+        }
+#pragma unroll
+        for (int j = 0; j < KB; ++j) {
+            if (kb + j < K) {
+                const float a = p.rt.coef[kb + j];
+                const bool first = p.rt.first[kb + j];
+#pragma unroll
+                for (int it = 0; it < ITERS; ++it) {
+                    float x[VEC];
+                    Elem<Tin>::unpack(raw[j][it], x);
+#pragma unroll
+                    for (int c = 0; c < VEC; ++c)
+                        acc[it][c] = first ? __fmul_rn(a, x[c]) : __fmaf_rn(a, x[c], acc[it][c]);
+                }
+                if (p.rt.last[kb + j]) {           // the group's partial is complete: fold it in
+                    const int g = p.rt.gid[kb + j];
+                    const float w = p.gt.W[g];
+#pragma unroll
+                    for (int it = 0; it < ITERS; ++it)
+#pragma unroll
+                        for (int c = 0; c < VEC; ++c)
+                            sum[it][c] = g == 0 ? __fmul_rn(w, acc[it][c]) : __fmaf_rn(w, acc[it][c], sum[it][c]);
+                }
+            }
+        }
+    }
+    const bool out_aligned = p.out_aligned[t.u];
+#pragma unroll
+    for (int it = 0; it < ITERS; ++it) {
+        float y[VEC];
+#pragma unroll
+        for (int c = 0; c < VEC; ++c) y[c] = __fmul_rn(sum[it][c], p.scale);
+        if (!EDGE || (out_aligned && e[it] + VEC <= t.ti.numel)) {
+            for (int c = 0; c < p.R; ++c)
+                store_out<Tout, VEC>(static_cast<Tout *>(ldg_ptr(&p.out_ptrs[static_cast<size_t>(c) * T + t.u])) + e[it], y);
+        } else if (e[it] < t.ti.numel) {
+            for (int c = 0; c < p.R; ++c) {
+                Tout *d = static_cast<Tout *>(ldg_ptr(&p.out_ptrs[static_cast<size_t>(c) * T + t.u]));
+#pragma unroll
+                for (int k = 0; k < VEC; ++k)
+                    if (e[it] + k < t.ti.numel) d[e[it] + k] = Elem<Tout>::narrow_one(y[k]);
+            }
+        }
+    }
+}
+
+template <typename Tin, typename Tout, int KB>
+__global__ void __launch_bounds__(NT) k_direct_sync(const __grid_constant__ DirectParams p) {
+    const TileRef t = locate_tile(p.tp);
+    if ((t.ti.flags & FLAG_ALIGNED) && p.out_aligned[t.u] && t.e0 + Elem<Tin>::TILE <= t.ti.numel)
+        direct_tile<Tin, Tout, KB, false>(p, t);
+    else
+        direct_tile<Tin, Tout, KB, true>(p, t);
 }
 
 // ------------------------------------------------------------------ flat inter-group combine into a combined buffer
