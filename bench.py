@@ -152,7 +152,9 @@ class Problem:
         kt.kt_bucket_pack(self.ctx, self.grads, wl.bucket_cap_bytes)
         self.plan = kt.kt_plan_query(self.ctx)
         n = self.plan.transport_numel
-        self.transport = kt.kt_ptrs([torch.zeros(n, device="cuda") for _ in range(wl.G)])
+        # the G buffers of a set are rows of one allocation: the relay then moves a chunk of all
+        # groups in one copy
+        self.transport = kt.kt_ptrs(list(torch.zeros(wl.G, n, device="cuda")))
         if arena:
             self.out_arena = torch.zeros(self.arena_numel, dtype=dt, device="cuda")
             self.out = [views(self.out_arena)]
@@ -162,8 +164,8 @@ class Problem:
         self.out_dtype = kt.KT_F32 if wl.dtype == "f32" else kt.KT_BF16
         self.main = torch.cuda.Stream()
         if wl.staged:
-            self.recv = kt.kt_ptrs([torch.zeros(n, device="cuda") for _ in range(wl.G)])
-            self.pinned = kt.kt_ptrs([torch.zeros(n).pin_memory() for _ in range(wl.G)])
+            self.recv = kt.kt_ptrs(list(torch.zeros(wl.G, n, device="cuda")))
+            self.pinned = kt.kt_ptrs(list(torch.zeros(wl.G, n).pin_memory()))
             self.side_d2h = torch.cuda.Stream()
             self.side_h2d = torch.cuda.Stream()
         self.k1_events = []

@@ -166,6 +166,8 @@ int kt_stage_to_host(kt_ctx *ctx, int dir, int bucket, float *const *transport,
  * down / up is what kt_stage_wait(KT_D2H / KT_H2D, bucket) waits for.
  * send, host_pinned, recv: host arrays of G pointers (device fp32, pinned host, device fp32),
  * same element offsets in all three.  chunk_bytes >= 256; the two copy streams must differ.
+ * With bucket == -1, if the G buffers of each list lie back to back in memory (rows of one
+ * allocation of G * transport_numel elements), a chunk of all groups moves in one copy.
  * Errors: KT_ERR_STATE, KT_ERR_SHAPE, KT_ERR_INVALID, KT_ERR_CUDA. */
 int kt_relay_through_host(kt_ctx *ctx, int bucket, float *const *send, float *const *host_pinned,
                           float *const *recv, int64_t chunk_bytes, void *main_stream,
@@ -204,6 +206,33 @@ int kt_unpack_scale(kt_ctx *ctx, const float *const *src, int from_combined,
  * Errors: KT_ERR_STATE, KT_ERR_SHAPE, KT_ERR_INVALID, KT_ERR_ALIGN, KT_ERR_NOMEM, KT_ERR_CUDA. */
 int kt_sync_direct(kt_ctx *ctx, void *const *out_grads, int R, int out_dtype, float scale,
                    int bucket, void *stream);
+
+/* Hierarchical Broadcast (model synchronisation).  The paper routes Broadcast through the
+ * same hierarchy as AllReduce (Section III, "broadcast for model synchronization"; Section
+ * III-A: inside a group directly, between groups through host RAM in the three copy steps).
+ * The tensors are the ones registered with kt_bucket_pack (here: parameters rather than
+ * gradients; the same context type, usually a second context).  The root rank's tensors are
+ * read, every other rank's registered tensors are WRITTEN; all copies are bit copies in the
+ * registered dtype, laid out in the flat buffers at the plan's offsets (zero padding).
+ *
+ * kt_bcast_send: one pass over the root's tensors; writes the flat send buffer of the root's
+ *        group (`send`: device, transport_numel elements of the registered dtype, 16-byte
+ *        aligned) and the tensors of the root's group mates.
+ * kt_bcast_relay: the bucket's range of `send` (device) goes to `host_pinned` (host, pinned,
+ *        same layout) and from there into recv[g] (device) of every group g other than the
+ *        root's, chunk by chunk on the two copy streams as in kt_relay_through_host;
+ *        completion is what kt_stage_wait(KT_D2H / KT_H2D, bucket) waits for.
+ *        recv: host array of G device pointers; the root group's entry is ignored.
+ * kt_bcast_recv: one pass over the receive buffers; every group other than the root's reads
+ *        recv[g] once and writes the tensors of all its members.  Passing the send buffer as
+ *        recv[g] skips the relay (groups that can reach each other directly).
+ * root: rank index in [0, K).  bucket as in kt_hier_reduce.
+ * Errors: KT_ERR_STATE, KT_ERR_SHAPE, KT_ERR_INVALID, KT_ERR_ALIGN, KT_ERR_CUDA. */
+int kt_bcast_send(kt_ctx *ctx, int root, int bucket, void *send, void *stream);
+int kt_bcast_relay(kt_ctx *ctx, int root, int bucket, const void *send, void *host_pinned,
+                   void *const *recv, int64_t chunk_bytes, void *main_stream, void *d2h_stream,
+                   void *h2d_stream);
+int kt_bcast_recv(kt_ctx *ctx, int root, int bucket, void *const *recv, void *stream);
 
 /* Standalone cast kernel: n elements from `in` (device, in_dtype) to `out` (device,
  * out_dtype); bf16 -> fp32 exact, fp32 -> bf16 round-to-nearest-even, same type = copy.

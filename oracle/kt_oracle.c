@@ -290,6 +290,25 @@ void kto_pack(const void *const *tensors, const int64_t *numel, const int64_t *t
 }
 
 /* ------------------------------------------------------------------------- */
+/* Hierarchical broadcast (model synchronisation; Section III routes Broadcast  */
+/* through the same hierarchy as AllReduce).  What it must produce is plain:    */
+/* every rank ends up with the root's tensors, bit for bit.  The flat buffer    */
+/* that crosses the host is the pack of the root's list; a receiving group      */
+/* copies each tensor out of it again:                                         */
+/*   out^(t)[j] = flat[tensor_offset[t] + j]  (bit copy, same dtype).           */
+/* ------------------------------------------------------------------------- */
+void kto_unpack_copy(const void *flat, const int64_t *numel, const int64_t *tensor_offset,
+                     int T, int elem_size, void *const *out)
+{
+    for (int t = 0; t < T; ++t) {
+        const unsigned char *src = (const unsigned char *)flat + tensor_offset[t] * elem_size;
+        unsigned char *dst = (unsigned char *)out[t];
+        for (int64_t j = 0; j < numel[t] * elem_size; ++j)
+            dst[j] = src[j];
+    }
+}
+
+/* ------------------------------------------------------------------------- */
 /* Intra-group reduce (Section III-A, first bullet: the collective among the    */
 /* homogeneous devices of one group), with the in-group batch-share weights:   */
 /*   P_g[i] = sum over the ranks r of group g, ascending r, of a_r * x_r[i].     */

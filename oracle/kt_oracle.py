@@ -57,6 +57,8 @@ def lib() -> C.CDLL:
         L.kto_f32_to_bf16.restype = None
         L.kto_pack.argtypes = [vpp, i64p, i64p, C.c_int, C.c_int, C.c_int64, C.c_void_p]
         L.kto_pack.restype = None
+        L.kto_unpack_copy.argtypes = [C.c_void_p, i64p, i64p, C.c_int, C.c_int, vpp]
+        L.kto_unpack_copy.restype = None
         L.kto_intra_reduce.argtypes = [vpp, C.c_int, i64p, i64p, C.c_int, C.c_int64, i32p, f32p,
                                        C.c_int, C.c_int, vpp]
         L.kto_intra_reduce.restype = None
@@ -175,6 +177,25 @@ def pack(tensors, plan: Plan, dtype: int) -> np.ndarray:
     lib().kto_pack(_ptr_array(tensors), _p(plan.numel, C.c_int64), _p(plan.tensor_offset, C.c_int64),
                    plan.T, _ELEM[dtype], plan.transport_numel, flat.ctypes.data)
     return flat
+
+
+def unpack_copy(flat: np.ndarray, plan: Plan, dtype: int):
+    """Bit copy of every tensor out of a flat buffer; returns the list of T flat arrays."""
+    assert flat.dtype == _NP[dtype] and flat.size == plan.transport_numel
+    out = [np.empty(int(n), _NP[dtype]) for n in plan.numel]
+    lib().kto_unpack_copy(flat.ctypes.data, _p(plan.numel, C.c_int64), _p(plan.tensor_offset, C.c_int64),
+                          plan.T, _ELEM[dtype], _ptr_array(out))
+    return out
+
+
+def broadcast(tensors, root: int, numel, dtype: int, bucket_cap_bytes: int):
+    """Model synchronisation from rank `root`: tensors[r][t] are the ranks' lists.  Returns
+    (new lists of every rank, the flat buffer that crosses the host, plan): the root keeps
+    its own arrays, every other rank gets bit copies taken out of the flat buffer."""
+    plan = bucket_plan(numel, bucket_cap_bytes)
+    flat = pack(tensors[root], plan, dtype)
+    out = [list(tensors[r]) if r == root else unpack_copy(flat, plan, dtype) for r in range(len(tensors))]
+    return out, flat, plan
 
 
 def intra_reduce(grads, plan: Plan, dtype: int, group_of, a, G: int):

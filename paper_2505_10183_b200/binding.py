@@ -25,7 +25,7 @@ KT_MAX_RANKS, KT_MAX_GROUPS = 64, 16
 
 EXPORTS = ["kt_schedule", "kt_groups_init", "kt_set_shares", "kt_set_coefficients",
            "kt_get_coefficients", "kt_bucket_pack", "kt_plan_buckets", "kt_plan_query", "kt_hier_reduce",
-           "kt_stage_to_host", "kt_relay_through_host", "kt_stage_wait", "kt_unpack_scale", "kt_sync_direct", "kt_cast", "kt_copy_tensors", "kt_sync_flat_static", "kt_launch_count",
+           "kt_stage_to_host", "kt_relay_through_host", "kt_stage_wait", "kt_unpack_scale", "kt_sync_direct", "kt_bcast_send", "kt_bcast_relay", "kt_bcast_recv", "kt_cast", "kt_copy_tensors", "kt_sync_flat_static", "kt_launch_count",
            "kt_last_error", "kt_destroy"]
 
 _DTYPES = {torch.float32: KT_F32, torch.bfloat16: KT_BF16}
@@ -61,6 +61,9 @@ def _load() -> C.CDLL:
         "kt_stage_wait": ([vp, C.c_int, C.c_int, vp, C.c_int], C.c_int),
         "kt_unpack_scale": ([vp, vpp, C.c_int, vpp, C.c_int, C.c_int, C.c_float, C.c_int, vp], C.c_int),
         "kt_sync_direct": ([vp, vpp, C.c_int, C.c_int, C.c_float, C.c_int, vp], C.c_int),
+        "kt_bcast_send": ([vp, C.c_int, C.c_int, vp, vp], C.c_int),
+        "kt_bcast_relay": ([vp, C.c_int, C.c_int, vp, vp, vpp, C.c_int64, vp, vp, vp], C.c_int),
+        "kt_bcast_recv": ([vp, C.c_int, C.c_int, vpp, vp], C.c_int),
         "kt_cast": ([vp, C.c_int, vp, C.c_int, C.c_int64, vp], C.c_int),
         "kt_copy_tensors": ([vpp, vpp, i64p, C.c_int, C.c_int, vp], C.c_int),
         "kt_sync_flat_static": ([i32p, i32p, C.c_int, C.c_int, vpp, C.c_int, C.c_int64, vp, C.c_int,
@@ -302,6 +305,31 @@ def kt_sync_direct(ctx: Ctx, out_grads: Union[PtrArray, Sequence[Sequence[torch.
     _check(_lib.kt_sync_direct(ctx.handle, op.array, R, out_dtype, C.c_float(scale), int(bucket),
                                _stream(stream)))
     ctx._keep["out"] = op
+
+
+def _recv_array(ctx: Ctx, recv: Sequence[Optional[torch.Tensor]]) -> C.Array:
+    if len(recv) != ctx.G:
+        raise KtError(KT_ERR_SHAPE, "expected %d receive buffers (the root group's may be None)" % ctx.G)
+    arr = (C.c_void_p * max(ctx.G, 1))()
+    for g, t in enumerate(recv):
+        arr[g] = t.data_ptr() if t is not None else None
+    return arr
+
+
+def kt_bcast_send(ctx: Ctx, root: int, send: torch.Tensor, bucket: int = -1, stream=None) -> None:
+    _check(_lib.kt_bcast_send(ctx.handle, int(root), int(bucket), C.c_void_p(send.data_ptr()), _stream(stream)))
+
+
+def kt_bcast_relay(ctx: Ctx, root: int, send: torch.Tensor, host_pinned: torch.Tensor,
+                   recv: Sequence[Optional[torch.Tensor]], d2h_stream, h2d_stream, bucket: int = -1,
+                   chunk_bytes: int = 4 << 20, main_stream=None) -> None:
+    _check(_lib.kt_bcast_relay(ctx.handle, int(root), int(bucket), C.c_void_p(send.data_ptr()),
+                               C.c_void_p(host_pinned.data_ptr()), _recv_array(ctx, recv), int(chunk_bytes),
+                               _stream(main_stream), _stream(d2h_stream), _stream(h2d_stream)))
+
+
+def kt_bcast_recv(ctx: Ctx, root: int, recv: Sequence[Optional[torch.Tensor]], bucket: int = -1, stream=None) -> None:
+    _check(_lib.kt_bcast_recv(ctx.handle, int(root), int(bucket), _recv_array(ctx, recv), _stream(stream)))
 
 
 def kt_cast(inp: torch.Tensor, out: torch.Tensor, stream=None) -> None:

@@ -694,6 +694,20 @@ int kt_relay_through_host(kt_ctx *c, int bucket, float *const *send, float *cons
         if (!send[g] || !host_pinned[g] || !recv[g]) return fail(KT_ERR_INVALID, "buffer %d is NULL", g);
     int64_t lo, n;
     bucket_range(c, bucket, &lo, &n);
+    // When the whole transport moves and the G buffers of each set lie back to back in memory
+    // (rows of one allocation), the relay treats them as one range: one copy per chunk and
+    // direction instead of G, which matters because every copy costs the link a few microseconds.
+    int groups = c->G;
+    if (bucket < 0) {
+        bool rows = true;
+        for (int g = 0; g + 1 < c->G; ++g)
+            rows = rows && send[g + 1] == send[g] + n && host_pinned[g + 1] == host_pinned[g] + n &&
+                   recv[g + 1] == recv[g] + n;
+        if (rows) {
+            n *= c->G;
+            groups = 1;
+        }
+    }
     // Uniform chunks (elements, a multiple of 64).  Shorter chunks at the two ends of the
     // pipeline were tried and measured slower: small copies use the host link badly.
     const int64_t chunk = chunk_bytes / 256 * 64;
@@ -714,11 +728,11 @@ int kt_relay_through_host(kt_ctx *c, int bucket, float *const *send, float *cons
     int64_t at = lo;
     for (int64_t k = 0; k < n_chunks; at += sizes[k], ++k) {
         const size_t len = static_cast<size_t>(sizes[k]) * sizeof(float);
-        for (int g = 0; g < c->G; ++g)
+        for (int g = 0; g < groups; ++g)
             KT_CUDA(cudaMemcpyAsync(host_pinned[g] + at, send[g] + at, len, cudaMemcpyDeviceToHost, ds));
         KT_CUDA(cudaEventRecord(c->chunk_events[k], ds));
         KT_CUDA(cudaStreamWaitEvent(hs, c->chunk_events[k], 0));
-        for (int g = 0; g < c->G; ++g)
+        for (int g = 0; g < groups; ++g)
             KT_CUDA(cudaMemcpyAsync(recv[g] + at, host_pinned[g] + at, len, cudaMemcpyHostToDevice, hs));
     }
     StageSlot &down = c->slots[KT_D2H][bucket + 1], &up = c->slots[KT_H2D][bucket + 1];
@@ -876,6 +890,120 @@ void kt_destroy(kt_ctx *c) {
             if (s.done) cudaEventDestroy(s.done);
     for (cudaEvent_t e : c->chunk_events) cudaEventDestroy(e);
     delete c;
+}
+
+}  // extern "C"
+
+// ---------------------------------------------------------------------- hierarchical broadcast
+namespace {
+
+int fill_bcast(const kt_ctx *c, int root, BcastParams *p) {
+    if (root < 0 || root >= c->K) return fail(KT_ERR_INVALID, "root = %d outside [0, %d)", root, c->K);
+    p->ptrs = const_cast<void *const *>(reinterpret_cast<const void *const *>(c->d_ptrs));
+    p->G = c->G;
+    p->g_root = c->group_of[root];
+    for (int g = 0; g < c->G; ++g) p->k_lo[g] = p->k_hi[g] = 0;
+    for (int k = 0; k < c->K; ++k) {
+        const int g = c->group_of[c->order[k]];
+        if (k == 0 || c->group_of[c->order[k - 1]] != g) p->k_lo[g] = static_cast<unsigned char>(k);
+        p->k_hi[g] = static_cast<unsigned char>(k + 1);
+        if (c->order[k] == root) p->k_root = k;
+    }
+    return KT_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int kt_bcast_send(kt_ctx *c, int root, int bucket, void *send, void *stream) {
+    if (int rc = check_ctx(c, true)) return rc;
+    if (!send) return fail(KT_ERR_INVALID, "send is NULL");
+    if (!aligned16(send)) return fail(KT_ERR_ALIGN, "send is not 16-byte aligned");
+    BcastParams p{};
+    if (int rc = fill_bcast(c, root, &p)) return rc;
+    if (int rc = make_tile_plan(c, bucket, &p.tp)) return rc;
+    if (p.tp.n_tiles == 0) return KT_OK;
+    p.flat[p.g_root] = send;
+    KT_CUDA(cudaSetDevice(c->device));
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (c->in_dtype == KT_F32) k_bcast_send<float><<<p.tp.n_tiles, NT, 0, s>>>(p);
+    else k_bcast_send<unsigned short><<<p.tp.n_tiles, NT, 0, s>>>(p);
+    c->launches += 1;
+    KT_CUDA(cudaGetLastError());
+    return KT_OK;
+}
+
+int kt_bcast_recv(kt_ctx *c, int root, int bucket, void *const *recv, void *stream) {
+    if (int rc = check_ctx(c, true)) return rc;
+    if (!recv) return fail(KT_ERR_INVALID, "recv is NULL");
+    BcastParams p{};
+    if (int rc = fill_bcast(c, root, &p)) return rc;
+    for (int g = 0; g < c->G; ++g) {
+        if (g == p.g_root) continue;
+        if (!recv[g]) return fail(KT_ERR_INVALID, "recv[%d] is NULL", g);
+        if (!aligned16(recv[g])) return fail(KT_ERR_ALIGN, "recv[%d] is not 16-byte aligned", g);
+        p.flat[g] = recv[g];
+    }
+    if (int rc = make_tile_plan(c, bucket, &p.tp)) return rc;
+    if (p.tp.n_tiles == 0 || c->G == 1) return KT_OK;
+    KT_CUDA(cudaSetDevice(c->device));
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (c->in_dtype == KT_F32) k_bcast_recv<float><<<p.tp.n_tiles, NT, 0, s>>>(p);
+    else k_bcast_recv<unsigned short><<<p.tp.n_tiles, NT, 0, s>>>(p);
+    c->launches += 1;
+    KT_CUDA(cudaGetLastError());
+    return KT_OK;
+}
+
+int kt_bcast_relay(kt_ctx *c, int root, int bucket, const void *send, void *host_pinned, void *const *recv,
+                   int64_t chunk_bytes, void *main_stream, void *d2h_stream, void *h2d_stream) {
+    if (int rc = check_ctx(c, true)) return rc;
+    if (!send || !host_pinned || !recv) return fail(KT_ERR_INVALID, "NULL argument");
+    if (root < 0 || root >= c->K) return fail(KT_ERR_INVALID, "root = %d outside [0, %d)", root, c->K);
+    if (bucket < -1 || bucket >= static_cast<int>(c->bucket_start.size()))
+        return fail(KT_ERR_SHAPE, "bucket %d out of range", bucket);
+    if (chunk_bytes < 256) return fail(KT_ERR_INVALID, "chunk_bytes must be >= 256");
+    if (d2h_stream == h2d_stream) return fail(KT_ERR_INVALID, "the two copy streams must differ");
+    const int g_root = c->group_of[root];
+    for (int g = 0; g < c->G; ++g)
+        if (g != g_root && !recv[g]) return fail(KT_ERR_INVALID, "recv[%d] is NULL", g);
+    int64_t lo, n;
+    bucket_range(c, bucket, &lo, &n);
+    const size_t es = c->in_dtype == KT_F32 ? 4 : 2;
+    const int64_t chunk = chunk_bytes / 256 * 256 / static_cast<int64_t>(es);   // elements per chunk
+    std::vector<int64_t> sizes;
+    for (int64_t left = n; left > 0; left -= sizes.back()) sizes.push_back(left < chunk ? left : chunk);
+    const int64_t n_chunks = static_cast<int64_t>(sizes.size());
+    KT_CUDA(cudaSetDevice(c->device));
+    while (static_cast<int64_t>(c->chunk_events.size()) < n_chunks) {
+        cudaEvent_t e;
+        KT_CUDA(cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
+        c->chunk_events.push_back(e);
+    }
+    cudaStream_t ms = static_cast<cudaStream_t>(main_stream);
+    cudaStream_t ds = static_cast<cudaStream_t>(d2h_stream), hs = static_cast<cudaStream_t>(h2d_stream);
+    KT_CUDA(cudaEventRecord(c->ev_main, ms));
+    KT_CUDA(cudaStreamWaitEvent(ds, c->ev_main, 0));
+    KT_CUDA(cudaStreamWaitEvent(hs, c->ev_main, 0));
+    const char *src = static_cast<const char *>(send);
+    char *host = static_cast<char *>(host_pinned);
+    int64_t at = lo;
+    for (int64_t k = 0; k < n_chunks; at += sizes[k], ++k) {
+        const size_t off = static_cast<size_t>(at) * es, len = static_cast<size_t>(sizes[k]) * es;
+        KT_CUDA(cudaMemcpyAsync(host + off, src + off, len, cudaMemcpyDeviceToHost, ds));
+        KT_CUDA(cudaEventRecord(c->chunk_events[k], ds));
+        KT_CUDA(cudaStreamWaitEvent(hs, c->chunk_events[k], 0));
+        for (int g = 0; g < c->G; ++g)
+            if (g != g_root)
+                KT_CUDA(cudaMemcpyAsync(static_cast<char *>(recv[g]) + off, host + off, len, cudaMemcpyHostToDevice, hs));
+    }
+    StageSlot &down = c->slots[KT_D2H][bucket + 1], &up = c->slots[KT_H2D][bucket + 1];
+    KT_CUDA(cudaEventRecord(down.done, ds));
+    down.recorded = true;
+    KT_CUDA(cudaEventRecord(up.done, hs));
+    up.recorded = true;
+    return KT_OK;
 }
 
 }  // extern "C"

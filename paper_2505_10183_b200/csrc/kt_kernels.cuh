@@ -107,6 +107,15 @@ struct DirectParams {
     float scale;
 };
 
+struct BcastParams {
+    TilePlan tp;
+    void *const *ptrs;                     // [K][T] registered tensors, group-major rank order
+    void *flat[KT_MAX_GROUPS];             // send: [g_root] is written; recv: [g != g_root] are read
+    unsigned char k_lo[KT_MAX_GROUPS];     // members of group g: ranks [k_lo[g], k_hi[g]) of that order
+    unsigned char k_hi[KT_MAX_GROUPS];
+    int G, g_root, k_root;
+};
+
 struct PackParams {
     TilePlan tp;
     const void *const *ptrs;           // [K][T], group-major rank order
@@ -537,6 +546,86 @@ __global__ void __launch_bounds__(NT) k_pack(const __grid_constant__ PackParams 
         const long long e = t.e0 + (it * NT + threadIdx.x) * VEC;
         // ext is a multiple of 8 elements, so a vector that starts below ext ends inside it
         if (e < t.ti.ext) *reinterpret_cast<uint4 *>(flat + e) = raw[it];
+    }
+}
+
+// ------------------------------------------------------------------ hierarchical broadcast (model synchronisation)
+// Section III-A routes Broadcast like AllReduce: inside the root's group directly, to the
+// other groups through host RAM.  Both kernels are bit copies.
+//
+// element c of a 16-byte vector written to d[c] for the elements below n (tails, misaligned tensors)
+template <typename Tv>
+__device__ __forceinline__ void store_elems(Tv *d, const uint4 &v, long long e, long long n) {
+    const unsigned w[4] = {v.x, v.y, v.z, v.w};
+    constexpr int VEC = Elem<Tv>::VEC;
+#pragma unroll
+    for (int c = 0; c < VEC; ++c) {
+        if (e + c >= n) break;
+        if constexpr (sizeof(Tv) == 4) d[e + c] = __uint_as_float(w[c]);
+        else d[e + c] = static_cast<unsigned short>(w[c / 2] >> (16 * (c & 1)));
+    }
+}
+
+// send side: the root's tensors are read once; every element goes to the flat send buffer of
+// the root's group (plan offsets, zero padding) and to the tensors of the root's group mates
+template <typename Tv>
+__global__ void __launch_bounds__(NT) k_bcast_send(const __grid_constant__ BcastParams p) {
+    constexpr int VEC = Elem<Tv>::VEC;
+    constexpr int ITERS = Elem<Tv>::TILE / (NT * VEC);
+    const TileRef t = locate_tile(p.tp);
+    const int T = p.tp.T;
+    const Tv *s = static_cast<const Tv *>(ldg_ptr(&p.ptrs[static_cast<size_t>(p.k_root) * T + t.u]));
+    Tv *flat = static_cast<Tv *>(p.flat[p.g_root]) + t.ti.dst_off;
+    const bool aligned = t.ti.flags & FLAG_ALIGNED;
+    uint4 raw[ITERS];
+    long long e[ITERS];
+#pragma unroll
+    for (int it = 0; it < ITERS; ++it) {
+        e[it] = t.e0 + (it * NT + threadIdx.x) * VEC;
+        if (aligned && e[it] + VEC <= t.ti.numel) raw[it] = ld_stream(s + e[it]);
+        else raw[it] = Elem<Tv>::gather(s, e[it], t.ti.numel);
+    }
+#pragma unroll
+    for (int it = 0; it < ITERS; ++it)
+        if (e[it] < t.ti.ext) *reinterpret_cast<uint4 *>(flat + e[it]) = raw[it];
+    for (int k = p.k_lo[p.g_root]; k < p.k_hi[p.g_root]; ++k) {
+        if (k == p.k_root) continue;
+        Tv *d = static_cast<Tv *>(ldg_ptr(&p.ptrs[static_cast<size_t>(k) * T + t.u]));
+#pragma unroll
+        for (int it = 0; it < ITERS; ++it) {
+            if (aligned && e[it] + VEC <= t.ti.numel) *reinterpret_cast<uint4 *>(d + e[it]) = raw[it];
+            else store_elems<Tv>(d, raw[it], e[it], t.ti.numel);
+        }
+    }
+}
+
+// receive side: every other group reads its own flat receive buffer once and writes the
+// tensors of all its members
+template <typename Tv>
+__global__ void __launch_bounds__(NT) k_bcast_recv(const __grid_constant__ BcastParams p) {
+    constexpr int VEC = Elem<Tv>::VEC;
+    constexpr int ITERS = Elem<Tv>::TILE / (NT * VEC);
+    const TileRef t = locate_tile(p.tp);
+    const int T = p.tp.T;
+    const bool aligned = t.ti.flags & FLAG_ALIGNED;
+    long long e[ITERS];
+#pragma unroll
+    for (int it = 0; it < ITERS; ++it) e[it] = t.e0 + (it * NT + threadIdx.x) * VEC;
+    for (int g = 0; g < p.G; ++g) {
+        if (g == p.g_root) continue;
+        const Tv *s = static_cast<const Tv *>(p.flat[g]) + t.ti.dst_off;
+        uint4 raw[ITERS];
+#pragma unroll
+        for (int it = 0; it < ITERS; ++it)   // ext is a multiple of 8 elements: a vector below ext is readable
+            raw[it] = e[it] < t.ti.ext ? ld_stream(s + e[it]) : make_uint4(0u, 0u, 0u, 0u);
+        for (int k = p.k_lo[g]; k < p.k_hi[g]; ++k) {
+            Tv *d = static_cast<Tv *>(ldg_ptr(&p.ptrs[static_cast<size_t>(k) * T + t.u]));
+#pragma unroll
+            for (int it = 0; it < ITERS; ++it) {
+                if (aligned && e[it] + VEC <= t.ti.numel) *reinterpret_cast<uint4 *>(d + e[it]) = raw[it];
+                else store_elems<Tv>(d, raw[it], e[it], t.ti.numel);
+            }
+        }
     }
 }
 

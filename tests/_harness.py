@@ -40,20 +40,28 @@ def shares_of(wl, kt=None):
 
 
 def run_gpu_path(kt, wl, dev_grads, shares, out_dtype=None, R=1, scale=1.0, per_bucket=False,
-                 use_combined=False, staged=False, relay_chunk=4 << 20):
+                 use_combined=False, staged=False, relay_chunk=4 << 20, rows=False):
     """Returns (out[c][t] tensors, transport list, plan, ctx)."""
     ctx = kt.kt_groups_init(wl.group_of, shares, wl.G)
     kt.kt_bucket_pack(ctx, dev_grads, wl.bucket_cap_bytes)
     plan = kt.kt_plan_query(ctx)
     n = plan.transport_numel
-    transport = [torch.full((n,), float("nan"), device="cuda") for _ in range(wl.G)]
+    # rows=True: the G buffers of each set are rows of one allocation (the relay then moves a
+    # chunk of all groups in one copy)
+    def buffers(pinned=False):
+        if rows:
+            whole = torch.full((wl.G, n), float("nan"), device=None if pinned else "cuda")
+            return list(whole.pin_memory() if pinned else whole)
+        return [torch.full((n,), float("nan")).pin_memory() if pinned else torch.full((n,), float("nan"), device="cuda")
+                for _ in range(wl.G)]
+    transport = buffers()
     odt = TORCH_DT[wl.dtype] if out_dtype is None else out_dtype
     out = [[torch.full((m,), float("nan"), dtype=odt, device="cuda") for m in wl.numel] for _ in range(R)]
     buckets = list(range(plan.n_buckets)) if per_bucket else [-1]
     src = transport
     if staged:
-        host = [torch.empty(n, dtype=torch.float32).pin_memory() for _ in range(wl.G)]
-        recv = [torch.full((n,), float("nan"), device="cuda") for _ in range(wl.G)]
+        host = buffers(pinned=True)
+        recv = buffers()
         side = torch.cuda.Stream()
         src = recv
     if staged in ("relay", "relay_all"):

@@ -96,6 +96,18 @@ def test_resnet18_staged_as_benchmarked(kt, oracle):
     compare_all(kt, oracle, wl, staged="relay", relay_chunk=1 << 30)
 
 
+def test_relay_with_group_buffers_as_rows_of_one_allocation(kt, oracle):
+    """The layout the benchmark uses: transport, pinned and receive buffers of the G groups
+    back to back, so that the relay moves a chunk of all groups in one copy.  Chunk sizes
+    that do and do not divide a row, three groups, and the per-bucket relay (which cannot merge)."""
+    wl = W.resnet18()
+    compare_all(kt, oracle, wl, staged="relay_all", relay_chunk=4 << 20, rows=True)
+    compare_all(kt, oracle, wl, staged="relay_all", relay_chunk=(3 << 20) + 256, rows=True)
+    compare_all(kt, oracle, wl, staged="relay", rows=True)
+    compare_all(kt, oracle, W.mobilenet_v2(), staged="relay_all", relay_chunk=1 << 20, rows=True)
+    compare_all(kt, oracle, W.tiny(), staged="relay_all", relay_chunk=256, rows=True)
+
+
 def test_resnet18_staged_bucket_by_bucket(kt, oracle):
     """The per-bucket route: reduce, copy down, copy up and unpack one bucket at a time."""
     wl = W.resnet18()

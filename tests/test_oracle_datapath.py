@@ -316,3 +316,39 @@ def test_threaded_slices_equal_single_thread(oracle):
     out, *_ = run_path(oracle, [[xr] for xr in x], [n], F32, [0, 0, 1, 1], [79, 79, 49, 49], 2)
     thr = oracle.sync_step_flat_threads(x, F32, [0, 0, 1, 1], [79, 79, 49, 49], 2, 1.0, F32, 3)
     assert np.array_equal(out[0], thr)
+
+
+# ----------------------------------------------------------------------------- broadcast
+@pytest.mark.parametrize("dtype", [F32, BF16])
+def test_broadcast_hands_every_rank_the_roots_bytes(oracle, dtype):
+    """Pin for the broadcast oracle: numpy's own array comparison on raw bit patterns, with
+    values a careless copy would change (NaNs with payloads, signalling NaNs, -0, denormals,
+    infinities), odd sizes and an empty tensor; the flat buffer holds the root's tensors at the
+    plan's offsets and zeros elsewhere (checked by numpy slicing, not by the oracle's unpack)."""
+    rng = np.random.default_rng(11)
+    numel = [0, 1, 7, 8, 9, 64, 1000, 4097]
+    K, root = 5, 3
+    udt = np.uint32 if dtype == F32 else np.uint16
+    special = np.array([0x7FC00001, 0x7F800001, 0xFFC12345, 0x80000000, 0x00000001, 0x807FFFFF,
+                        0x7F800000, 0xFF800000], dtype=np.uint32)
+    special = special if dtype == F32 else (special >> 16).astype(np.uint16) | np.uint16(1)
+    ranks = []
+    for r in range(K):
+        row = []
+        for n in numel:
+            bits = rng.integers(0, np.iinfo(udt).max, size=n, dtype=udt, endpoint=True)
+            bits[: min(n, special.size)] = special[: min(n, special.size)]
+            row.append(bits.view(np.float32) if dtype == F32 else bits)
+        ranks.append(row)
+    before_root = [a.copy() for a in ranks[root]]
+    out, flat, plan = oracle.broadcast(ranks, root, numel, dtype, 4096)
+    covered = np.zeros(plan.transport_numel, bool)
+    for t, n in enumerate(numel):
+        off = int(plan.tensor_offset[t])
+        assert np.array_equal(flat[off:off + n].view(udt), before_root[t].view(udt))
+        covered[off:off + n] = True
+    assert not flat.view(udt)[~covered].any()
+    for r in range(K):
+        for t in range(len(numel)):
+            assert out[r][t].dtype == before_root[t].dtype
+            assert np.array_equal(out[r][t].view(udt), before_root[t].view(udt)), (r, t)
