@@ -45,6 +45,7 @@ extern "C" {
 #endif
 
 typedef struct kt_ctx kt_ctx;
+typedef struct kt_adapt kt_adapt;
 
 typedef enum { KT_F32 = 0, KT_BF16 = 1 } kt_dtype;
 
@@ -74,6 +75,45 @@ typedef enum { KT_D2H = 0, KT_H2D = 1 } kt_stage_dir;
  * then the higher rank).  Requires 1 <= K <= KT_MAX_RANKS and global_batch >= K.
  * Errors: KT_ERR_INVALID. */
 int kt_schedule(const double *step_times, int K, int global_batch, int32_t *shares_out);
+
+/* Online adaptation of the scores (Section III-C, "Online Adaptation": monitor computation
+ * times per batch during training and adjust the scores; the paper leaves the rule open).
+ * Rule used here: a rank's measured step time T_r was spent on its current share b_r, so
+ * tau_r = T_r / b_r (time per sample) is what reflects its speed; tau_r is smoothed with an
+ * exponential moving average of factor alpha (first observation initialises it); every
+ * `period` observations kt_schedule is run on the smoothed tau; the result replaces the
+ * shares in use only if the step time it predicts, max_r tau_r * b_r, is below
+ * (1 - hysteresis) times the prediction for the shares in use.
+ * kt_adapt_create: shares[K] (host) are the shares in use at the start, summing to
+ *        global_batch; alpha in (0, 1]; period >= 1; hysteresis in [0, 1).
+ * kt_adapt_observe: step_times[K] (host), finite and > 0, measured with the shares in use;
+ *        shares_out[K] (host, may be NULL) receives the shares to use from now on, *changed
+ *        (may be NULL) whether they differ from before.  Pure host arithmetic in double.
+ * kt_adapt_state: read-back of the smoothed per-sample times, shares, observation count
+ *        (each may be NULL).
+ * Errors: KT_ERR_INVALID, KT_ERR_NOMEM. */
+int kt_adapt_create(const int32_t *shares, int K, int global_batch, double alpha, int period,
+                    double hysteresis, kt_adapt **out);
+int kt_adapt_observe(kt_adapt *state, const double *step_times, int32_t *shares_out, int *changed);
+int kt_adapt_state(const kt_adapt *state, double *per_sample_out, int32_t *shares_out,
+                   int64_t *count_out);
+void kt_adapt_destroy(kt_adapt *state);
+
+/* Load-adaptive sampler (Section III-C "Dynamic Data Allocation"; Section IV-A: a sampler
+ * that takes the per-device scores and distributes dataset indices accordingly).  With
+ * B = sum of shares and c_r = shares[0] + ... + shares[r-1]: step s of an epoch consumes
+ * positions [s*B, (s+1)*B) of the epoch's index list, rank r the shares[r] consecutive
+ * positions from s*B + c_r on; rank r's epoch list is its slices of all steps in order,
+ *   out[r][s*shares[r] + j] = list[(s*B + c_r + j) mod dataset_size].
+ * kt_sampler_steps: steps per epoch: floor(D / B) with drop_last, else ceil(D / B) (the list
+ *        is continued from its own start); negative kt_status on bad arguments.
+ * kt_sampler_indices: list (device, int64[dataset_size], or NULL for the identity = no
+ *        shuffling) is the epoch's permutation, drawn by the caller; shares[K] (host);
+ *        out: host array of K device pointers, out[r] holding steps * shares[r] int64.
+ *        One kernel on `stream`.  Errors: KT_ERR_INVALID, KT_ERR_SHAPE, KT_ERR_ALIGN, KT_ERR_CUDA. */
+int64_t kt_sampler_steps(int64_t dataset_size, int64_t global_batch, int drop_last);
+int kt_sampler_indices(const int64_t *list, int64_t dataset_size, const int32_t *shares, int K,
+                       int drop_last, int64_t *const *out, void *stream);
 
 /* Sections III-A (groups of homogeneous devices) and III-C (shares).
  * group_of[K] (host): group index of every rank, each in [0, G), no group empty.

@@ -120,6 +120,117 @@ int kto_schedule(const double *step_times, int K, int global_batch, int32_t *sha
 }
 
 /* ------------------------------------------------------------------------- */
+/* Online adaptation of the scores (Section III-C names it as future work:      */
+/* "continuously monitor computation times per batch during training and        */
+/* dynamically adjust scores").  The paper gives no rule; the reading used:     */
+/*  - a rank's measured step time T_r was spent on b_r samples, so its speed    */
+/*    shows in the per-sample time tau_r = T_r / b_r (the initial benchmark of   */
+/*    Section III-C gives every device the same amount of data, where time and   */
+/*    per-sample time are proportional);                                       */
+/*  - tau_r is smoothed by an exponential moving average with factor alpha      */
+/*    (the first observation initialises it);                                  */
+/*  - every `period` observations the schedule of Section III-C is recomputed   */
+/*    from the smoothed per-sample times; the new shares are adopted only if     */
+/*    the step time they predict, max_r tau_r * b_r, is below (1 - hysteresis)   */
+/*    times the one predicted for the shares in use, so that measurement noise   */
+/*    does not make the shares flip back and forth.                            */
+/* State is held by the caller: ema[K] (doubles), shares[K], *count.            */
+/* Returns 1 if the shares changed, 0 if not, KTO_ERR_INVALID on bad input.      */
+/* ------------------------------------------------------------------------- */
+int kto_adapt_observe(double *ema, int32_t *shares, int64_t *count, int K, int global_batch,
+                      double alpha, int period, double hysteresis, const double *step_times)
+{
+    if (!ema || !shares || !count || !step_times || K < 1 || period < 1 || !(alpha > 0.0) ||
+        !(alpha <= 1.0) || !(hysteresis >= 0.0) || !(hysteresis < 1.0))
+        return KTO_ERR_INVALID;
+    for (int r = 0; r < K; ++r)
+        if (!(step_times[r] > 0.0) || !isfinite(step_times[r]) || shares[r] < 1)
+            return KTO_ERR_INVALID;
+    for (int r = 0; r < K; ++r) {
+        double tau = step_times[r] / (double)shares[r];
+        if (*count == 0)
+            ema[r] = tau;
+        else
+            ema[r] = (1.0 - alpha) * ema[r] + alpha * tau;
+    }
+    *count += 1;
+    if (*count % period != 0)
+        return 0;
+    int32_t *cand = (int32_t *)malloc(sizeof(int32_t) * (size_t)K);
+    if (!cand)
+        return KTO_ERR_INVALID;
+    if (kto_schedule(ema, K, global_batch, cand) != KTO_OK) {
+        free(cand);
+        return KTO_ERR_INVALID;
+    }
+    double now = 0.0, then = 0.0;
+    int differs = 0;
+    for (int r = 0; r < K; ++r) {
+        double a = ema[r] * (double)shares[r], b = ema[r] * (double)cand[r];
+        if (a > now)
+            now = a;
+        if (b > then)
+            then = b;
+        if (cand[r] != shares[r])
+            differs = 1;
+    }
+    int adopt = differs && then < (1.0 - hysteresis) * now;
+    if (adopt)
+        for (int r = 0; r < K; ++r)
+            shares[r] = cand[r];
+    free(cand);
+    return adopt;
+}
+
+/* ------------------------------------------------------------------------- */
+/* Load-adaptive sampler (Section III-C "Dynamic Data Allocation", Section IV-A  */
+/* "DistributedSampler Override": the sampler takes the per-device scores and   */
+/* distributes dataset indices accordingly).  With the integer shares b_r of     */
+/* the schedule, B = sum b_r and c_r = b_0 + ... + b_{r-1}:                       */
+/*  - an epoch has S = floor(D / B) steps when the incomplete last batch is      */
+/*    dropped, else S = ceil(D / B), the index list being continued from its     */
+/*    own start (position p reads list entry p mod D);                         */
+/*  - step s consumes positions [s B, (s+1) B) of the epoch's index list; rank r  */
+/*    takes the b_r consecutive positions starting at s B + c_r;                */
+/*  - rank r's epoch list is its slices of steps 0..S-1 one after the other:     */
+/*      out_r[s b_r + j] = list[(s B + c_r + j) mod D],  0 <= j < b_r.            */
+/* list is the epoch's permutation of 0..D-1 (NULL = identity, no shuffling);   */
+/* how it is drawn is outside this function.                                   */
+/* ------------------------------------------------------------------------- */
+int64_t kto_sampler_steps(int64_t dataset_size, int64_t global_batch, int drop_last)
+{
+    if (dataset_size < 1 || global_batch < 1)
+        return -1;
+    if (drop_last)
+        return dataset_size / global_batch;
+    return (dataset_size + global_batch - 1) / global_batch;
+}
+
+int kto_sampler_indices(const int64_t *list, int64_t dataset_size, const int32_t *shares, int K,
+                        int drop_last, int64_t *const *out)
+{
+    if (!shares || !out || K < 1 || dataset_size < 1)
+        return KTO_ERR_INVALID;
+    int64_t B = 0;
+    for (int r = 0; r < K; ++r) {
+        if (shares[r] < 1)
+            return KTO_ERR_INVALID;
+        B += shares[r];
+    }
+    const int64_t S = kto_sampler_steps(dataset_size, B, drop_last);
+    int64_t c = 0; /* c_r */
+    for (int r = 0; r < K; ++r) {
+        for (int64_t s = 0; s < S; ++s)
+            for (int64_t j = 0; j < shares[r]; ++j) {
+                int64_t p = (s * B + c + j) % dataset_size;
+                out[r][s * shares[r] + j] = list ? list[p] : p;
+            }
+        c += shares[r];
+    }
+    return KTO_OK;
+}
+
+/* ------------------------------------------------------------------------- */
 /* Weights of the two-level mean (Section III-A groups, Section III-C shares).  */
 /* B_g = sum of the shares of group g, B = sum of all shares.                  */
 /* a_r = b_r / B_g  (weight of rank r inside its group),                       */

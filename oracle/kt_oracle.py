@@ -47,6 +47,13 @@ def lib() -> C.CDLL:
         vpp = C.POINTER(C.c_void_p)
         L.kto_schedule.argtypes = [f64p, C.c_int, C.c_int, i32p]
         L.kto_schedule.restype = C.c_int
+        L.kto_adapt_observe.argtypes = [f64p, i32p, i64p, C.c_int, C.c_int, C.c_double, C.c_int,
+                                        C.c_double, f64p]
+        L.kto_adapt_observe.restype = C.c_int
+        L.kto_sampler_steps.argtypes = [C.c_int64, C.c_int64, C.c_int]
+        L.kto_sampler_steps.restype = C.c_int64
+        L.kto_sampler_indices.argtypes = [i64p, C.c_int64, i32p, C.c_int, C.c_int, vpp]
+        L.kto_sampler_indices.restype = C.c_int
         L.kto_coefficients.argtypes = [i32p, i32p, C.c_int, C.c_int, f32p, f32p, f32p]
         L.kto_coefficients.restype = C.c_int
         L.kto_bucket_plan.argtypes = [i64p, C.c_int, C.c_int64, i64p, i32p, i64p, i64p, i32p, i64p]
@@ -104,6 +111,53 @@ def schedule(step_times, global_batch: int) -> np.ndarray:
     rc = lib().kto_schedule(_p(t, C.c_double), int(t.size), int(global_batch), _p(out, C.c_int32))
     if rc != 0:
         raise OracleError("kto_schedule: invalid arguments")
+    return out
+
+
+class Adapter:
+    """Caller-held state of the online adaptation: smoothed per-sample times, the shares in
+    use and the number of observations so far."""
+
+    def __init__(self, shares, global_batch: int, alpha: float, period: int, hysteresis: float):
+        self.shares = np.ascontiguousarray(shares, dtype=np.int32).copy()
+        self.ema = np.zeros(self.shares.size, np.float64)
+        self.count = C.c_int64(0)
+        self.B, self.alpha, self.period, self.hysteresis = int(global_batch), float(alpha), int(period), float(hysteresis)
+
+    def observe(self, step_times) -> bool:
+        t = np.ascontiguousarray(step_times, dtype=np.float64)
+        if t.size != self.shares.size:
+            raise OracleError("expected %d step times" % self.shares.size)
+        rc = lib().kto_adapt_observe(_p(self.ema, C.c_double), _p(self.shares, C.c_int32), C.byref(self.count),
+                                     int(t.size), self.B, self.alpha, self.period, self.hysteresis,
+                                     _p(t, C.c_double))
+        if rc < 0:
+            raise OracleError("kto_adapt_observe: invalid arguments")
+        return bool(rc)
+
+
+def sampler_steps(dataset_size: int, global_batch: int, drop_last: bool) -> int:
+    s = lib().kto_sampler_steps(int(dataset_size), int(global_batch), int(bool(drop_last)))
+    if s < 0:
+        raise OracleError("kto_sampler_steps: invalid arguments")
+    return int(s)
+
+
+def sampler_indices(index_list, dataset_size: int, shares, drop_last: bool):
+    """Returns the list of K per-rank epoch index arrays (int64)."""
+    b = np.ascontiguousarray(shares, dtype=np.int32)
+    if b.size < 1 or (b < 1).any() or dataset_size < 1:
+        raise OracleError("kto_sampler_indices: invalid arguments")
+    S = sampler_steps(dataset_size, int(b.sum()), drop_last)
+    out = [np.empty(S * int(v), np.int64) for v in b]
+    lst = None
+    if index_list is not None:
+        lst = np.ascontiguousarray(index_list, dtype=np.int64)
+        assert lst.size == dataset_size
+    rc = lib().kto_sampler_indices(_p(lst, C.c_int64) if lst is not None else None, int(dataset_size),
+                                   _p(b, C.c_int32), int(b.size), int(bool(drop_last)), _ptr_array(out))
+    if rc != 0:
+        raise OracleError("kto_sampler_indices: invalid arguments")
     return out
 
 

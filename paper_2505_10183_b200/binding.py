@@ -23,7 +23,8 @@ KT_OK, KT_ERR_INVALID, KT_ERR_SHAPE, KT_ERR_ALIGN = 0, -1, -2, -3
 KT_ERR_CUDA, KT_ERR_TIMEOUT, KT_ERR_STATE, KT_ERR_NOMEM = -4, -5, -6, -7
 KT_MAX_RANKS, KT_MAX_GROUPS = 64, 16
 
-EXPORTS = ["kt_schedule", "kt_groups_init", "kt_set_shares", "kt_set_coefficients",
+EXPORTS = ["kt_schedule", "kt_adapt_create", "kt_adapt_observe", "kt_adapt_state", "kt_adapt_destroy",
+           "kt_sampler_steps", "kt_sampler_indices", "kt_groups_init", "kt_set_shares", "kt_set_coefficients",
            "kt_get_coefficients", "kt_bucket_pack", "kt_plan_buckets", "kt_plan_query", "kt_hier_reduce",
            "kt_stage_to_host", "kt_relay_through_host", "kt_stage_wait", "kt_unpack_scale", "kt_sync_direct", "kt_bcast_send", "kt_bcast_relay", "kt_bcast_recv", "kt_cast", "kt_copy_tensors", "kt_sync_flat_static", "kt_launch_count",
            "kt_last_error", "kt_destroy"]
@@ -48,6 +49,12 @@ def _load() -> C.CDLL:
     vpp = C.POINTER(C.c_void_p)
     sigs = {
         "kt_schedule": ([C.POINTER(C.c_double), C.c_int, C.c_int, i32p], C.c_int),
+        "kt_adapt_create": ([i32p, C.c_int, C.c_int, C.c_double, C.c_int, C.c_double, vpp], C.c_int),
+        "kt_adapt_observe": ([vp, C.POINTER(C.c_double), i32p, C.POINTER(C.c_int)], C.c_int),
+        "kt_adapt_state": ([vp, C.POINTER(C.c_double), i32p, i64p], C.c_int),
+        "kt_adapt_destroy": ([vp], None),
+        "kt_sampler_steps": ([C.c_int64, C.c_int64, C.c_int], C.c_int64),
+        "kt_sampler_indices": ([vp, C.c_int64, i32p, C.c_int, C.c_int, vpp, vp], C.c_int),
         "kt_groups_init": ([i32p, i32p, C.c_int, C.c_int, vpp], C.c_int),
         "kt_set_shares": ([vp, i32p], C.c_int),
         "kt_set_coefficients": ([vp, f32p, f32p], C.c_int),
@@ -147,6 +154,81 @@ def kt_schedule(step_times: Sequence[float], global_batch: int) -> List[int]:
     out = (C.c_int32 * max(K, 1))()
     _check(_lib.kt_schedule(t, K, int(global_batch), out))
     return [int(out[i]) for i in range(K)]
+
+
+class Adapt:
+    """Handle of the online adaptation state (kt_adapt_create)."""
+
+    def __init__(self, handle: int, K: int):
+        self.handle = C.c_void_p(handle)
+        self.K = K
+
+    def __del__(self):
+        try:
+            kt_adapt_destroy(self)
+        except Exception:
+            pass
+
+
+def kt_adapt_create(shares: Sequence[int], global_batch: int, alpha: float, period: int, hysteresis: float) -> Adapt:
+    h = C.c_void_p()
+    _check(_lib.kt_adapt_create(_i32(shares), len(shares), int(global_batch), float(alpha), int(period),
+                                float(hysteresis), C.byref(h)))
+    return Adapt(h.value, len(shares))
+
+
+def kt_adapt_observe(state: Adapt, step_times: Sequence[float]):
+    """Returns (shares to use from now on, whether they changed)."""
+    if len(step_times) != state.K:
+        raise KtError(KT_ERR_SHAPE, "expected %d step times" % state.K)
+    t = (C.c_double * state.K)(*[float(x) for x in step_times])
+    out = (C.c_int32 * state.K)()
+    changed = C.c_int(0)
+    _check(_lib.kt_adapt_observe(state.handle, t, out, C.byref(changed)))
+    return [int(v) for v in out], bool(changed.value)
+
+
+def kt_adapt_state(state: Adapt):
+    """Returns (smoothed per-sample times, shares in use, number of observations)."""
+    tau = (C.c_double * state.K)()
+    b = (C.c_int32 * state.K)()
+    n = C.c_int64(0)
+    _check(_lib.kt_adapt_state(state.handle, tau, b, C.byref(n)))
+    return [float(v) for v in tau], [int(v) for v in b], int(n.value)
+
+
+def kt_adapt_destroy(state: Adapt) -> None:
+    if state.handle is not None and state.handle.value:
+        _lib.kt_adapt_destroy(state.handle)
+        state.handle = C.c_void_p(None)
+
+
+def kt_sampler_steps(dataset_size: int, global_batch: int, drop_last: bool) -> int:
+    s = int(_lib.kt_sampler_steps(int(dataset_size), int(global_batch), int(bool(drop_last))))
+    _check(s if s < 0 else 0)
+    return s
+
+
+def kt_sampler_indices(index_list: Optional[torch.Tensor], dataset_size: int, shares: Sequence[int],
+                       out: Sequence[torch.Tensor], drop_last: bool = False, stream=None) -> None:
+    """index_list: int64 device tensor of dataset_size entries (the epoch's permutation) or None;
+    out[r]: int64 device tensor of kt_sampler_steps(...) * shares[r] entries."""
+    K = len(shares)
+    if len(out) != K:
+        raise KtError(KT_ERR_SHAPE, "expected %d output tensors" % K)
+    if any(t.dtype != torch.int64 or not t.is_contiguous() for t in out):
+        raise KtError(KT_ERR_SHAPE, "out: int64 contiguous tensors expected")
+    if index_list is not None and (index_list.dtype != torch.int64 or index_list.numel() != dataset_size
+                                   or not index_list.is_contiguous()):
+        raise KtError(KT_ERR_SHAPE, "index_list: int64 contiguous tensor of dataset_size entries expected")
+    if K >= 1 and all(int(b) >= 1 for b in shares) and dataset_size >= 1:
+        steps = kt_sampler_steps(dataset_size, sum(int(b) for b in shares), drop_last)
+        if any(t.numel() != steps * int(b) for t, b in zip(out, shares)):
+            raise KtError(KT_ERR_SHAPE, "out[r] must hold steps * shares[r] = %d * shares[r] entries" % steps)
+    pa = PtrArray(out)
+    _check(_lib.kt_sampler_indices(C.c_void_p(index_list.data_ptr()) if index_list is not None else None,
+                                   int(dataset_size), _i32(shares), K, int(bool(drop_last)), pa.array,
+                                   _stream(stream)))
 
 
 def kt_groups_init(group_of: Sequence[int], shares: Sequence[int], G: Optional[int] = None) -> Ctx:

@@ -18,6 +18,7 @@
 
 #include "kt_kernels.cuh"
 
+#include <algorithm>
 #include <chrono>
 #include <cmath>
 #include <cstdarg>
@@ -890,6 +891,128 @@ void kt_destroy(kt_ctx *c) {
             if (s.done) cudaEventDestroy(s.done);
     for (cudaEvent_t e : c->chunk_events) cudaEventDestroy(e);
     delete c;
+}
+
+}  // extern "C"
+
+// ---------------------------------------------------------------------- online adaptation and sampler
+struct kt_adapt {
+    int K = 0, B = 0, period = 1;
+    double alpha = 1.0, hysteresis = 0.0;
+    int64_t count = 0;
+    std::vector<double> tau;        // smoothed per-sample time of every rank
+    std::vector<int32_t> shares;    // shares in use
+};
+
+extern "C" {
+
+int kt_adapt_create(const int32_t *shares, int K, int global_batch, double alpha, int period, double hysteresis,
+                    kt_adapt **out) {
+    if (!out) return fail(KT_ERR_INVALID, "out is NULL");
+    *out = nullptr;
+    if (K < 1 || K > KT_MAX_RANKS) return fail(KT_ERR_INVALID, "K = %d outside [1, %d]", K, KT_MAX_RANKS);
+    if (int rc = check_shares(shares, K)) return rc;
+    long long sum = 0;
+    for (int r = 0; r < K; ++r) sum += shares[r];
+    if (sum != global_batch) return fail(KT_ERR_INVALID, "shares add up to %lld, global_batch is %d", sum, global_batch);
+    if (!(alpha > 0.0) || !(alpha <= 1.0)) return fail(KT_ERR_INVALID, "alpha must lie in (0, 1]");
+    if (period < 1) return fail(KT_ERR_INVALID, "period must be >= 1");
+    if (!(hysteresis >= 0.0) || !(hysteresis < 1.0)) return fail(KT_ERR_INVALID, "hysteresis must lie in [0, 1)");
+    kt_adapt *a = new (std::nothrow) kt_adapt();
+    if (!a) return fail(KT_ERR_NOMEM, "out of host memory");
+    a->K = K;
+    a->B = global_batch;
+    a->alpha = alpha;
+    a->period = period;
+    a->hysteresis = hysteresis;
+    a->tau.assign(K, 0.0);
+    a->shares.assign(shares, shares + K);
+    *out = a;
+    return KT_OK;
+}
+
+int kt_adapt_observe(kt_adapt *a, const double *step_times, int32_t *shares_out, int *changed) {
+    if (!a || !step_times) return fail(KT_ERR_INVALID, "NULL argument");
+    for (int r = 0; r < a->K; ++r)
+        if (!(step_times[r] > 0.0) || !std::isfinite(step_times[r]))
+            return fail(KT_ERR_INVALID, "step_times[%d] must be finite and > 0", r);
+    const bool fresh = a->count == 0;
+    for (int r = 0; r < a->K; ++r) {
+        const double per_sample = step_times[r] / static_cast<double>(a->shares[r]);
+        a->tau[r] = fresh ? per_sample : (1.0 - a->alpha) * a->tau[r] + a->alpha * per_sample;
+    }
+    a->count += 1;
+    int adopted = 0;
+    if (a->count % a->period == 0) {
+        std::vector<int32_t> next(a->K);
+        if (int rc = kt_schedule(a->tau.data(), a->K, a->B, next.data())) return rc;
+        double cost_now = 0.0, cost_next = 0.0;
+        for (int r = 0; r < a->K; ++r) {
+            cost_now = std::max(cost_now, a->tau[r] * static_cast<double>(a->shares[r]));
+            cost_next = std::max(cost_next, a->tau[r] * static_cast<double>(next[r]));
+        }
+        if (next != a->shares && cost_next < (1.0 - a->hysteresis) * cost_now) {
+            a->shares.swap(next);
+            adopted = 1;
+        }
+    }
+    if (shares_out) std::memcpy(shares_out, a->shares.data(), a->K * sizeof(int32_t));
+    if (changed) *changed = adopted;
+    return KT_OK;
+}
+
+int kt_adapt_state(const kt_adapt *a, double *per_sample_out, int32_t *shares_out, int64_t *count_out) {
+    if (!a) return fail(KT_ERR_INVALID, "state is NULL");
+    if (per_sample_out) std::memcpy(per_sample_out, a->tau.data(), a->K * sizeof(double));
+    if (shares_out) std::memcpy(shares_out, a->shares.data(), a->K * sizeof(int32_t));
+    if (count_out) *count_out = a->count;
+    return KT_OK;
+}
+
+void kt_adapt_destroy(kt_adapt *a) { delete a; }
+
+int64_t kt_sampler_steps(int64_t dataset_size, int64_t global_batch, int drop_last) {
+    if (dataset_size < 1 || global_batch < 1) {
+        fail(KT_ERR_INVALID, "dataset_size and global_batch must be >= 1");
+        return KT_ERR_INVALID;
+    }
+    return drop_last ? dataset_size / global_batch : (dataset_size + global_batch - 1) / global_batch;
+}
+
+int kt_sampler_indices(const int64_t *list, int64_t dataset_size, const int32_t *shares, int K, int drop_last,
+                       int64_t *const *out, void *stream) {
+    if (!out) return fail(KT_ERR_INVALID, "out is NULL");
+    if (K < 1 || K > KT_MAX_RANKS) return fail(KT_ERR_INVALID, "K = %d outside [1, %d]", K, KT_MAX_RANKS);
+    if (int rc = check_shares(shares, K)) return rc;
+    if (dataset_size < 1) return fail(KT_ERR_INVALID, "dataset_size must be >= 1");
+    SamplerParams p{};
+    long long B = 0;
+    for (int r = 0; r < K; ++r) {
+        p.start[r] = static_cast<int>(B);
+        B += shares[r];
+        if (B > 0x7FFFFFFFLL) return fail(KT_ERR_SHAPE, "global batch too large");
+    }
+    p.start[K] = static_cast<int>(B);
+    const int64_t steps = kt_sampler_steps(dataset_size, B, drop_last);
+    if (steps == 0) return KT_OK;
+    for (int r = 0; r < K; ++r) {
+        if (!out[r]) return fail(KT_ERR_INVALID, "out[%d] is NULL", r);
+        if (reinterpret_cast<uintptr_t>(out[r]) % 8) return fail(KT_ERR_ALIGN, "out[%d] is not 8-byte aligned", r);
+        p.out[r] = reinterpret_cast<long long *>(out[r]);
+    }
+    if (reinterpret_cast<uintptr_t>(list) % 8) return fail(KT_ERR_ALIGN, "list is not 8-byte aligned");
+    p.list = reinterpret_cast<const long long *>(list);
+    p.D = dataset_size;
+    p.B = static_cast<int>(B);
+    p.K = K;
+    p.total = steps * B;
+    int dev = 0, sms = 0;
+    KT_CUDA(cudaGetDevice(&dev));
+    KT_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev));
+    const long long blocks = (p.total + NT - 1) / NT, cap = static_cast<long long>(sms) * 8;
+    k_sampler<<<static_cast<int>(blocks < cap ? blocks : cap), NT, 0, static_cast<cudaStream_t>(stream)>>>(p);
+    KT_CUDA(cudaGetLastError());
+    return KT_OK;
 }
 
 }  // extern "C"

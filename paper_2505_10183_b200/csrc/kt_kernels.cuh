@@ -629,6 +629,35 @@ __global__ void __launch_bounds__(NT) k_bcast_recv(const __grid_constant__ Bcast
     }
 }
 
+// ------------------------------------------------------------------ load-adaptive sampler (Section III-C, dynamic data allocation)
+// Position p of the epoch's index list belongs to step s = p / B; inside the step rank r owns
+// the b_r positions from c_r on.  out_r[s * b_r + j] = list[(s * B + c_r + j) mod D].
+struct SamplerParams {
+    const long long *list;              // epoch permutation (device) or NULL for the identity
+    long long D;                        // dataset size
+    long long total;                    // S * B positions
+    int B, K;
+    int start[KT_MAX_RANKS + 1];        // c_r, start[K] = B
+    long long *out[KT_MAX_RANKS];
+};
+
+__global__ void __launch_bounds__(NT) k_sampler(const __grid_constant__ SamplerParams p) {
+    for (long long pos = blockIdx.x * static_cast<long long>(NT) + threadIdx.x; pos < p.total;
+         pos += static_cast<long long>(gridDim.x) * NT) {
+        const long long step = pos / p.B;
+        const int w = static_cast<int>(pos - step * p.B);
+        int lo = 0, hi = p.K;                           // rank with start[r] <= w < start[r + 1]
+        while (hi - lo > 1) {
+            const int mid = (lo + hi) >> 1;
+            if (p.start[mid] <= w) lo = mid; else hi = mid;
+        }
+        const long long src = pos % p.D;
+        const long long v = p.list ? __ldg(p.list + src) : src;
+        const int b = p.start[lo + 1] - p.start[lo];
+        p.out[lo][step * b + (w - p.start[lo])] = v;
+    }
+}
+
 // ------------------------------------------------------------------ standalone casts
 __global__ void __launch_bounds__(NT) k_cast_bf16_to_f32(const unsigned short *in, float *out, long long n) {
     for (long long i = blockIdx.x * static_cast<long long>(NT) + threadIdx.x; i < n;
