@@ -288,6 +288,43 @@ def large_bucket_roofline(kt, peak: float, K: int = 4, bytes_per_rank: int = 256
             "k_direct_sync": row(direct_bytes, direct)}
 
 
+def broadcast_phases(kt, wl, peak: float, chunk_bytes: int) -> dict:
+    """Model synchronisation on the same tensor list: root rank 0's parameters to every rank,
+    inside its group directly, to the other groups through pinned host memory."""
+    dt = torch.float32 if wl.dtype == "f32" else torch.bfloat16
+    params = [[t.cuda() for t in W.split_tensors(W.rank_gradients(wl, r, "cuda"), wl.numel)] for r in range(wl.K)]
+    ctx = kt.kt_groups_init(wl.group_of, [1] * wl.K, wl.G)
+    kt.kt_bucket_pack(ctx, params, wl.bucket_cap_bytes)
+    n = kt.kt_plan_query(ctx).transport_numel
+    send = torch.zeros(n, dtype=dt, device="cuda")
+    pinned = torch.zeros(n, dtype=dt).pin_memory()
+    g_root = wl.group_of[0]
+    recv = [None if g == g_root else torch.zeros(n, dtype=dt, device="cuda") for g in range(wl.G)]
+    main, s1, s2 = torch.cuda.Stream(), torch.cuda.Stream(), torch.cuda.Stream()
+    k_root = sum(1 for g in wl.group_of if g == g_root)
+    es, N = wl.elem_size, wl.N
+    send_bytes = N * es * (1 + 1 + (k_root - 1))
+    recv_bytes = N * es * ((wl.G - 1) + (wl.K - k_root))
+    with torch.cuda.stream(main):
+        t_send = time_launches(lambda: kt.kt_bcast_send(ctx, 0, send, stream=main), main, 20)
+        t_recv = time_launches(lambda: kt.kt_bcast_recv(ctx, 0, recv, stream=main), main, 20)
+
+        def whole():
+            kt.kt_bcast_send(ctx, 0, send, stream=main)
+            kt.kt_bcast_relay(ctx, 0, send, pinned, recv, s1, s2, chunk_bytes=chunk_bytes, main_stream=main)
+            kt.kt_stage_wait(ctx, kt.KT_H2D, main_stream=main)
+            kt.kt_bcast_recv(ctx, 0, recv, stream=main)
+        t_all = time_launches(whole, main, 10)
+    kt.kt_destroy(ctx)
+    return {"what": "broadcast of rank 0's %d tensors (%s) to all %d ranks; %d other group(s) served through "
+                    "pinned host memory" % (wl.T, wl.dtype, wl.K, wl.G - 1),
+            "k_bcast_send": {"us": round(t_send * 1e6, 2), "GBps": round(send_bytes / t_send / 1e9, 1),
+                             "frac": round(send_bytes / t_send / 1e9 / peak, 4), "bytes": send_bytes},
+            "k_bcast_recv": {"us": round(t_recv * 1e6, 2), "GBps": round(recv_bytes / t_recv / 1e9, 1),
+                             "frac": round(recv_bytes / t_recv / 1e9 / peak, 4), "bytes": recv_bytes},
+            "ms_whole": round(t_all * 1e3, 4), "relay_bytes_down": N * es, "relay_bytes_up": N * es * (wl.G - 1)}
+
+
 def max_over_ranks(seconds, dist, device) -> list:
     """Every replica times its own steps; the job is as slow as its slowest replica."""
     if dist is None:
@@ -413,6 +450,7 @@ def run_ours(args) -> dict:
                                       "up on two streams at the same time"}
     if rank == 0 and world == 1 and not args.no_large_bucket:
         result["roofline_large_bucket"] = large_bucket_roofline(kt, peak)
+        result["broadcast"] = broadcast_phases(kt, wl, peak, args_chunk(args))
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         result["cpu_baseline"] = cpu_baseline(wl, prob.shares, budget_s=args.cpu_seconds)
     if dist is not None:

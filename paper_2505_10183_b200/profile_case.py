@@ -3,8 +3,9 @@
     python -m paper_2505_10183_b200.profile_case --K 4 --bytes 67108864 --dtype f32 --launches 3
 
 One flat gradient buffer per rank (ranks 0..K/2-1 in group 0, the rest in group 1), the
-fused intra-group reduce and the combine+unpack kernel launched `launches` times each,
-after one warm-up launch of each.  Prints the CUDA-event time of every launch.
+fused intra-group reduce, the combine+unpack kernel, the one-pass direct kernel and the two
+broadcast kernels launched `launches` times each, after one warm-up launch of each.  Prints
+the CUDA-event time of every launch.
 """
 from __future__ import annotations
 
@@ -37,18 +38,24 @@ def main() -> None:
     transport = kt.kt_ptrs([torch.zeros(n, device="cuda") for _ in range(wl.G)])
     out = kt.kt_ptrs([torch.zeros(m, dtype=dt, device="cuda") for m in wl.numel])
     odt = kt.KT_F32 if wl.dtype == "f32" else kt.KT_BF16
-    times = {"k1_us": [], "k2_us": []}
+    send = torch.zeros(n, dtype=dt, device="cuda")
+    recv = [None if g == wl.group_of[0] else send for g in range(wl.G)]
+    steps = [("k1_us", lambda: kt.kt_hier_reduce(ctx, kt.KT_INTRA, transport)),
+             ("k2_us", lambda: kt.kt_unpack_scale(ctx, transport, out, out_dtype=odt, R=1)),
+             ("direct_us", lambda: kt.kt_sync_direct(ctx, out, out_dtype=odt, R=1)),
+             ("bcast_send_us", lambda: kt.kt_bcast_send(ctx, 0, send)),
+             ("bcast_recv_us", lambda: kt.kt_bcast_recv(ctx, 0, recv))]
+    times = {name: [] for name, _ in steps}
     for i in range(args.launches + 1):
-        ev = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(len(steps) + 1)]
         ev[0].record()
-        kt.kt_hier_reduce(ctx, kt.KT_INTRA, transport)
-        ev[1].record()
-        kt.kt_unpack_scale(ctx, transport, out, out_dtype=odt, R=1)
-        ev[2].record()
+        for j, (_, fn) in enumerate(steps):
+            fn()
+            ev[j + 1].record()
         torch.cuda.synchronize()
         if i:
-            times["k1_us"].append(round(ev[0].elapsed_time(ev[1]) * 1e3, 2))
-            times["k2_us"].append(round(ev[1].elapsed_time(ev[2]) * 1e3, 2))
+            for j, (name, _) in enumerate(steps):
+                times[name].append(round(ev[j].elapsed_time(ev[j + 1]) * 1e3, 2))
     k1_bytes = wl.K * wl.N * wl.elem_size + wl.G * wl.N * 4
     k2_bytes = wl.G * wl.N * 4 + wl.N * wl.elem_size
     print(json.dumps({"case": wl.name, "k1_bytes": k1_bytes, "k2_bytes": k2_bytes, **times}))
