@@ -131,6 +131,7 @@ class Problem:
             starts.append(pos)
             pos += -(-m // 64) * 64
         self.arena_numel = pos
+        self.arena_starts = starts
 
         def views(buf):
             return [buf[s:s + m] for s, m in zip(starts, wl.numel)]
@@ -438,7 +439,8 @@ def run_ours(args) -> dict:
                 "h2d_bytes_per_step": e2e["h2d"], "d2h_bytes_per_step": e2e["d2h"],
                 "ms_per_step": round(e2e["seconds"] / args.steps * 1e3, 4),
                 "layout": "one pinned host buffer and one device buffer per rank, tensors at multiples of "
-                          "64 elements (views): K copies in, 1 copy out, through kt_copy_tensors"},
+                          "64 elements (views); per bucket K copies in and 1 copy out through kt_copy_tensors, "
+                          "buckets pipelined over the two directions of the host link"},
         "gpu_launches": int(launches),
         "clocks": clocks,
     }
@@ -468,44 +470,100 @@ def args_chunk(args) -> int:
     return int(getattr(args, "relay_chunk_mib", 4)) << 20
 
 
+class HostResidentStep:
+    """The end-to-end arm: every rank's gradients start in pinned host memory, the reduced
+    gradients end there.
+
+    Host side: one pinned buffer per rank holding that rank's tensors, each at a multiple of 64
+    elements; device side: the same layout, the per-parameter tensors being views.  A bucket of a
+    rank is then one contiguous range and crosses the host link in one copy (with hundreds of
+    small tensors a copy per tensor would cost more than the bytes).  The step is pipelined
+    bucket by bucket over the two directions of the link: while the gradients of bucket b+1
+    still come up, bucket b is reduced and its partials already go down; the reduced gradients
+    of a bucket go down while the partials of the next come back up."""
+
+    def __init__(self, wl, kt, chunk_bytes: int, device_values: bool = True):
+        self.wl, self.kt = wl, kt
+        prob = self.prob = Problem(wl, kt, device_values=device_values, chunk_bytes=chunk_bytes, arena=True)
+        self.host_in = [a.cpu().pin_memory() for a in prob.grad_arenas]
+        self.host_out = torch.zeros_like(prob.out_arena, device="cpu").pin_memory()
+        for a in prob.grad_arenas:       # whatever reaches the kernels must have crossed the link
+            a.zero_()
+        es = prob.grad_arenas[0].element_size()
+        self.copies_in, self.copies_out, self.h2d_bytes, self.d2h_bytes = [], [], 0, 0
+        for b in range(prob.plan.n_buckets):
+            ts = [t for t in range(wl.T) if prob.plan.bucket_of[t] == b]
+            lo, hi = min(ts), max(ts)
+            off = prob.arena_starts[lo] * es
+            size = (prob.arena_starts[hi] + -(-wl.numel[hi] // 64) * 64) * es - off
+            P = kt.PtrArray.from_addresses
+            self.copies_in.append((P([a.data_ptr() + off for a in prob.grad_arenas], prob.grad_arenas),
+                                   P([h.data_ptr() + off for h in self.host_in], self.host_in), [size] * wl.K))
+            self.copies_out.append((P([self.host_out.data_ptr() + off], self.host_out),
+                                    P([prob.out_arena.data_ptr() + off], prob.out_arena), [size]))
+            self.h2d_bytes += size * wl.K
+            self.d2h_bytes += size
+        self.up = prob.side_h2d if wl.staged else torch.cuda.Stream()
+        self.down = prob.side_d2h if wl.staged else torch.cuda.Stream()
+
+    def step(self):
+        kt, prob, wl = self.kt, self.prob, self.wl
+        main, up, down, ctx = prob.main, self.up, self.down, prob.ctx
+        nb = prob.plan.n_buckets
+        start = torch.cuda.Event()
+        start.record(main)
+        up.wait_event(start)
+        down.wait_event(start)
+        arrived = []
+        for b in range(nb):
+            kt.kt_copy_tensors(*self.copies_in[b], kt.KT_H2D, stream=up)
+            e = torch.cuda.Event()
+            e.record(up)
+            arrived.append(e)
+        for b in range(nb):
+            main.wait_event(arrived[b])
+            kt.kt_hier_reduce(ctx, kt.KT_INTRA, prob.transport, bucket=b, stream=main)
+            if wl.staged:
+                kt.kt_relay_through_host(ctx, prob.transport, prob.pinned, prob.recv, down, up, bucket=b,
+                                         chunk_bytes=prob.chunk_bytes, main_stream=main)
+        for b in range(nb):
+            if wl.staged:
+                kt.kt_stage_wait(ctx, kt.KT_H2D, bucket=b, main_stream=main)
+            kt.kt_unpack_scale(ctx, prob.recv if wl.staged else prob.transport, prob.out_ptrs, scale=1.0, bucket=b,
+                               out_dtype=prob.out_dtype, R=1, stream=main)
+            e = torch.cuda.Event()
+            e.record(main)
+            down.wait_event(e)
+            kt.kt_copy_tensors(*self.copies_out[b], kt.KT_D2H, stream=down)
+        done = torch.cuda.Event()
+        done.record(down)
+        main.wait_event(done)       # the step ends when the reduced gradients are on the host
+
+    def result_tensors(self):
+        """The reduced per-parameter gradients as they arrived in pinned host memory."""
+        return [self.host_out[s:s + m] for s, m in zip(self.prob.arena_starts, self.wl.numel)]
+
+
 def run_e2e(prob, kt, args, barrier) -> dict:
     """Same step, but every step first copies all ranks' gradients from pinned host memory
     to the device and ends with the reduced gradients copied back to pinned host memory."""
-    # Host side: one pinned buffer per rank holding that rank's tensors, each at a multiple of
-    # 64 elements; device side: the same layout, the per-parameter tensors being views.  A rank
-    # then crosses the host link in one copy instead of one per tensor (with hundreds of small
-    # tensors the per-copy cost would otherwise dominate).
-    import ctypes
     wl = prob.wl
     del prob
-    prob = Problem(wl, kt, chunk_bytes=args_chunk(args), arena=True)
-    host_in = [a.cpu().pin_memory() for a in prob.grad_arenas]
-    host_out = [torch.empty_like(prob.out_arena, device="cpu").pin_memory()]
-    dst, src = kt.kt_ptrs(prob.grad_arenas), kt.kt_ptrs(host_in)
-    sizes = [a.numel() * a.element_size() for a in prob.grad_arenas]
-    sizes_c = (ctypes.c_int64 * len(sizes))(*sizes)
-    o_dst, o_src = kt.kt_ptrs(host_out), kt.kt_ptrs([prob.out_arena])
-    o_sizes = [prob.out_arena.numel() * prob.out_arena.element_size()]
-    o_sizes_c = (ctypes.c_int64 * len(o_sizes))(*o_sizes)
-
-    def one():
-        kt.kt_copy_tensors(dst, src, sizes_c, kt.KT_H2D, stream=prob.main)
-        prob.step()
-        kt.kt_copy_tensors(o_dst, o_src, o_sizes_c, kt.KT_D2H, stream=prob.main)
-
+    arm = HostResidentStep(wl, kt, args_chunk(args))
+    main = arm.prob.main
     for _ in range(max(1, min(args.warmup, 3))):
-        one()
+        arm.step()
     barrier()
     a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    a.record(prob.main)
+    a.record(main)
     for _ in range(args.steps):
-        one()
-    b.record(prob.main)
+        arm.step()
+    b.record(main)
     barrier()
-    if not bool(host_out[0].any()):
+    if not bool(arm.host_out.any()):
         raise RuntimeError("end-to-end arm: the result buffer on the host is all zero")
-    kt.kt_destroy(prob.ctx)
-    return {"seconds": a.elapsed_time(b) * 1e-3, "h2d": sum(sizes), "d2h": sum(o_sizes)}
+    kt.kt_destroy(arm.prob.ctx)
+    return {"seconds": a.elapsed_time(b) * 1e-3, "h2d": arm.h2d_bytes, "d2h": arm.d2h_bytes}
 
 
 # ----------------------------------------------------------------------------- the oracle as CPU baseline

@@ -105,6 +105,17 @@ class PtrArray:
             self.array[i] = t.data_ptr() if t.numel() > 0 else (t.data_ptr() or None)
 
 
+    @classmethod
+    def from_addresses(cls, addresses: Sequence[int], keep=None) -> "PtrArray":
+        """A pointer array from raw addresses (e.g. offsets into tensors held elsewhere);
+        `keep` is stored so that whatever owns the memory stays alive with the array."""
+        self = cls([])
+        self.tensors = keep
+        self.n = len(addresses)
+        self.array = (C.c_void_p * max(self.n, 1))(*[int(a) if a else None for a in addresses])
+        return self
+
+
 Ptrs = Union[PtrArray, Sequence[torch.Tensor]]
 
 

@@ -108,6 +108,27 @@ def test_relay_with_group_buffers_as_rows_of_one_allocation(kt, oracle):
     compare_all(kt, oracle, W.tiny(), staged="relay_all", relay_chunk=256, rows=True)
 
 
+@pytest.mark.parametrize("name", ["resnet18", "resnet50", "mobilenet_v2"])
+def test_host_resident_step_as_benchmarked(kt, oracle, name):
+    """The benchmark's end-to-end arm (gradients start in pinned host memory, buckets pipelined
+    over both directions of the host link, results end in pinned host memory), run twice in a
+    row, against the oracle on the same host bytes."""
+    import bench
+    wl = W.by_name(name)
+    arm = bench.HostResidentStep(wl, kt, 4 << 20, device_values=False)
+    shares = arm.prob.shares
+    with torch.cuda.stream(arm.prob.main):
+        arm.step()
+        arm.step()
+    torch.cuda.synchronize()
+    host = [[W.as_numpy(t) for t in W.split_tensors(W.rank_gradients(wl, r, "cpu"), wl.numel)] for r in range(wl.K)]
+    want, _, _, _ = H.run_oracle_path(oracle, wl, host, shares)
+    for t, got in enumerate(arm.result_tensors()):
+        H.assert_bit_equal(got, want[t], "%s out[%d]" % (name, t))
+    assert arm.h2d_bytes >= wl.K * wl.N * wl.elem_size and arm.d2h_bytes >= wl.N * wl.elem_size
+    kt.kt_destroy(arm.prob.ctx)
+
+
 def test_resnet18_staged_bucket_by_bucket(kt, oracle):
     """The per-bucket route: reduce, copy down, copy up and unpack one bucket at a time."""
     wl = W.resnet18()
