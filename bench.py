@@ -116,7 +116,8 @@ class ClockSampler:
 class Problem:
     """Device state of one replica: gradients, context, transport / receive / pinned buffers."""
 
-    def __init__(self, wl, kt, device_values: bool = True, chunk_bytes: int = 4 << 20, arena: bool = False):
+    def __init__(self, wl, kt, device_values: bool = True, chunk_bytes: int = 4 << 20, arena: bool = False,
+                 transport_dtype=torch.float32):
         """arena=False: every gradient and output tensor is its own allocation (as per-parameter
         gradients are).  arena=True: the tensors of one rank are views into one buffer, each at
         a multiple of 64 elements, so that a whole rank moves between host and device in one
@@ -150,12 +151,14 @@ class Problem:
                 self.grads.append([t.cuda() for t in W.split_tensors(flat, wl.numel)])
             del flat
         self.ctx = kt.kt_groups_init(wl.group_of, self.shares, wl.G)
+        if transport_dtype != torch.float32:
+            kt.kt_set_transport_dtype(self.ctx, kt.KT_BF16)
         kt.kt_bucket_pack(self.ctx, self.grads, wl.bucket_cap_bytes)
         self.plan = kt.kt_plan_query(self.ctx)
         n = self.plan.transport_numel
         # the G buffers of a set are rows of one allocation: the relay then moves a chunk of all
         # groups in one copy
-        self.transport = kt.kt_ptrs(list(torch.zeros(wl.G, n, device="cuda")))
+        self.transport = kt.kt_ptrs(list(torch.zeros(wl.G, n, dtype=transport_dtype, device="cuda")))
         if arena:
             self.out_arena = torch.zeros(self.arena_numel, dtype=dt, device="cuda")
             self.out = [views(self.out_arena)]
@@ -165,8 +168,8 @@ class Problem:
         self.out_dtype = kt.KT_F32 if wl.dtype == "f32" else kt.KT_BF16
         self.main = torch.cuda.Stream()
         if wl.staged:
-            self.recv = kt.kt_ptrs(list(torch.zeros(wl.G, n, device="cuda")))
-            self.pinned = kt.kt_ptrs(list(torch.zeros(wl.G, n).pin_memory()))
+            self.recv = kt.kt_ptrs(list(torch.zeros(wl.G, n, dtype=transport_dtype, device="cuda")))
+            self.pinned = kt.kt_ptrs(list(torch.zeros(wl.G, n, dtype=transport_dtype).pin_memory()))
             self.side_d2h = torch.cuda.Stream()
             self.side_h2d = torch.cuda.Stream()
         self.k1_events = []
@@ -326,6 +329,30 @@ def broadcast_phases(kt, wl, peak: float, chunk_bytes: int) -> dict:
             "ms_whole": round(t_all * 1e3, 4), "relay_bytes_down": N * es, "relay_bytes_up": N * es * (wl.G - 1)}
 
 
+def narrow_transport_step(kt, wl, chunk_bytes: int, steps: int) -> dict:
+    """The same step with the library's bf16 transport (an extension: partials rounded once
+    to bf16, half the bytes on the host link).  Reported beside the headline, never as it."""
+    prob = Problem(wl, kt, chunk_bytes=chunk_bytes, transport_dtype=torch.bfloat16)
+    with torch.cuda.stream(prob.main):
+        for _ in range(3):
+            prob.step()
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(prob.main)
+        for _ in range(steps):
+            prob.step(time_k1=True)
+        b.record(prob.main)
+        torch.cuda.synchronize()
+    ms = a.elapsed_time(b) / steps
+    out = {"ms_per_step": round(ms, 4), "k1_us": round(prob.k1_seconds() / steps * 1e6, 2),
+           "k2_us": round(prob.k2_seconds() / steps * 1e6, 2),
+           "staging_bytes_each_way": wl.G * wl.N * 2 if wl.staged else 0,
+           "note": "extension, not the paper's method: fp32 accumulation, partials stored as bf16 "
+                   "(one extra rounding, <= 2^-8 relative)"}
+    kt.kt_destroy(prob.ctx)
+    return out
+
+
 def max_over_ranks(seconds, dist, device) -> list:
     """Every replica times its own steps; the job is as slow as its slowest replica."""
     if dist is None:
@@ -453,6 +480,7 @@ def run_ours(args) -> dict:
     if rank == 0 and world == 1 and not args.no_large_bucket:
         result["roofline_large_bucket"] = large_bucket_roofline(kt, peak)
         result["broadcast"] = broadcast_phases(kt, wl, peak, args_chunk(args))
+        result["bf16_transport"] = narrow_transport_step(kt, wl, args_chunk(args), min(args.steps, 20))
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         result["cpu_baseline"] = cpu_baseline(wl, prob.shares, budget_s=args.cpu_seconds)
     if dist is not None:

@@ -131,6 +131,19 @@ int kt_set_shares(kt_ctx *ctx, const int32_t *shares);
  * the hierarchy (a_r = b_r, W_g = 1) with a final scale of 1/B in kt_unpack_scale. */
 int kt_set_coefficients(kt_ctx *ctx, const float *a, const float *W);
 
+/* Element type of the transport buffers: KT_F32 (the default, and what the method asks
+ * for) or KT_BF16.  The bf16 transport is an extension of this library, not of the paper:
+ * it halves the bytes that cross the host link, which is where Section III-A and Section V
+ * locate the cost, at the price of one extra rounding of every group partial (at most
+ * 2^-8 relative).  With KT_BF16 the fused reduce still accumulates in fp32 and rounds each P_g to
+ * nearest-even when it stores it; the combine widens exactly.  Every `transport`,
+ * `host_pinned`, `send`, `recv` and non-combined `src` argument of the calls below then
+ * addresses bf16 buffers of transport_numel elements (pass them through the float* parameter
+ * by a pointer cast); `combined` stays fp32.  kt_sync_direct keeps its partials in fp32
+ * registers and is therefore bit-identical to the fp32-transport route only.
+ * Takes effect for calls made after it returns.  Errors: KT_ERR_INVALID. */
+int kt_set_transport_dtype(kt_ctx *ctx, int dtype);
+
 /* Read back the weights in use: a_out[K], W_out[G] (host, either may be NULL). */
 int kt_get_coefficients(const kt_ctx *ctx, float *a_out, float *W_out);
 

@@ -308,15 +308,23 @@ def flat_reduce_f64(x, dtype: int, shares):
 
 # --------------------------------------------------------------------------- whole path
 def sync_step(grads, numel, dtype: int, group_of, shares, G: int, bucket_cap_bytes: int,
-              scale: float = 1.0, out_dtype: int | None = None):
+              scale: float = 1.0, out_dtype: int | None = None, transport_dtype: int = F32):
     """The whole path on one thread: plan, intra-group reduce, combine, unpack.
+
+    transport_dtype BF16 (an extension, not the paper's method): every group partial is
+    rounded to bf16 (nearest-even) when it is stored in the transport and widened exactly when
+    the combine reads it; the returned partials are then the uint16 patterns.
 
     Returns (out tensors, transport partials, combined buffer, plan)."""
     out_dtype = dtype if out_dtype is None else out_dtype
     plan = bucket_plan(numel, bucket_cap_bytes)
     a, W, _ = coefficients(group_of, shares, G)
     partials = intra_reduce(grads, plan, dtype, group_of, a, G)
-    S = combine(partials, W)
+    if transport_dtype == BF16:
+        partials = [f32_to_bf16(p) for p in partials]
+        S = combine([bf16_to_f32(p) for p in partials], W)
+    else:
+        S = combine(partials, W)
     out = unpack_scale(S, plan, scale, out_dtype)
     return out, partials, S, plan
 

@@ -25,7 +25,7 @@ KT_MAX_RANKS, KT_MAX_GROUPS = 64, 16
 
 EXPORTS = ["kt_schedule", "kt_adapt_create", "kt_adapt_observe", "kt_adapt_state", "kt_adapt_destroy",
            "kt_sampler_steps", "kt_sampler_indices", "kt_groups_init", "kt_set_shares", "kt_set_coefficients",
-           "kt_get_coefficients", "kt_bucket_pack", "kt_plan_buckets", "kt_plan_query", "kt_hier_reduce",
+           "kt_get_coefficients", "kt_set_transport_dtype", "kt_bucket_pack", "kt_plan_buckets", "kt_plan_query", "kt_hier_reduce",
            "kt_stage_to_host", "kt_relay_through_host", "kt_stage_wait", "kt_unpack_scale", "kt_sync_direct", "kt_bcast_send", "kt_bcast_relay", "kt_bcast_recv", "kt_cast", "kt_copy_tensors", "kt_sync_flat_static", "kt_launch_count",
            "kt_last_error", "kt_destroy"]
 
@@ -59,6 +59,7 @@ def _load() -> C.CDLL:
         "kt_set_shares": ([vp, i32p], C.c_int),
         "kt_set_coefficients": ([vp, f32p, f32p], C.c_int),
         "kt_get_coefficients": ([vp, f32p, f32p], C.c_int),
+        "kt_set_transport_dtype": ([vp, C.c_int], C.c_int),
         "kt_bucket_pack": ([vp, vpp, i64p, C.c_int, C.c_int, C.c_int64, vpp, vp], C.c_int),
         "kt_plan_buckets": ([i64p, C.c_int, C.c_int64, i32p, i64p, i64p, i64p, i32p, i64p], C.c_int),
         "kt_plan_query": ([vp, i32p, i64p, i64p, i64p, i32p, i64p], C.c_int),
@@ -262,6 +263,11 @@ def kt_set_coefficients(ctx: Ctx, a: Sequence[float], W: Sequence[float]) -> Non
     if len(a) != ctx.K or len(W) != ctx.G:
         raise KtError(KT_ERR_SHAPE, "expected %d rank and %d group weights" % (ctx.K, ctx.G))
     _check(_lib.kt_set_coefficients(ctx.handle, (C.c_float * ctx.K)(*a), (C.c_float * ctx.G)(*W)))
+
+
+def kt_set_transport_dtype(ctx: Ctx, dtype: int) -> None:
+    """KT_F32 (default) or KT_BF16: element type of the transport / pinned / receive buffers."""
+    _check(_lib.kt_set_transport_dtype(ctx.handle, int(dtype)))
 
 
 def kt_get_coefficients(ctx: Ctx):

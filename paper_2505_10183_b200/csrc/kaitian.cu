@@ -72,6 +72,7 @@ struct kt_ctx {
     bool planned = false;
     int T = 0;
     int in_dtype = KT_F32;
+    int transport_dtype = KT_F32;                    // element type of the transport buffers
     int tile = TILE_F32;                             // elements per work unit (by gradient dtype)
     std::vector<int64_t> numel, tensor_offset;       // user tensor order
     std::vector<int32_t> bucket_of;
@@ -254,21 +255,32 @@ int launch_k1(kt_ctx *c, const K1Params &p, cudaStream_t s) {
     // one CTA per tile; ranks are streamed in batches of KT_KB whatever K is: small batches keep
     // the register count at 64 and four CTAs resident per SM, which hides the tile look-up of
     // one CTA behind the loads of the others (measured: +12 % on ragged lists with K = 8)
-    k1_intra_reduce<Tin, KT_KB><<<p.tp.n_tiles, NT, 0, s>>>(p);
+    if (c->transport_dtype == KT_F32)
+        k1_intra_reduce<Tin, float, KT_KB><<<p.tp.n_tiles, NT, 0, s>>>(p);
+    else
+        k1_intra_reduce<Tin, unsigned short, KT_KB><<<p.tp.n_tiles, NT, 0, s>>>(p);
     c->launches += 1;
     KT_CUDA(cudaGetLastError());
     return KT_OK;
 }
 
 // combine + unpack: the tile size is the plan's (fixed by the gradient dtype), the vector
-// width follows the output dtype
-template <typename Tout>
-void launch_k2(int tile, int n_tiles, cudaStream_t s, const K2Params &p) {
+// width follows the output dtype, the loads the type of the source buffers
+template <typename Tout, typename TT>
+void launch_k2_typed(int tile, int n_tiles, cudaStream_t s, const K2Params &p) {
     if (tile == TILE_F32)
-        k2_combine_unpack<Tout, TILE_F32><<<n_tiles, NT, 0, s>>>(p);
+        k2_combine_unpack<Tout, TT, TILE_F32><<<n_tiles, NT, 0, s>>>(p);
     else
-        k2_combine_unpack<Tout, TILE_BF16><<<n_tiles, NT, 0, s>>>(p);
+        k2_combine_unpack<Tout, TT, TILE_BF16><<<n_tiles, NT, 0, s>>>(p);
 }
+
+template <typename Tout>
+void launch_k2(int tile, int n_tiles, cudaStream_t s, const K2Params &p, int src_dtype = KT_F32) {
+    if (src_dtype == KT_F32) launch_k2_typed<Tout, float>(tile, n_tiles, s, p);
+    else launch_k2_typed<Tout, unsigned short>(tile, n_tiles, s, p);
+}
+
+size_t transport_elem_size(const kt_ctx *c) { return c->transport_dtype == KT_F32 ? 4 : 2; }
 
 int check_out_args(const kt_ctx *c, void *const *out_grads, int R, int out_dtype) {
     if (!out_grads) return fail(KT_ERR_INVALID, "out_grads is NULL");
@@ -438,6 +450,13 @@ int kt_set_coefficients(kt_ctx *c, const float *a, const float *W) {
     if (!a || !W) return fail(KT_ERR_INVALID, "NULL argument");
     for (int k = 0; k < c->K; ++k) c->rt.coef[k] = a[c->order[k]];
     for (int g = 0; g < c->G; ++g) c->gt.W[g] = W[g];
+    return KT_OK;
+}
+
+int kt_set_transport_dtype(kt_ctx *c, int dtype) {
+    if (int rc = check_ctx(c, false)) return rc;
+    if (dtype != KT_F32 && dtype != KT_BF16) return fail(KT_ERR_INVALID, "unknown transport dtype %d", dtype);
+    c->transport_dtype = dtype;
     return KT_OK;
 }
 
@@ -641,7 +660,10 @@ int kt_hier_reduce(kt_ctx *c, int phase, int bucket, float *const *transport, fl
             p.gt = c->gt;
             for (int g = 0; g < c->G; ++g) p.src[g] = transport[g];
             const long long n4 = n / 4;   // bucket ranges are multiples of 64 elements
-            k_combine_flat<<<grid_for(c, k_combine_flat, 0, (n4 + NT - 1) / NT), NT, 0, s>>>(p, combined, lo, n4);
+            if (c->transport_dtype == KT_F32)
+                k_combine_flat<float><<<grid_for(c, k_combine_flat<float>, 0, (n4 + NT - 1) / NT), NT, 0, s>>>(p, combined, lo, n4);
+            else
+                k_combine_flat<unsigned short><<<grid_for(c, k_combine_flat<unsigned short>, 0, (n4 + NT - 1) / NT), NT, 0, s>>>(p, combined, lo, n4);
             c->launches += 1;
             KT_CUDA(cudaGetLastError());
         }
@@ -670,11 +692,13 @@ int kt_stage_to_host(kt_ctx *c, int dir, int bucket, float *const *transport, fl
         StageSlot &all = c->slots[KT_D2H][0];
         if (bucket >= 0 && all.recorded) KT_CUDA(cudaStreamWaitEvent(ss, all.done, 0));
     }
+    const size_t es = transport_elem_size(c);
     for (int g = 0; g < c->G && n > 0; ++g) {
+        char *dev = reinterpret_cast<char *>(transport[g]) + lo * es, *host = reinterpret_cast<char *>(host_pinned[g]) + lo * es;
         if (dir == KT_D2H)
-            KT_CUDA(cudaMemcpyAsync(host_pinned[g] + lo, transport[g] + lo, n * sizeof(float), cudaMemcpyDeviceToHost, ss));
+            KT_CUDA(cudaMemcpyAsync(host, dev, n * es, cudaMemcpyDeviceToHost, ss));
         else
-            KT_CUDA(cudaMemcpyAsync(transport[g] + lo, host_pinned[g] + lo, n * sizeof(float), cudaMemcpyHostToDevice, ss));
+            KT_CUDA(cudaMemcpyAsync(dev, host, n * es, cudaMemcpyHostToDevice, ss));
     }
     StageSlot &slot = c->slots[dir][bucket + 1];
     KT_CUDA(cudaEventRecord(slot.done, ss));
@@ -699,11 +723,14 @@ int kt_relay_through_host(kt_ctx *c, int bucket, float *const *send, float *cons
     // (rows of one allocation), the relay treats them as one range: one copy per chunk and
     // direction instead of G, which matters because every copy costs the link a few microseconds.
     int groups = c->G;
+    const size_t es = transport_elem_size(c);
+    auto at_elem = [es](float *base, int64_t elem) { return reinterpret_cast<char *>(base) + elem * es; };
     if (bucket < 0) {
         bool rows = true;
         for (int g = 0; g + 1 < c->G; ++g)
-            rows = rows && send[g + 1] == send[g] + n && host_pinned[g + 1] == host_pinned[g] + n &&
-                   recv[g + 1] == recv[g] + n;
+            rows = rows && at_elem(send[g], n) == at_elem(send[g + 1], 0) &&
+                   at_elem(host_pinned[g], n) == at_elem(host_pinned[g + 1], 0) &&
+                   at_elem(recv[g], n) == at_elem(recv[g + 1], 0);
         if (rows) {
             n *= c->G;
             groups = 1;
@@ -711,7 +738,7 @@ int kt_relay_through_host(kt_ctx *c, int bucket, float *const *send, float *cons
     }
     // Uniform chunks (elements, a multiple of 64).  Shorter chunks at the two ends of the
     // pipeline were tried and measured slower: small copies use the host link badly.
-    const int64_t chunk = chunk_bytes / 256 * 64;
+    const int64_t chunk = chunk_bytes / 256 * 256 / static_cast<int64_t>(es);
     std::vector<int64_t> sizes;
     for (int64_t left = n; left > 0; left -= sizes.back()) sizes.push_back(left < chunk ? left : chunk);
     const int64_t n_chunks = static_cast<int64_t>(sizes.size());
@@ -728,13 +755,13 @@ int kt_relay_through_host(kt_ctx *c, int bucket, float *const *send, float *cons
     KT_CUDA(cudaStreamWaitEvent(hs, c->ev_main, 0));
     int64_t at = lo;
     for (int64_t k = 0; k < n_chunks; at += sizes[k], ++k) {
-        const size_t len = static_cast<size_t>(sizes[k]) * sizeof(float);
+        const size_t len = static_cast<size_t>(sizes[k]) * es;
         for (int g = 0; g < groups; ++g)
-            KT_CUDA(cudaMemcpyAsync(host_pinned[g] + at, send[g] + at, len, cudaMemcpyDeviceToHost, ds));
+            KT_CUDA(cudaMemcpyAsync(at_elem(host_pinned[g], at), at_elem(send[g], at), len, cudaMemcpyDeviceToHost, ds));
         KT_CUDA(cudaEventRecord(c->chunk_events[k], ds));
         KT_CUDA(cudaStreamWaitEvent(hs, c->chunk_events[k], 0));
         for (int g = 0; g < groups; ++g)
-            KT_CUDA(cudaMemcpyAsync(recv[g] + at, host_pinned[g] + at, len, cudaMemcpyHostToDevice, hs));
+            KT_CUDA(cudaMemcpyAsync(at_elem(recv[g], at), at_elem(host_pinned[g], at), len, cudaMemcpyHostToDevice, hs));
     }
     StageSlot &down = c->slots[KT_D2H][bucket + 1], &up = c->slots[KT_H2D][bucket + 1];
     KT_CUDA(cudaEventRecord(down.done, ds));
@@ -793,10 +820,11 @@ int kt_unpack_scale(kt_ctx *c, const float *const *src, int from_combined, void 
     p.out_aligned = static_cast<const unsigned char *>(c->d_out) + sz_ptrs;
     p.R = R;
     p.scale = scale;
+    const int src_dtype = from_combined ? KT_F32 : c->transport_dtype;
     if (out_dtype == KT_F32)
-        launch_k2<float>(tp.tile, tp.n_tiles, s, p);
+        launch_k2<float>(tp.tile, tp.n_tiles, s, p, src_dtype);
     else
-        launch_k2<unsigned short>(tp.tile, tp.n_tiles, s, p);
+        launch_k2<unsigned short>(tp.tile, tp.n_tiles, s, p, src_dtype);
     c->launches += 1;
     KT_CUDA(cudaGetLastError());
     return KT_OK;
@@ -1273,8 +1301,8 @@ extern "C" int kt_sync_flat_static(const int32_t *group_of, const int32_t *share
     }
     // the reduce writes every element of the partials it uses, padding included, so nothing
     // left over from an earlier call is ever read
-    if (in_dtype == KT_F32) k1_intra_reduce<float, KT_KB><<<n_tiles, NT, 0, s>>>(p1);
-    else k1_intra_reduce<unsigned short, KT_KB><<<n_tiles, NT, 0, s>>>(p1);
+    if (in_dtype == KT_F32) k1_intra_reduce<float, float, KT_KB><<<n_tiles, NT, 0, s>>>(p1);
+    else k1_intra_reduce<unsigned short, float, KT_KB><<<n_tiles, NT, 0, s>>>(p1);
     KT_CUDA(cudaGetLastError());
     if (out_dtype == KT_F32) launch_k2<float>(tile, n_tiles, s, p2);
     else launch_k2<unsigned short>(tile, n_tiles, s, p2);

@@ -80,14 +80,14 @@ struct TilePlan {         // which tiles a launch covers and how to decode them
 struct K1Params {
     TilePlan tp;
     const void *const *ptrs;           // [K][T] device pointer table
-    float *transport[KT_MAX_GROUPS];
+    void *transport[KT_MAX_GROUPS];    // fp32, or bf16 when the context's transport is narrowed
     RankTab rt;
     int wide;                          // every transport base is 32-byte aligned
 };
 
 struct K2Params {
     TilePlan tp;
-    const float *src[KT_MAX_GROUPS];   // partials (or one combined buffer)
+    const void *src[KT_MAX_GROUPS];    // partials (fp32 or bf16 transport), or one fp32 combined buffer
     GroupTab gt;
     void *const *out_ptrs;             // [R][T] device pointer table
     const unsigned char *out_aligned;  // [T] all R destinations 16-byte aligned
@@ -171,6 +171,48 @@ __device__ __forceinline__ void load_vec(const float *s, float4 (&v)[Q], bool wi
     } else {
 #pragma unroll
         for (int q = 0; q < Q; ++q) v[q] = __ldcs(reinterpret_cast<const float4 *>(s) + q);
+    }
+}
+
+// The same for a transport of type TT (float, or unsigned short = bf16): VEC partial sums are
+// written as they are or narrowed to nearest-even; VEC transport elements are read and widened.
+template <typename TT, int VEC>
+__device__ __forceinline__ void store_transport(void *base, long long at, const float (&a)[VEC], bool wide) {
+    if constexpr (sizeof(TT) == 4) {
+        store_vec<VEC>(static_cast<float *>(base) + at, a, wide);
+    } else {
+        unsigned short *d = static_cast<unsigned short *>(base) + at;
+        if constexpr (VEC == 8)
+            *reinterpret_cast<uint4 *>(d) = make_uint4(pack_bf16x2(a[0], a[1]), pack_bf16x2(a[2], a[3]),
+                                                       pack_bf16x2(a[4], a[5]), pack_bf16x2(a[6], a[7]));
+        else
+            *reinterpret_cast<uint2 *>(d) = make_uint2(pack_bf16x2(a[0], a[1]), pack_bf16x2(a[2], a[3]));
+    }
+}
+
+template <typename TT, int VEC>
+__device__ __forceinline__ void load_transport(const void *base, long long at, float (&x)[VEC], bool wide) {
+    if constexpr (sizeof(TT) == 4) {
+        float4 v[VEC / 4];
+        load_vec<VEC / 4>(static_cast<const float *>(base) + at, v, wide);
+#pragma unroll
+        for (int q = 0; q < VEC / 4; ++q) {
+            x[4 * q] = v[q].x; x[4 * q + 1] = v[q].y; x[4 * q + 2] = v[q].z; x[4 * q + 3] = v[q].w;
+        }
+    } else {
+        const unsigned short *s = static_cast<const unsigned short *>(base) + at;
+        unsigned w[VEC / 2];
+        if constexpr (VEC == 8) {
+            const uint4 v = ld_stream(s);
+            w[0] = v.x; w[1] = v.y; w[2] = v.z; w[3] = v.w;
+        } else {
+            asm volatile("ld.global.nc.L1::no_allocate.v2.u32 {%0,%1}, [%2];" : "=r"(w[0]), "=r"(w[1]) : "l"(s));
+        }
+#pragma unroll
+        for (int q = 0; q < VEC / 2; ++q) {
+            x[2 * q] = __uint_as_float(w[q] << 16);
+            x[2 * q + 1] = __uint_as_float(w[q] & 0xFFFF0000u);
+        }
     }
 }
 
@@ -265,7 +307,7 @@ __device__ __forceinline__ TileRef locate_tile(const TilePlan &tp) {
 
 // ------------------------------------------------------------------ K1: fused pack + widen + weighted intra-group reduce
 // P_g[off_u + e] = sum_{r in g} a_r * f32(x_r^(u)[e]), zero in the padding.
-template <typename Tin, int KB, bool EDGE>
+template <typename Tin, typename TT, int KB, bool EDGE>
 __device__ __forceinline__ void k1_tile(const K1Params &p, const TileRef &t) {
     constexpr int VEC = Elem<Tin>::VEC;
     constexpr int TILE = Elem<Tin>::TILE;
@@ -307,7 +349,7 @@ __device__ __forceinline__ void k1_tile(const K1Params &p, const TileRef &t) {
                         acc[it][c] = first ? __fmul_rn(a, x[c]) : __fmaf_rn(a, x[c], acc[it][c]);
                 }
                 if (p.rt.last[kb + j]) {
-                    float *d = p.transport[p.rt.gid[kb + j]] + t.ti.dst_off;
+                    void *d = p.transport[p.rt.gid[kb + j]];
 #pragma unroll
                     for (int it = 0; it < ITERS; ++it) {
                         if (EDGE) {
@@ -316,7 +358,7 @@ __device__ __forceinline__ void k1_tile(const K1Params &p, const TileRef &t) {
                             for (int c = 0; c < VEC; ++c)   // padding is +0 whatever the weights
                                 if (e[it] + c >= t.ti.numel) acc[it][c] = 0.f;
                         }
-                        store_vec<VEC>(d + e[it], acc[it], p.wide);
+                        store_transport<TT, VEC>(d, t.ti.dst_off + e[it], acc[it], p.wide);
                     }
                 }
             }
@@ -324,22 +366,21 @@ __device__ __forceinline__ void k1_tile(const K1Params &p, const TileRef &t) {
     }
 }
 
-template <typename Tin, int KB>
-__global__ void __launch_bounds__(NT) k1_intra_reduce(const __grid_constant__ K1Params p) {
+template <typename Tin, typename TT, int KB>
+__global__ void __launch_bounds__(NT, 4) k1_intra_reduce(const __grid_constant__ K1Params p) {
     const TileRef t = locate_tile(p.tp);
     if ((t.ti.flags & FLAG_ALIGNED) && t.e0 + Elem<Tin>::TILE <= t.ti.numel)
-        k1_tile<Tin, KB, false>(p, t);
+        k1_tile<Tin, TT, KB, false>(p, t);
     else
-        k1_tile<Tin, KB, true>(p, t);
+        k1_tile<Tin, TT, KB, true>(p, t);
 }
 
 // ------------------------------------------------------------------ K2: inter-group combine + scale + cast + unpack
 // out_c^(u)[e] = cast(scale * sum_g W_g P_g[off_u + e]) for every copy c < R.
-template <typename Tout, int TILE, bool EDGE>
+template <typename Tout, typename TT, int TILE, bool EDGE>
 __device__ __forceinline__ void k2_tile(const K2Params &p, const TileRef &t) {
     constexpr int VEC = Elem<Tout>::VEC;
     constexpr int ITERS = TILE / (NT * VEC);
-    constexpr int Q = VEC / 4;
     const int G = p.gt.G;
     const int T = p.tp.T;
     const bool aligned = p.out_aligned[t.u];
@@ -349,29 +390,23 @@ __device__ __forceinline__ void k2_tile(const K2Params &p, const TileRef &t) {
 
     float acc[ITERS][VEC];
     for (int g = 0; g < G; ++g) {
-        const float *s = p.src[g] + t.ti.dst_off;
         const float w = p.gt.W[g];
-        float4 v[ITERS][Q];
+        float x[ITERS][VEC];
 #pragma unroll
         for (int it = 0; it < ITERS; ++it) {
             // the transport holds ext elements per tensor, so a vector below ext is readable
             if (!EDGE || e[it] < t.ti.ext) {
-                load_vec<Q>(s + e[it], v[it], p.wide);
+                load_transport<TT, VEC>(p.src[g], t.ti.dst_off + e[it], x[it], p.wide);
             } else {
 #pragma unroll
-                for (int q = 0; q < Q; ++q) v[it][q] = make_float4(0.f, 0.f, 0.f, 0.f);
+                for (int c = 0; c < VEC; ++c) x[it][c] = 0.f;
             }
         }
 #pragma unroll
-        for (int it = 0; it < ITERS; ++it) {
+        for (int it = 0; it < ITERS; ++it)
 #pragma unroll
-            for (int q = 0; q < Q; ++q) {
-                const float x[4] = {v[it][q].x, v[it][q].y, v[it][q].z, v[it][q].w};
-#pragma unroll
-                for (int c = 0; c < 4; ++c)
-                    acc[it][4 * q + c] = g == 0 ? __fmul_rn(w, x[c]) : __fmaf_rn(w, x[c], acc[it][4 * q + c]);
-            }
-        }
+            for (int c = 0; c < VEC; ++c)
+                acc[it][c] = g == 0 ? __fmul_rn(w, x[it][c]) : __fmaf_rn(w, x[it][c], acc[it][c]);
     }
 #pragma unroll
     for (int it = 0; it < ITERS; ++it) {
@@ -393,13 +428,13 @@ __device__ __forceinline__ void k2_tile(const K2Params &p, const TileRef &t) {
     }
 }
 
-template <typename Tout, int TILE>
+template <typename Tout, typename TT, int TILE>
 __global__ void __launch_bounds__(NT) k2_combine_unpack(const __grid_constant__ K2Params p) {
     const TileRef t = locate_tile(p.tp);
     if (p.out_aligned[t.u] && t.e0 + TILE <= t.ti.numel)
-        k2_tile<Tout, TILE, false>(p, t);
+        k2_tile<Tout, TT, TILE, false>(p, t);
     else
-        k2_tile<Tout, TILE, true>(p, t);
+        k2_tile<Tout, TT, TILE, true>(p, t);
 }
 
 // ------------------------------------------------------------------ direct path: reduce, combine, scale, cast, unpack in one pass
@@ -504,22 +539,22 @@ __global__ void __launch_bounds__(NT) k_direct_sync(const __grid_constant__ Dire
 }
 
 // ------------------------------------------------------------------ flat inter-group combine into a combined buffer
+template <typename TT>
 __global__ void __launch_bounds__(NT) k_combine_flat(const __grid_constant__ K2Params p, float *combined,
                                                      long long lo, long long n4) {
     const int G = p.gt.G;
     for (long long i = blockIdx.x * static_cast<long long>(NT) + threadIdx.x; i < n4;
          i += static_cast<long long>(gridDim.x) * NT) {
         const long long e = lo + 4 * i;
-        float4 v = *reinterpret_cast<const float4 *>(p.src[0] + e);
-        const float w0 = p.gt.W[0];
-        float4 acc = make_float4(__fmul_rn(w0, v.x), __fmul_rn(w0, v.y), __fmul_rn(w0, v.z), __fmul_rn(w0, v.w));
-        for (int g = 1; g < G; ++g) {
-            v = *reinterpret_cast<const float4 *>(p.src[g] + e);
+        float acc[4];
+        for (int g = 0; g < G; ++g) {
+            float x[4];
+            load_transport<TT, 4>(p.src[g], e, x, false);
             const float w = p.gt.W[g];
-            acc.x = __fmaf_rn(w, v.x, acc.x); acc.y = __fmaf_rn(w, v.y, acc.y);
-            acc.z = __fmaf_rn(w, v.z, acc.z); acc.w = __fmaf_rn(w, v.w, acc.w);
+#pragma unroll
+            for (int c = 0; c < 4; ++c) acc[c] = g == 0 ? __fmul_rn(w, x[c]) : __fmaf_rn(w, x[c], acc[c]);
         }
-        *reinterpret_cast<float4 *>(combined + e) = acc;
+        *reinterpret_cast<float4 *>(combined + e) = make_float4(acc[0], acc[1], acc[2], acc[3]);
     }
 }
 

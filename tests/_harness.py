@@ -40,20 +40,23 @@ def shares_of(wl, kt=None):
 
 
 def run_gpu_path(kt, wl, dev_grads, shares, out_dtype=None, R=1, scale=1.0, per_bucket=False,
-                 use_combined=False, staged=False, relay_chunk=4 << 20, rows=False):
+                 use_combined=False, staged=False, relay_chunk=4 << 20, rows=False, transport_dtype=torch.float32):
     """Returns (out[c][t] tensors, transport list, plan, ctx)."""
     ctx = kt.kt_groups_init(wl.group_of, shares, wl.G)
+    if transport_dtype != torch.float32:
+        kt.kt_set_transport_dtype(ctx, kt.KT_BF16)
     kt.kt_bucket_pack(ctx, dev_grads, wl.bucket_cap_bytes)
     plan = kt.kt_plan_query(ctx)
     n = plan.transport_numel
     # rows=True: the G buffers of each set are rows of one allocation (the relay then moves a
     # chunk of all groups in one copy)
     def buffers(pinned=False):
+        tdt = transport_dtype
         if rows:
-            whole = torch.full((wl.G, n), float("nan"), device=None if pinned else "cuda")
+            whole = torch.full((wl.G, n), float("nan"), dtype=tdt, device=None if pinned else "cuda")
             return list(whole.pin_memory() if pinned else whole)
-        return [torch.full((n,), float("nan")).pin_memory() if pinned else torch.full((n,), float("nan"), device="cuda")
-                for _ in range(wl.G)]
+        return [torch.full((n,), float("nan"), dtype=tdt).pin_memory() if pinned
+                else torch.full((n,), float("nan"), dtype=tdt, device="cuda") for _ in range(wl.G)]
     transport = buffers()
     odt = TORCH_DT[wl.dtype] if out_dtype is None else out_dtype
     out = [[torch.full((m,), float("nan"), dtype=odt, device="cuda") for m in wl.numel] for _ in range(R)]
@@ -97,10 +100,10 @@ def run_gpu_path(kt, wl, dev_grads, shares, out_dtype=None, R=1, scale=1.0, per_
     return out, transport, plan, ctx
 
 
-def run_oracle_path(oracle, wl, host_grads, shares, out_dtype=None, scale=1.0):
+def run_oracle_path(oracle, wl, host_grads, shares, out_dtype=None, scale=1.0, transport_dtype=0):
     odt = ORACLE_DT[wl.dtype] if out_dtype is None else out_dtype
     return oracle.sync_step(host_grads, wl.numel, ORACLE_DT[wl.dtype], wl.group_of, shares, wl.G,
-                            wl.bucket_cap_bytes, scale, odt)
+                            wl.bucket_cap_bytes, scale, odt, transport_dtype)
 
 
 def bits(a: np.ndarray) -> np.ndarray:

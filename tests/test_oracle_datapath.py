@@ -352,3 +352,33 @@ def test_broadcast_hands_every_rank_the_roots_bytes(oracle, dtype):
         for t in range(len(numel)):
             assert out[r][t].dtype == before_root[t].dtype
             assert np.array_equal(out[r][t].view(udt), before_root[t].view(udt)), (r, t)
+
+
+# ----------------------------------------------------------------------------- bf16 transport (extension)
+def test_bf16_transport_rounds_partials_once_and_stays_within_the_bf16_bar(oracle):
+    """Pins for the oracle's bf16-transport reading: (1) where every partial is representable
+    in bf16 the result equals the fp32-transport result bit for bit; (2) otherwise the error
+    against the fp64 mean is bounded by the one extra rounding, 2^-8 of sum_g W_g |P_g| (bf16 keeps
+    8 significant bits, so half a unit in the last place is 2^-8 relative), inside
+    inside 1e-2; (3) the stored partials are the library cast of the fp32 partials."""
+    rng = np.random.default_rng(4)
+    numel = [5, 64, 1000, 4097]
+    group_of, shares = [0, 0, 1, 1], [1, 1, 1, 1]          # a = 1/2, W = 1/2: powers of two
+    # (1) values with few mantissa bits: sums of two, scaled by 1/2, stay bf16-representable
+    coarse = [[(rng.integers(-8, 9, size=n) * 2.0 ** -10).astype(np.float32) for n in numel] for _ in range(4)]
+    a = oracle.sync_step(coarse, numel, F32, group_of, shares, 2, 1 << 20)
+    b = oracle.sync_step(coarse, numel, F32, group_of, shares, 2, 1 << 20, transport_dtype=BF16)
+    for t in range(len(numel)):
+        assert np.array_equal(a[0][t].view(np.uint32), b[0][t].view(np.uint32))
+    # (2), (3) generic values
+    shares = [79, 79, 49, 49]
+    fine = [[(rng.standard_normal(n) * 1e-3).astype(np.float32) for n in numel] for _ in range(4)]
+    out32, parts32, _, _ = oracle.sync_step(fine, numel, F32, group_of, shares, 2, 1 << 20)
+    out16, parts16, _, _ = oracle.sync_step(fine, numel, F32, group_of, shares, 2, 1 << 20, transport_dtype=BF16)
+    for g in range(2):
+        lib = torch.from_numpy(parts32[g]).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
+        assert np.array_equal(parts16[g], lib)
+    F, absF = oracle.flat_reduce_f64([np.concatenate(x) for x in fine], F32, shares)
+    got = np.concatenate(out16)
+    err = np.abs(got - F) / absF
+    assert err.max() <= 2.0 ** -8 + 1e-6 and err.max() > 1e-6      # one bf16 rounding, and it is there
