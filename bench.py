@@ -353,6 +353,28 @@ def narrow_transport_step(kt, wl, chunk_bytes: int, steps: int) -> dict:
     return out
 
 
+def recorded_step(kt, prob, steps: int) -> dict:
+    """The step recorded once and replayed with one submission per step (kt_graph_*): what the
+    sync costs when the host-side cost of the individual calls is out of the way."""
+    main = prob.main
+    torch.cuda.synchronize()
+    kt.kt_graph_begin(prob.ctx, main)
+    prob.step()
+    graph = kt.kt_graph_end(prob.ctx, main)
+    for _ in range(3):
+        kt.kt_graph_launch(graph, main)
+    torch.cuda.synchronize()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record(main)
+    for _ in range(steps):
+        kt.kt_graph_launch(graph, main)
+    b.record(main)
+    torch.cuda.synchronize()
+    out = {"ms_per_step": round(a.elapsed_time(b) / steps, 4), "recorded_operations": kt.kt_graph_nodes(graph)}
+    kt.kt_graph_destroy(graph)
+    return out
+
+
 def max_over_ranks(seconds, dist, device) -> list:
     """Every replica times its own steps; the job is as slow as its slowest replica."""
     if dist is None:
@@ -414,6 +436,7 @@ def run_ours(args) -> dict:
         per_step = [a.elapsed_time(b) for a, b in zip([t_start] + marks[:-1], marks)]
         k1_s = prob.k1_seconds()
         direct_s = time_launches(prob.direct, prob.main, args.steps)
+        recorded = recorded_step(kt, prob, args.steps)
 
         # end to end: gradients start in pinned host memory, the result ends there
         e2e = run_e2e(prob, kt, args, barrier)
@@ -454,6 +477,7 @@ def run_ours(args) -> dict:
                        "direct_us": round(direct_s * 1e6, 2),
                        "direct_note": "kt_sync_direct: the same arithmetic in one pass without transport or "
                                       "relay (what a collective inside one vendor group costs); not part of the step"},
+            "recorded_step": recorded,
             "latency_ms": {"p50": round(statistics.median(per_step), 4),
                            "p95": round(sorted(per_step)[int(0.95 * (len(per_step) - 1))], 4)},
         },

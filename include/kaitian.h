@@ -46,6 +46,7 @@ extern "C" {
 
 typedef struct kt_ctx kt_ctx;
 typedef struct kt_adapt kt_adapt;
+typedef struct kt_graph kt_graph;
 
 typedef enum { KT_F32 = 0, KT_BF16 = 1 } kt_dtype;
 
@@ -334,6 +335,24 @@ int kt_copy_tensors(void *const *dst, const void *const *src, const int64_t *byt
 int kt_sync_flat_static(const int32_t *group_of, const int32_t *shares, int K, int G,
                         const void *const *grads, int in_dtype, int64_t n, void *out, int out_dtype,
                         float scale, void *stream);
+
+/* One submission per step.  A synchronisation step is a fixed sequence of launches, copies
+ * and event waits (the paper's step is one AllReduce call per bucket, Section III); between
+ * kt_graph_begin and kt_graph_end every call of this library made by the calling thread on
+ * `stream` (and on copy streams it pulls in: kt_stage_to_host, kt_relay_through_host) is
+ * recorded instead of executed; kt_graph_launch then replays the whole sequence with one
+ * submission, which removes the per-call host cost that dominates small tensor lists.
+ * Rules while recording: the context must have run the same sequence once before (so that
+ * its device tables are uploaded and its events exist); every copy stream must be waited
+ * for with kt_stage_wait(..., timeout_ms < 0) before kt_graph_end; pointers, sizes, shares
+ * and scale are frozen into the recording (record again after kt_set_shares).
+ * kt_graph_nodes: number of recorded operations.  The graph owns no buffers.
+ * Errors: KT_ERR_STATE, KT_ERR_INVALID, KT_ERR_NOMEM, KT_ERR_CUDA. */
+int kt_graph_begin(kt_ctx *ctx, void *stream);
+int kt_graph_end(kt_ctx *ctx, void *stream, kt_graph **out);
+int kt_graph_launch(kt_graph *graph, void *stream);
+int64_t kt_graph_nodes(const kt_graph *graph);
+void kt_graph_destroy(kt_graph *graph);
 
 /* Number of kernels this context has launched so far (for launch accounting). */
 int64_t kt_launch_count(const kt_ctx *ctx);

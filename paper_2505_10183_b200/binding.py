@@ -24,7 +24,8 @@ KT_ERR_CUDA, KT_ERR_TIMEOUT, KT_ERR_STATE, KT_ERR_NOMEM = -4, -5, -6, -7
 KT_MAX_RANKS, KT_MAX_GROUPS = 64, 16
 
 EXPORTS = ["kt_schedule", "kt_adapt_create", "kt_adapt_observe", "kt_adapt_state", "kt_adapt_destroy",
-           "kt_sampler_steps", "kt_sampler_indices", "kt_groups_init", "kt_set_shares", "kt_set_coefficients",
+           "kt_sampler_steps", "kt_sampler_indices", "kt_graph_begin", "kt_graph_end", "kt_graph_launch",
+           "kt_graph_nodes", "kt_graph_destroy", "kt_groups_init", "kt_set_shares", "kt_set_coefficients",
            "kt_get_coefficients", "kt_set_transport_dtype", "kt_bucket_pack", "kt_plan_buckets", "kt_plan_query", "kt_hier_reduce",
            "kt_stage_to_host", "kt_relay_through_host", "kt_stage_wait", "kt_unpack_scale", "kt_sync_direct", "kt_bcast_send", "kt_bcast_relay", "kt_bcast_recv", "kt_cast", "kt_copy_tensors", "kt_sync_flat_static", "kt_launch_count",
            "kt_last_error", "kt_destroy"]
@@ -55,6 +56,11 @@ def _load() -> C.CDLL:
         "kt_adapt_destroy": ([vp], None),
         "kt_sampler_steps": ([C.c_int64, C.c_int64, C.c_int], C.c_int64),
         "kt_sampler_indices": ([vp, C.c_int64, i32p, C.c_int, C.c_int, vpp, vp], C.c_int),
+        "kt_graph_begin": ([vp, vp], C.c_int),
+        "kt_graph_end": ([vp, vp, vpp], C.c_int),
+        "kt_graph_launch": ([vp, vp], C.c_int),
+        "kt_graph_nodes": ([vp], C.c_int64),
+        "kt_graph_destroy": ([vp], None),
         "kt_groups_init": ([i32p, i32p, C.c_int, C.c_int, vpp], C.c_int),
         "kt_set_shares": ([vp, i32p], C.c_int),
         "kt_set_coefficients": ([vp, f32p, f32p], C.c_int),
@@ -467,6 +473,43 @@ def kt_sync_flat_static(group_of: Sequence[int], shares: Sequence[int], grads: S
     _check(_lib.kt_sync_flat_static(_i32(group_of), _i32(shares), K, int(G), ptrs, _DTYPES[grads[0].dtype],
                                     n, C.c_void_p(out.data_ptr()), _DTYPES[out.dtype], C.c_float(scale),
                                     _stream(stream)))
+
+
+class Graph:
+    """Handle of a recorded step (kt_graph_end)."""
+
+    def __init__(self, handle: int):
+        self.handle = C.c_void_p(handle)
+
+    def __del__(self):
+        try:
+            kt_graph_destroy(self)
+        except Exception:
+            pass
+
+
+def kt_graph_begin(ctx: Ctx, stream=None) -> None:
+    _check(_lib.kt_graph_begin(ctx.handle, _stream(stream)))
+
+
+def kt_graph_end(ctx: Ctx, stream=None) -> Graph:
+    h = C.c_void_p()
+    _check(_lib.kt_graph_end(ctx.handle, _stream(stream), C.byref(h)))
+    return Graph(h.value)
+
+
+def kt_graph_launch(graph: Graph, stream=None) -> None:
+    _check(_lib.kt_graph_launch(graph.handle, _stream(stream)))
+
+
+def kt_graph_nodes(graph: Graph) -> int:
+    return int(_lib.kt_graph_nodes(graph.handle))
+
+
+def kt_graph_destroy(graph: Graph) -> None:
+    if graph.handle is not None and graph.handle.value:
+        _lib.kt_graph_destroy(graph.handle)
+        graph.handle = C.c_void_p(None)
 
 
 def kt_launch_count(ctx: Ctx) -> int:

@@ -923,6 +923,70 @@ void kt_destroy(kt_ctx *c) {
 
 }  // extern "C"
 
+// ---------------------------------------------------------------------- one-submission step (CUDA graph)
+struct kt_graph {
+    cudaGraph_t graph = nullptr;
+    cudaGraphExec_t exec = nullptr;
+    int device = 0;
+    size_t nodes = 0;
+};
+
+extern "C" {
+
+int kt_graph_begin(kt_ctx *c, void *stream) {
+    if (int rc = check_ctx(c, true)) return rc;
+    KT_CUDA(cudaSetDevice(c->device));
+    // thread-local mode: other threads of the process may keep allocating while this one records
+    KT_CUDA(cudaStreamBeginCapture(static_cast<cudaStream_t>(stream), cudaStreamCaptureModeThreadLocal));
+    return KT_OK;
+}
+
+int kt_graph_end(kt_ctx *c, void *stream, kt_graph **out) {
+    if (!out) return fail(KT_ERR_INVALID, "out is NULL");
+    *out = nullptr;
+    if (int rc = check_ctx(c, true)) return rc;
+    cudaGraph_t g = nullptr;
+    cudaError_t e = cudaStreamEndCapture(static_cast<cudaStream_t>(stream), &g);
+    if (e != cudaSuccess) {
+        cudaGetLastError();
+        return fail(KT_ERR_CUDA, "cudaStreamEndCapture: %s (a copy stream that was not waited for, or a call "
+                                 "that cannot be recorded, ends a recording this way)", cudaGetErrorString(e));
+    }
+    kt_graph *h = new (std::nothrow) kt_graph();
+    if (!h) {
+        cudaGraphDestroy(g);
+        return fail(KT_ERR_NOMEM, "out of host memory");
+    }
+    h->graph = g;
+    h->device = c->device;
+    cudaGraphGetNodes(g, nullptr, &h->nodes);
+    e = cudaGraphInstantiate(&h->exec, g, 0);
+    if (e != cudaSuccess) {
+        cudaGraphDestroy(g);
+        delete h;
+        return fail(KT_ERR_CUDA, "cudaGraphInstantiate: %s", cudaGetErrorString(e));
+    }
+    *out = h;
+    return KT_OK;
+}
+
+int kt_graph_launch(kt_graph *g, void *stream) {
+    if (!g || !g->exec) return fail(KT_ERR_INVALID, "graph is NULL");
+    KT_CUDA(cudaGraphLaunch(g->exec, static_cast<cudaStream_t>(stream)));
+    return KT_OK;
+}
+
+int64_t kt_graph_nodes(const kt_graph *g) { return g ? static_cast<int64_t>(g->nodes) : 0; }
+
+void kt_graph_destroy(kt_graph *g) {
+    if (!g) return;
+    if (g->exec) cudaGraphExecDestroy(g->exec);
+    if (g->graph) cudaGraphDestroy(g->graph);
+    delete g;
+}
+
+}  // extern "C"
+
 // ---------------------------------------------------------------------- online adaptation and sampler
 struct kt_adapt {
     int K = 0, B = 0, period = 1;
