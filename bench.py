@@ -391,8 +391,13 @@ def job_throughput(bytes_per_step: int, steps: int, world: int, slowest_seconds:
 
 def run_ours(args) -> dict:
     from paper_2505_10183_b200 import build as kt_build
-    if kt_build.is_stale() and int(os.environ.get("LOCAL_RANK", "0")) == 0:
-        kt_build.build()                     # in-tree, sm_100a; a failed build ends the run
+    if kt_build.is_stale():
+        if int(os.environ.get("LOCAL_RANK", "0")) == 0:
+            kt_build.build()                 # in-tree, sm_100a; a failed build ends the run
+        else:                                # the other ranks wait for rank 0's build
+            deadline = time.time() + 600
+            while kt_build.is_stale() and time.time() < deadline:
+                time.sleep(0.5)
     from paper_2505_10183_b200 import binding as kt
 
     world = int(os.environ.get("WORLD_SIZE", "1"))
