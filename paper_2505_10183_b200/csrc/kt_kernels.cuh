@@ -367,7 +367,7 @@ __device__ __forceinline__ void k1_tile(const K1Params &p, const TileRef &t) {
 }
 
 template <typename Tin, typename TT, int KB>
-__global__ void __launch_bounds__(NT, 4) k1_intra_reduce(const __grid_constant__ K1Params p) {
+__global__ void __launch_bounds__(NT, 1024 / NT) k1_intra_reduce(const __grid_constant__ K1Params p) {
     const TileRef t = locate_tile(p.tp);
     if ((t.ti.flags & FLAG_ALIGNED) && t.e0 + Elem<Tin>::TILE <= t.ti.numel)
         k1_tile<Tin, TT, KB, false>(p, t);
