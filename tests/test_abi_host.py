@@ -108,3 +108,35 @@ def test_missing_library_fails_loudly(tmp_path, monkeypatch):
         sys.modules.pop("paper_2505_10183_b200.binding", None)
         if saved is not None:
             sys.modules["paper_2505_10183_b200.binding"] = saved
+
+
+def test_header_is_plain_c_and_links_against_the_library(tmp_path):
+    """The boundary is a C ABI: the header must compile as C99 on its own, and a C program
+    that calls the pure host entry points must link against the built library and run."""
+    import subprocess
+    from paper_2505_10183_b200 import build
+    src = tmp_path / "abi.c"
+    src.write_text(r'''
+#include "kaitian.h"
+#include <stdio.h>
+int main(void) {
+    double t[4] = {1.0, 1.0, 1.6, 1.6};
+    int32_t b[4];
+    if (kt_schedule(t, 4, 256, b) != KT_OK) return 1;
+    if (b[0] != 79 || b[1] != 79 || b[2] != 49 || b[3] != 49) return 2;
+    int64_t numel[3] = {10, 100, 5}, off[3], total = 0;
+    int32_t nb = 0;
+    if (kt_plan_buckets(numel, 3, 1 << 20, &nb, 0, 0, off, 0, &total) != KT_OK) return 3;
+    if (nb != 1 || off[2] != 0 || off[1] != 8 || off[0] != 112 || total != 128) return 4;
+    if (kt_schedule(t, 4, 2, b) != KT_ERR_INVALID || kt_last_error(0)[0] == 0) return 5;
+    if (kt_sampler_steps(50000, 256, 0) != 196) return 6;
+    printf("ok\n");
+    return 0;
+}
+''')
+    exe = tmp_path / "abi"
+    inc = os.path.join(ROOT, "include")
+    subprocess.check_call(["gcc", "-std=c99", "-Wall", "-Werror", "-pedantic", "-I", inc, "-fsyntax-only", str(src)])
+    subprocess.check_call(["gcc", "-std=c99", "-I", inc, str(src), "-o", str(exe), build.LIB, "-lm", "-ldl", "-lpthread", "-lrt",
+                           "-lstdc++", "-Wl,-rpath," + os.path.dirname(build.LIB)])
+    assert subprocess.check_output([str(exe)]).decode().strip() == "ok"
