@@ -62,6 +62,7 @@ typedef enum {
 } kt_status;
 
 typedef enum { KT_INTRA = 1, KT_INTER = 2, KT_BOTH = 3 } kt_phase;
+typedef enum { KT_ROUTE_DIRECT = 0, KT_ROUTE_RELAY = 1 } kt_route_kind;
 typedef enum { KT_D2H = 0, KT_H2D = 1 } kt_stage_dir;
 
 #define KT_MAX_RANKS 64
@@ -245,6 +246,20 @@ int kt_stage_wait(kt_ctx *ctx, int dir, int bucket, void *main_stream, int timeo
 int kt_unpack_scale(kt_ctx *ctx, const float *const *src, int from_combined,
                     void *const *out_grads, int R, int out_dtype, float scale, int bucket,
                     void *stream);
+
+/* Section III-B, step 1: before a collective runs, look at the participating ranks and
+ * decide whether it stays inside one group of like accelerators or spans several.
+ * group_of[K] (host): group index of every rank, each in [0, G), as in kt_groups_init.
+ * participants[n] (host): distinct rank indices in [0, K), n >= 1.
+ * *route receives KT_ROUTE_DIRECT when all participants belong to one group (step 2: the
+ * collective goes straight to the device-side reduction, kt_sync_direct) and KT_ROUTE_RELAY
+ * when they span groups (step 3: kt_hier_reduce, the relay through host memory,
+ * kt_unpack_scale).  groups_out (host, may be NULL, room for G entries) receives the
+ * ascending list of groups that take part, *n_groups_out (may be NULL) their number.
+ * Pure host function, no context and no device needed.
+ * Errors: KT_ERR_INVALID (NULL, n < 1, rank or group out of range, rank repeated). */
+int kt_route(const int32_t *group_of, int K, int G, const int32_t *participants, int n,
+             int *route, int32_t *groups_out, int *n_groups_out);
 
 /* The direct path: the whole synchronisation in one pass, without transport buffers.
  * Section III-B: a collective whose participants need no host relay (one vendor group, or

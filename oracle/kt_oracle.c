@@ -231,6 +231,30 @@ int kto_sampler_indices(const int64_t *list, int64_t dataset_size, const int32_t
 }
 
 /* ------------------------------------------------------------------------- */
+/* Dispatch decision (Section III-B, steps 1-3): a collective whose              */
+/* participating ranks all sit in one group of like accelerators is homogeneous  */
+/* (returns 0: handled inside the group); one whose participants span groups is  */
+/* heterogeneous (returns 1: needs the relay through host memory).              */
+/* Returns KTO_ERR_INVALID for an empty list, a rank out of range or a repeat.    */
+/* ------------------------------------------------------------------------- */
+int kto_route(const int32_t *group_of, int K, const int32_t *participants, int n)
+{
+    if (!group_of || !participants || K < 1 || n < 1)
+        return KTO_ERR_INVALID;
+    for (int i = 0; i < n; ++i) {
+        if (participants[i] < 0 || participants[i] >= K)
+            return KTO_ERR_INVALID;
+        for (int j = 0; j < i; ++j)
+            if (participants[j] == participants[i])
+                return KTO_ERR_INVALID;
+    }
+    for (int i = 1; i < n; ++i)
+        if (group_of[participants[i]] != group_of[participants[0]])
+            return 1;
+    return 0;
+}
+
+/* ------------------------------------------------------------------------- */
 /* Weights of the two-level mean (Section III-A groups, Section III-C shares).  */
 /* B_g = sum of the shares of group g, B = sum of all shares.                  */
 /* a_r = b_r / B_g  (weight of rank r inside its group),                       */

@@ -54,6 +54,8 @@ def lib() -> C.CDLL:
         L.kto_sampler_steps.restype = C.c_int64
         L.kto_sampler_indices.argtypes = [i64p, C.c_int64, i32p, C.c_int, C.c_int, vpp]
         L.kto_sampler_indices.restype = C.c_int
+        L.kto_route.argtypes = [i32p, C.c_int, i32p, C.c_int]
+        L.kto_route.restype = C.c_int
         L.kto_coefficients.argtypes = [i32p, i32p, C.c_int, C.c_int, f32p, f32p, f32p]
         L.kto_coefficients.restype = C.c_int
         L.kto_bucket_plan.argtypes = [i64p, C.c_int, C.c_int64, i64p, i32p, i64p, i64p, i32p, i64p]
@@ -159,6 +161,16 @@ def sampler_indices(index_list, dataset_size: int, shares, drop_last: bool):
     if rc != 0:
         raise OracleError("kto_sampler_indices: invalid arguments")
     return out
+
+
+def route(group_of, participants) -> int:
+    """0: all participants in one group (homogeneous), 1: they span groups (relay needed)."""
+    g = np.ascontiguousarray(group_of, dtype=np.int32)
+    p = np.ascontiguousarray(participants, dtype=np.int32)
+    rc = lib().kto_route(_p(g, C.c_int32), int(g.size), _p(p, C.c_int32), int(p.size))
+    if rc < 0:
+        raise OracleError("kto_route: invalid arguments")
+    return rc
 
 
 def coefficients(group_of, shares, G: int):

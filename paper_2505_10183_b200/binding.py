@@ -19,6 +19,7 @@ from . import build as _build
 KT_F32, KT_BF16 = 0, 1
 KT_INTRA, KT_INTER, KT_BOTH = 1, 2, 3
 KT_D2H, KT_H2D = 0, 1
+KT_ROUTE_DIRECT, KT_ROUTE_RELAY = 0, 1
 KT_OK, KT_ERR_INVALID, KT_ERR_SHAPE, KT_ERR_ALIGN = 0, -1, -2, -3
 KT_ERR_CUDA, KT_ERR_TIMEOUT, KT_ERR_STATE, KT_ERR_NOMEM = -4, -5, -6, -7
 KT_MAX_RANKS, KT_MAX_GROUPS = 64, 16
@@ -26,7 +27,7 @@ KT_MAX_RANKS, KT_MAX_GROUPS = 64, 16
 EXPORTS = ["kt_schedule", "kt_adapt_create", "kt_adapt_observe", "kt_adapt_state", "kt_adapt_destroy",
            "kt_sampler_steps", "kt_sampler_indices", "kt_graph_begin", "kt_graph_end", "kt_graph_launch",
            "kt_graph_nodes", "kt_graph_destroy", "kt_groups_init", "kt_set_shares", "kt_set_coefficients",
-           "kt_get_coefficients", "kt_set_transport_dtype", "kt_bucket_pack", "kt_plan_buckets", "kt_plan_query", "kt_hier_reduce",
+           "kt_get_coefficients", "kt_set_transport_dtype", "kt_route", "kt_bucket_pack", "kt_plan_buckets", "kt_plan_query", "kt_hier_reduce",
            "kt_stage_to_host", "kt_relay_through_host", "kt_stage_wait", "kt_unpack_scale", "kt_sync_direct", "kt_bcast_send", "kt_bcast_relay", "kt_bcast_recv", "kt_cast", "kt_copy_tensors", "kt_sync_flat_static", "kt_launch_count",
            "kt_last_error", "kt_destroy"]
 
@@ -66,6 +67,7 @@ def _load() -> C.CDLL:
         "kt_set_coefficients": ([vp, f32p, f32p], C.c_int),
         "kt_get_coefficients": ([vp, f32p, f32p], C.c_int),
         "kt_set_transport_dtype": ([vp, C.c_int], C.c_int),
+        "kt_route": ([i32p, C.c_int, C.c_int, i32p, C.c_int, C.POINTER(C.c_int), i32p, C.POINTER(C.c_int)], C.c_int),
         "kt_bucket_pack": ([vp, vpp, i64p, C.c_int, C.c_int, C.c_int64, vpp, vp], C.c_int),
         "kt_plan_buckets": ([i64p, C.c_int, C.c_int64, i32p, i64p, i64p, i64p, i32p, i64p], C.c_int),
         "kt_plan_query": ([vp, i32p, i64p, i64p, i64p, i32p, i64p], C.c_int),
@@ -274,6 +276,17 @@ def kt_set_coefficients(ctx: Ctx, a: Sequence[float], W: Sequence[float]) -> Non
 def kt_set_transport_dtype(ctx: Ctx, dtype: int) -> None:
     """KT_F32 (default) or KT_BF16: element type of the transport / pinned / receive buffers."""
     _check(_lib.kt_set_transport_dtype(ctx.handle, int(dtype)))
+
+
+def kt_route(group_of: Sequence[int], participants: Sequence[int], G: Optional[int] = None):
+    """Returns (KT_ROUTE_DIRECT or KT_ROUTE_RELAY, ascending list of the groups that take part)."""
+    K = len(group_of)
+    G = (max(group_of) + 1 if K else 0) if G is None else G
+    route, ng = C.c_int(-1), C.c_int(0)
+    groups = (C.c_int32 * max(G, 1))()
+    _check(_lib.kt_route(_i32(group_of) if K else None, K, int(G), _i32(participants) if participants else None,
+                         len(participants), C.byref(route), groups, C.byref(ng)))
+    return int(route.value), [int(groups[i]) for i in range(ng.value)]
 
 
 def kt_get_coefficients(ctx: Ctx):

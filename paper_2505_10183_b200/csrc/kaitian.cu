@@ -462,6 +462,33 @@ int kt_set_transport_dtype(kt_ctx *c, int dtype) {
     return KT_OK;
 }
 
+int kt_route(const int32_t *group_of, int K, int G, const int32_t *participants, int n, int *route,
+             int32_t *groups_out, int *n_groups_out) {
+    if (!group_of || !participants || !route) return fail(KT_ERR_INVALID, "NULL argument");
+    if (K < 1 || K > KT_MAX_RANKS) return fail(KT_ERR_INVALID, "K = %d outside [1, %d]", K, KT_MAX_RANKS);
+    if (G < 1 || G > KT_MAX_GROUPS) return fail(KT_ERR_INVALID, "G = %d outside [1, %d]", G, KT_MAX_GROUPS);
+    if (n < 1) return fail(KT_ERR_INVALID, "n = %d must be >= 1", n);
+    for (int r = 0; r < K; ++r)
+        if (group_of[r] < 0 || group_of[r] >= G) return fail(KT_ERR_INVALID, "group_of[%d] = %d outside [0, %d)", r, group_of[r], G);
+    std::vector<char> seen_rank(K, 0), seen_group(G, 0);
+    for (int i = 0; i < n; ++i) {
+        const int r = participants[i];
+        if (r < 0 || r >= K) return fail(KT_ERR_INVALID, "participants[%d] = %d outside [0, %d)", i, r, K);
+        if (seen_rank[r]) return fail(KT_ERR_INVALID, "rank %d is listed twice", r);
+        seen_rank[r] = 1;
+        seen_group[group_of[r]] = 1;
+    }
+    int count = 0;
+    for (int g = 0; g < G; ++g)
+        if (seen_group[g]) {
+            if (groups_out) groups_out[count] = g;
+            ++count;
+        }
+    if (n_groups_out) *n_groups_out = count;
+    *route = count == 1 ? KT_ROUTE_DIRECT : KT_ROUTE_RELAY;
+    return KT_OK;
+}
+
 int kt_get_coefficients(const kt_ctx *c, float *a_out, float *W_out) {
     if (int rc = check_ctx(c, false)) return rc;
     if (a_out)

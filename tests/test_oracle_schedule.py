@@ -193,3 +193,35 @@ def test_weights_of_named_configs(oracle):
 def test_weights_invalid(oracle, group_of, shares, G):
     with pytest.raises(ValueError):
         oracle.coefficients(group_of, shares, G)
+
+
+# ----------------------------------------------------------------------------- dispatch decision (Section III-B)
+def test_route_decision_against_set_arithmetic_and_the_library(oracle):
+    """Pin: Python set arithmetic on the paper's testbed shapes (2 GPUs + 2 MLUs and the other
+    five configurations of Section IV-C) and on random layouts; the library's kt_route must
+    give the same answer and the list of groups involved."""
+    import random
+    from paper_2505_10183_b200 import binding as kt
+    # the paper's configurations: G = GPU group 0, M = MLU group 1
+    for group_of, parts, want in (([0, 0], [0, 1], 0), ([1, 1], [0, 1], 0), ([0, 1], [0, 1], 1),
+                                  ([0, 0, 1], [0, 1, 2], 1), ([0, 1, 1], [1, 2], 0), ([0, 0, 1, 1], [0, 1, 2, 3], 1),
+                                  ([0, 0, 1, 1], [2, 3], 0), ([0, 0, 1, 1], [1], 0)):
+        assert oracle.route(group_of, parts) == want
+    rnd = random.Random(8)
+    for _ in range(300):
+        K = rnd.randint(1, 20)
+        G = rnd.randint(1, min(K, 6))
+        group_of = list(range(G)) + [rnd.randrange(G) for _ in range(K - G)]
+        rnd.shuffle(group_of)
+        parts = rnd.sample(range(K), rnd.randint(1, K))
+        groups = sorted({group_of[r] for r in parts})
+        want = 0 if len(groups) == 1 else 1
+        assert oracle.route(group_of, parts) == want
+        assert kt.kt_route(group_of, parts, G) == (want, groups)
+    for bad in ([], [0, 0], [5], [-1]):
+        with pytest.raises(oracle.OracleError):
+            oracle.route([0, 1, 1], bad)
+    for bad in ([], [0, 0], [5], [-1]):
+        with pytest.raises(kt.KtError) as e:
+            kt.kt_route([0, 1, 1], bad, 2)
+        assert e.value.status == kt.KT_ERR_INVALID
