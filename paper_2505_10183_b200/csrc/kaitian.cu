@@ -83,9 +83,9 @@ struct kt_ctx {
     std::vector<TInfo> info;                         // [T], transport order
 
     // device tables
-    void *d_tables = nullptr;        // one allocation: info | grad ptrs | tile descriptors
+    void *d_tables = nullptr;        // one allocation: prefix | info | grad ptrs
     size_t d_tables_bytes = 0;
-    TileDesc *d_desc = nullptr;      // nullptr when the plan holds a single tensor
+    int *d_prefix = nullptr;
     TInfo *d_info = nullptr;
     const void **d_ptrs = nullptr;
     void *d_out = nullptr;           // out pointer table + aligned flags
@@ -210,7 +210,7 @@ int grid_for(kt_ctx *c, Kern kernel, size_t smem, long long units) {
 int make_tile_plan(const kt_ctx *c, int bucket, TilePlan *tp) {
     if (bucket < -1 || bucket >= static_cast<int>(c->bucket_start.size()))
         return fail(KT_ERR_SHAPE, "bucket %d out of range [-1, %d)", bucket, (int)c->bucket_start.size());
-    tp->desc = c->d_desc;
+    tp->prefix = c->d_prefix;
     tp->info = c->d_info;
     tp->T = c->T;
     tp->u_lo = bucket < 0 ? 0 : c->bucket_u_lo[bucket];
@@ -218,8 +218,6 @@ int make_tile_plan(const kt_ctx *c, int bucket, TilePlan *tp) {
     tp->tile_lo = c->prefix[tp->u_lo];
     tp->n_tiles = c->prefix[tp->u_hi] - tp->tile_lo;
     tp->tile = c->tile;
-    tp->single = tp->u_hi - tp->u_lo == 1;
-    if (tp->single) tp->one = c->info[tp->u_lo];
     tp->tables = c->d_tables;
     tp->table_bytes = static_cast<int>(c->d_tables_bytes < static_cast<size_t>(NT) * 128 ? c->d_tables_bytes
                                                                                           : static_cast<size_t>(NT) * 128);
@@ -553,38 +551,20 @@ int kt_bucket_pack(kt_ctx *c, const void *const *grads, const int64_t *numel, in
         for (int u = 0; u < T; ++u)
             ptrs[static_cast<size_t>(k) * T + u] = grads[static_cast<size_t>(c->order[k]) * T + (T - 1 - u)];
 
-    // ---- tile descriptors: one 16-byte entry per tile so that a CTA finds its work with one load
-    // (a plan of a single tensor needs none: its tiles are decoded by arithmetic)
-    std::vector<TileDesc> desc;
-    if (T > 1) {
-        desc.resize(prefix[T]);
-        for (int u = 0; u < T; ++u) {
-            const TInfo &ti = info[u];
-            const int tiles = prefix[u + 1] - prefix[u];
-            if (tiles > static_cast<int>(DESC_INDEX)) return fail(KT_ERR_SHAPE, "tensor too large for one plan");
-            for (int j = 0; j < tiles; ++j) {
-                unsigned bits = static_cast<unsigned>(j);
-                if ((static_cast<int64_t>(j) + 1) * tile <= ti.numel) bits |= DESC_WHOLE;
-                if (ti.flags & FLAG_ALIGNED) bits |= DESC_ALIGNED;
-                desc[prefix[u] + j] = TileDesc{u, static_cast<int>(bits), ti.dst_off};
-            }
-        }
-    }
-
-    // ---- upload (one allocation, three 256-byte aligned regions: records | pointers | descriptors)
+    // ---- upload (one allocation, three 256-byte aligned regions)
     KT_CUDA(cudaSetDevice(c->device));
+    const size_t sz_prefix = round_up((T + 1) * sizeof(int), 256);
     const size_t sz_info = round_up(T * sizeof(TInfo), 256);
     const size_t sz_ptrs = round_up(ptrs.size() * sizeof(void *), 256);
-    const size_t sz_desc = round_up(desc.size() * sizeof(TileDesc), 256);
     void *d = nullptr;
-    if (cudaMalloc(&d, sz_info + sz_ptrs + sz_desc) != cudaSuccess) {
+    if (cudaMalloc(&d, sz_prefix + sz_info + sz_ptrs) != cudaSuccess) {
         cudaGetLastError();
-        return fail(KT_ERR_NOMEM, "device allocation of %zu bytes failed", sz_info + sz_ptrs + sz_desc);
+        return fail(KT_ERR_NOMEM, "device allocation of %zu bytes failed", sz_prefix + sz_info + sz_ptrs);
     }
-    std::vector<char> staging(sz_info + sz_ptrs + sz_desc, 0);
-    std::memcpy(staging.data(), info.data(), T * sizeof(TInfo));
-    std::memcpy(staging.data() + sz_info, ptrs.data(), ptrs.size() * sizeof(void *));
-    if (!desc.empty()) std::memcpy(staging.data() + sz_info + sz_ptrs, desc.data(), desc.size() * sizeof(TileDesc));
+    std::vector<char> staging(sz_prefix + sz_info + sz_ptrs, 0);
+    std::memcpy(staging.data(), prefix.data(), (T + 1) * sizeof(int));
+    std::memcpy(staging.data() + sz_prefix, info.data(), T * sizeof(TInfo));
+    std::memcpy(staging.data() + sz_prefix + sz_info, ptrs.data(), ptrs.size() * sizeof(void *));
     cudaError_t e = cudaMemcpy(d, staging.data(), staging.size(), cudaMemcpyHostToDevice);
     if (e != cudaSuccess) {
         cudaFree(d);
@@ -592,10 +572,10 @@ int kt_bucket_pack(kt_ctx *c, const void *const *grads, const int64_t *numel, in
     }
     if (c->d_tables) cudaFree(c->d_tables);
     c->d_tables = d;
-    c->d_tables_bytes = sz_info + sz_ptrs + sz_desc;
-    c->d_info = static_cast<TInfo *>(d);
-    c->d_ptrs = reinterpret_cast<const void **>(static_cast<char *>(d) + sz_info);
-    c->d_desc = desc.empty() ? nullptr : reinterpret_cast<TileDesc *>(static_cast<char *>(d) + sz_info + sz_ptrs);
+    c->d_tables_bytes = sz_prefix + sz_info + sz_ptrs;
+    c->d_prefix = static_cast<int *>(d);
+    c->d_info = reinterpret_cast<TInfo *>(static_cast<char *>(d) + sz_prefix);
+    c->d_ptrs = reinterpret_cast<const void **>(static_cast<char *>(d) + sz_prefix + sz_info);
 
     c->T = T;
     c->in_dtype = in_dtype;
@@ -1281,6 +1261,8 @@ namespace {
 constexpr size_t STATIC_TABLE_BYTES = 4096;
 
 struct alignas(256) StaticTables {      // image of the first STATIC_TABLE_BYTES of the scratch
+    int prefix[8];                      // tiles before tensor 0 and 1
+    alignas(32) TInfo info;             // the one tensor
     alignas(8) const void *in_ptrs[KT_MAX_RANKS];
     void *out_ptr[1];
     unsigned char out_aligned[8];
@@ -1355,11 +1337,12 @@ extern "C" int kt_sync_flat_static(const int32_t *group_of, const int32_t *share
     }
     const int tile = in_dtype == KT_F32 ? TILE_F32 : TILE_BF16;
     const int n_tiles = static_cast<int>((stride + tile - 1) / tile);
-    TInfo one{};                        // the one tensor travels in the launch parameters
-    one.dst_off = 0;
-    one.numel = n;
-    one.ext = stride;
-    one.flags = all_aligned ? FLAG_ALIGNED : 0;
+    tab.prefix[0] = 0;
+    tab.prefix[1] = n_tiles;
+    tab.info.dst_off = 0;
+    tab.info.numel = n;
+    tab.info.ext = stride;
+    tab.info.flags = all_aligned ? FLAG_ALIGNED : 0;
     tab.out_ptr[0] = out;
     tab.out_aligned[0] = aligned16(out) ? 1 : 0;
 
@@ -1384,16 +1367,14 @@ extern "C" int kt_sync_flat_static(const int32_t *group_of, const int32_t *share
     KT_CUDA(cudaMemcpyAsync(scratch, &tab, sizeof(tab), cudaMemcpyHostToDevice, s));
 
     TilePlan tp{};
-    tp.desc = nullptr;
-    tp.info = nullptr;
+    tp.prefix = reinterpret_cast<const int *>(scratch + offsetof(StaticTables, prefix));
+    tp.info = reinterpret_cast<const TInfo *>(scratch + offsetof(StaticTables, info));
     tp.T = 1;
     tp.u_lo = 0;
     tp.u_hi = 1;
     tp.tile_lo = 0;
     tp.n_tiles = n_tiles;
     tp.tile = tile;
-    tp.single = 1;
-    tp.one = one;
     tp.tables = scratch;
     tp.table_bytes = static_cast<int>(sizeof(StaticTables));
     float *partials = reinterpret_cast<float *>(scratch + STATIC_TABLE_BYTES);

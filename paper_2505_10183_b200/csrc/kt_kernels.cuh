@@ -5,9 +5,9 @@
 // Work decomposition.  The fp32 transport is cut into tiles of TILE elements that never
 // cross a tensor boundary; one CTA handles one tile (the grid is the tile count, so the
 // hardware scheduler balances ragged tensor lists and partial waves by itself).  A CTA
-// reads its 16-byte tile descriptor (tensor, position, transport offset: one load, no
-// search), then streams the K rank buffers of that tile with 128-bit loads, all loads of a
-// batch of ranks issued before the first multiply.  Interior tiles of 16-byte aligned tensors run without predicates; tiles
+// finds its tensor by binary search in the per-tensor tile prefix, then streams the K rank
+// buffers of that tile with 128-bit loads, all loads of a batch of ranks issued before the
+// first multiply.  Interior tiles of 16-byte aligned tensors run without predicates; tiles
 // that hold a tensor's tail, zero padding, or a misaligned tensor use the same code with
 // per-vector predicates and element loads only where a vector would cross the end.
 //
@@ -65,26 +65,15 @@ struct GroupTab {
     int G;
 };
 
-struct TileDesc {         // one per tile, transport order
-    int u;                // tensor the tile belongs to
-    int j;                // tile index inside the tensor, plus the two flag bits below
-    long long dst_off;    // transport offset of the tensor (copy of its record's field)
-};
-constexpr unsigned DESC_WHOLE = 1u << 31;     // the tile lies wholly inside the tensor (no tail, no padding)
-constexpr unsigned DESC_ALIGNED = 1u << 30;   // all K sources of the tensor are 16-byte aligned
-constexpr unsigned DESC_INDEX = (1u << 30) - 1;
-
 struct TilePlan {         // which tiles a launch covers and how to decode them
-    const TileDesc *desc; // [tiles of the whole plan]; unused when `single`
+    const int *prefix;    // [T+1] tiles before tensor u
     const TInfo *info;    // [T]
     int T;
     int u_lo, u_hi;       // tensors [u_lo, u_hi) take part
-    int tile_lo;          // first tile of tensor u_lo
-    int n_tiles;          // tiles of tensors [u_lo, u_hi)
-    int tile;             // elements per tile the descriptors were built for
-    int single;           // the launch covers exactly one tensor: its record travels in `one`
-    TInfo one;            // ... and tiles are decoded without any table
-    const void *tables;   // start of the table allocation (records, pointers, descriptors) ...
+    int tile_lo;          // prefix[u_lo]
+    int n_tiles;          // prefix[u_hi] - prefix[u_lo]
+    int tile;             // elements per tile the prefix was built for
+    const void *tables;   // start of the table allocation (prefix, records, pointers) ...
     int table_bytes;      // ... and how much of it is worth prefetching (0: nothing)
 };
 
@@ -277,58 +266,42 @@ template <> struct Elem<unsigned short> {
     }
 };
 
-// What a CTA works on: tensor u (transport order), first element of the tile inside it, the
-// tensor's transport offset, and the tensor's record.  The record's loads are issued here but
-// nothing waits for them until a field is used: interior tiles need none of its fields.
+// What a CTA works on: tensor u (transport order), its record, first element of the tile.
 struct TileRef {
     int u;
-    bool whole;           // the tile lies wholly inside the tensor
-    bool src_aligned;     // all K sources of the tensor are 16-byte aligned
-    long long e0;
-    long long dst_off;
     TInfo ti;
+    long long e0;
 };
 
-#ifndef KT_DESC_AHEAD
-#define KT_DESC_AHEAD 1184       /* descriptors are pulled into L2 this many tiles (two waves) ahead */
-#endif
-
-// Tile -> tensor.  One 16-byte load of the tile's descriptor (every thread of the CTA reads
-// the same address), or plain arithmetic when the launch covers a single tensor.  The first
-// CTAs of a launch pull the head of the tables into L2 up front and every CTA pulls a
-// descriptor line two waves ahead, so that look-ups do not wait for DRAM.
+// Tile -> tensor: the u with prefix[u] <= tile < prefix[u + 1] (prefix is non-decreasing, so
+// empty tensors never match).  One memory round trip: thread i tests tensor u_lo + i (in
+// strides of the CTA when there are more tensors than threads), the one that matches
+// publishes it through shared memory.  The first CTAs of a launch also pull the small tables
+// into L2 up front, so that the dependent look-ups that follow (record, pointers) do not
+// each wait for DRAM while the machine is still empty.
 __device__ __forceinline__ TileRef locate_tile(const TilePlan &tp) {
+    __shared__ int s_u;
     const int tile = blockIdx.x + tp.tile_lo;
     if (blockIdx.x < KT_WARM_CTAS) {
         const char *line = static_cast<const char *>(tp.tables) + 128 * threadIdx.x;
         if (128 * threadIdx.x < tp.table_bytes) asm volatile("prefetch.global.L2 [%0];" ::"l"(line));
     }
-    TileRef r;
-    if (tp.single) {
-        r.u = tp.u_lo;
-        r.ti = tp.one;
-        r.e0 = static_cast<long long>(blockIdx.x) * tp.tile;
-        r.dst_off = tp.one.dst_off;
-        r.whole = r.e0 + tp.tile <= tp.one.numel;
-        r.src_aligned = tp.one.flags & FLAG_ALIGNED;
-        return r;
+    for (int u = tp.u_lo + threadIdx.x; u < tp.u_hi; u += NT) {
+        const int a = __ldg(tp.prefix + u), b = __ldg(tp.prefix + u + 1);
+        if (a <= tile && tile < b) s_u = u;
     }
-    if (threadIdx.x == 0 && static_cast<int>(blockIdx.x) + KT_DESC_AHEAD < tp.n_tiles)
-        asm volatile("prefetch.global.L2 [%0];" ::"l"(tp.desc + tile + KT_DESC_AHEAD));
-    const int4 d = __ldg(reinterpret_cast<const int4 *>(tp.desc + tile));
-    r.u = d.x;
-    const unsigned dj = static_cast<unsigned>(d.y);
-    r.whole = dj & DESC_WHOLE;
-    r.src_aligned = dj & DESC_ALIGNED;
-    r.e0 = static_cast<long long>(dj & DESC_INDEX) * tp.tile;
-    r.dst_off = (static_cast<long long>(d.w) << 32) | static_cast<unsigned>(d.z);
-    const int4 *rec = reinterpret_cast<const int4 *>(tp.info + r.u);
+    __syncthreads();
+    const int lo = s_u;
+    TileRef r;
+    r.u = lo;
+    const int4 *rec = reinterpret_cast<const int4 *>(tp.info + lo);
     const int4 a = __ldg(rec), b = __ldg(rec + 1);
-    r.ti.dst_off = r.dst_off;
+    r.ti.dst_off = (static_cast<long long>(a.y) << 32) | static_cast<unsigned>(a.x);
     r.ti.numel = (static_cast<long long>(a.w) << 32) | static_cast<unsigned>(a.z);
     r.ti.ext = (static_cast<long long>(b.y) << 32) | static_cast<unsigned>(b.x);
     r.ti.flags = b.z;
     r.ti.pad_ = 0;
+    r.e0 = static_cast<long long>(tile - __ldg(tp.prefix + lo)) * tp.tile;
     return r;
 }
 
@@ -341,7 +314,7 @@ __device__ __forceinline__ void k1_tile(const K1Params &p, const TileRef &t) {
     constexpr int ITERS = TILE / (NT * VEC);
     const int K = p.rt.K;
     const int T = p.tp.T;
-    const bool aligned = t.src_aligned;
+    const bool aligned = t.ti.flags & FLAG_ALIGNED;
     long long e[ITERS];
 #pragma unroll
     for (int it = 0; it < ITERS; ++it) e[it] = t.e0 + (it * NT + threadIdx.x) * VEC;
@@ -385,7 +358,7 @@ __device__ __forceinline__ void k1_tile(const K1Params &p, const TileRef &t) {
                             for (int c = 0; c < VEC; ++c)   // padding is +0 whatever the weights
                                 if (e[it] + c >= t.ti.numel) acc[it][c] = 0.f;
                         }
-                        store_transport<TT, VEC>(d, t.dst_off + e[it], acc[it], p.wide);
+                        store_transport<TT, VEC>(d, t.ti.dst_off + e[it], acc[it], p.wide);
                     }
                 }
             }
@@ -396,7 +369,7 @@ __device__ __forceinline__ void k1_tile(const K1Params &p, const TileRef &t) {
 template <typename Tin, typename TT, int KB>
 __global__ void __launch_bounds__(NT, 1024 / NT) k1_intra_reduce(const __grid_constant__ K1Params p) {
     const TileRef t = locate_tile(p.tp);
-    if (t.src_aligned && t.whole)
+    if ((t.ti.flags & FLAG_ALIGNED) && t.e0 + Elem<Tin>::TILE <= t.ti.numel)
         k1_tile<Tin, TT, KB, false>(p, t);
     else
         k1_tile<Tin, TT, KB, true>(p, t);
@@ -411,8 +384,6 @@ __device__ __forceinline__ void k2_tile(const K2Params &p, const TileRef &t) {
     const int G = p.gt.G;
     const int T = p.tp.T;
     const bool aligned = p.out_aligned[t.u];
-    // the destination of the first copy is fetched now, beside the partials, not after them
-    Tout *const first_out = static_cast<Tout *>(ldg_ptr(&p.out_ptrs[t.u]));
     long long e[ITERS];
 #pragma unroll
     for (int it = 0; it < ITERS; ++it) e[it] = t.e0 + (it * NT + threadIdx.x) * VEC;
@@ -425,7 +396,7 @@ __device__ __forceinline__ void k2_tile(const K2Params &p, const TileRef &t) {
         for (int it = 0; it < ITERS; ++it) {
             // the transport holds ext elements per tensor, so a vector below ext is readable
             if (!EDGE || e[it] < t.ti.ext) {
-                load_transport<TT, VEC>(p.src[g], t.dst_off + e[it], x[it], p.wide);
+                load_transport<TT, VEC>(p.src[g], t.ti.dst_off + e[it], x[it], p.wide);
             } else {
 #pragma unroll
                 for (int c = 0; c < VEC; ++c) x[it][c] = 0.f;
@@ -444,12 +415,11 @@ __device__ __forceinline__ void k2_tile(const K2Params &p, const TileRef &t) {
         for (int c = 0; c < VEC; ++c) y[c] = __fmul_rn(acc[it][c], p.scale);
         if (!EDGE || (aligned && e[it] + VEC <= t.ti.numel)) {
             const uint4 o = Elem<Tout>::narrow(y);
-            *reinterpret_cast<uint4 *>(first_out + e[it]) = o;
-            for (int c = 1; c < p.R; ++c)
+            for (int c = 0; c < p.R; ++c)
                 *reinterpret_cast<uint4 *>(static_cast<Tout *>(ldg_ptr(&p.out_ptrs[static_cast<size_t>(c) * T + t.u])) + e[it]) = o;
         } else if (e[it] < t.ti.numel) {
             for (int c = 0; c < p.R; ++c) {
-                Tout *d = c == 0 ? first_out : static_cast<Tout *>(ldg_ptr(&p.out_ptrs[static_cast<size_t>(c) * T + t.u]));
+                Tout *d = static_cast<Tout *>(ldg_ptr(&p.out_ptrs[static_cast<size_t>(c) * T + t.u]));
 #pragma unroll
                 for (int k = 0; k < VEC; ++k)
                     if (e[it] + k < t.ti.numel) d[e[it] + k] = Elem<Tout>::narrow_one(y[k]);
@@ -461,7 +431,7 @@ __device__ __forceinline__ void k2_tile(const K2Params &p, const TileRef &t) {
 template <typename Tout, typename TT, int TILE>
 __global__ void __launch_bounds__(NT) k2_combine_unpack(const __grid_constant__ K2Params p) {
     const TileRef t = locate_tile(p.tp);
-    if (p.out_aligned[t.u] && t.whole)
+    if (p.out_aligned[t.u] && t.e0 + TILE <= t.ti.numel)
         k2_tile<Tout, TT, TILE, false>(p, t);
     else
         k2_tile<Tout, TT, TILE, true>(p, t);
@@ -493,7 +463,7 @@ __device__ __forceinline__ void direct_tile(const DirectParams &p, const TileRef
     constexpr int ITERS = TILE / (NT * VEC);
     const int K = p.rt.K;
     const int T = p.tp.T;
-    const bool aligned = t.src_aligned;
+    const bool aligned = t.ti.flags & FLAG_ALIGNED;
     long long e[ITERS];
 #pragma unroll
     for (int it = 0; it < ITERS; ++it) e[it] = t.e0 + (it * NT + threadIdx.x) * VEC;
@@ -562,7 +532,7 @@ __device__ __forceinline__ void direct_tile(const DirectParams &p, const TileRef
 template <typename Tin, typename Tout, int KB>
 __global__ void __launch_bounds__(NT) k_direct_sync(const __grid_constant__ DirectParams p) {
     const TileRef t = locate_tile(p.tp);
-    if (t.src_aligned && t.whole && p.out_aligned[t.u])
+    if ((t.ti.flags & FLAG_ALIGNED) && p.out_aligned[t.u] && t.e0 + Elem<Tin>::TILE <= t.ti.numel)
         direct_tile<Tin, Tout, KB, false>(p, t);
     else
         direct_tile<Tin, Tout, KB, true>(p, t);
@@ -597,8 +567,8 @@ __global__ void __launch_bounds__(NT) k_pack(const __grid_constant__ PackParams 
     const TileRef t = locate_tile(p.tp);
     const int k = blockIdx.y;
     const Tin *s = static_cast<const Tin *>(ldg_ptr(&p.ptrs[static_cast<size_t>(k) * p.tp.T + t.u]));
-    Tin *flat = static_cast<Tin *>(p.flat[k]) + t.dst_off;
-    const bool aligned = t.src_aligned;
+    Tin *flat = static_cast<Tin *>(p.flat[k]) + t.ti.dst_off;
+    const bool aligned = t.ti.flags & FLAG_ALIGNED;
     uint4 raw[ITERS];
 #pragma unroll
     for (int it = 0; it < ITERS; ++it) {
@@ -640,8 +610,8 @@ __global__ void __launch_bounds__(NT) k_bcast_send(const __grid_constant__ Bcast
     const TileRef t = locate_tile(p.tp);
     const int T = p.tp.T;
     const Tv *s = static_cast<const Tv *>(ldg_ptr(&p.ptrs[static_cast<size_t>(p.k_root) * T + t.u]));
-    Tv *flat = static_cast<Tv *>(p.flat[p.g_root]) + t.dst_off;
-    const bool aligned = t.src_aligned;
+    Tv *flat = static_cast<Tv *>(p.flat[p.g_root]) + t.ti.dst_off;
+    const bool aligned = t.ti.flags & FLAG_ALIGNED;
     uint4 raw[ITERS];
     long long e[ITERS];
 #pragma unroll
@@ -672,13 +642,13 @@ __global__ void __launch_bounds__(NT) k_bcast_recv(const __grid_constant__ Bcast
     constexpr int ITERS = Elem<Tv>::TILE / (NT * VEC);
     const TileRef t = locate_tile(p.tp);
     const int T = p.tp.T;
-    const bool aligned = t.src_aligned;
+    const bool aligned = t.ti.flags & FLAG_ALIGNED;
     long long e[ITERS];
 #pragma unroll
     for (int it = 0; it < ITERS; ++it) e[it] = t.e0 + (it * NT + threadIdx.x) * VEC;
     for (int g = 0; g < p.G; ++g) {
         if (g == p.g_root) continue;
-        const Tv *s = static_cast<const Tv *>(p.flat[g]) + t.dst_off;
+        const Tv *s = static_cast<const Tv *>(p.flat[g]) + t.ti.dst_off;
         uint4 raw[ITERS];
 #pragma unroll
         for (int it = 0; it < ITERS; ++it)   // ext is a multiple of 8 elements: a vector below ext is readable
