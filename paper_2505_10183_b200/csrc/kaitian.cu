@@ -218,6 +218,8 @@ int make_tile_plan(const kt_ctx *c, int bucket, TilePlan *tp) {
     tp->tile_lo = c->prefix[tp->u_lo];
     tp->n_tiles = c->prefix[tp->u_hi] - tp->tile_lo;
     tp->tile = c->tile;
+    tp->single = tp->u_hi - tp->u_lo == 1;
+    if (tp->single) tp->one = c->info[tp->u_lo];
     tp->tables = c->d_tables;
     tp->table_bytes = static_cast<int>(c->d_tables_bytes < static_cast<size_t>(NT) * 128 ? c->d_tables_bytes
                                                                                           : static_cast<size_t>(NT) * 128);
@@ -1375,6 +1377,8 @@ extern "C" int kt_sync_flat_static(const int32_t *group_of, const int32_t *share
     tp.tile_lo = 0;
     tp.n_tiles = n_tiles;
     tp.tile = tile;
+    tp.single = 1;
+    tp.one = tab.info;
     tp.tables = scratch;
     tp.table_bytes = static_cast<int>(sizeof(StaticTables));
     float *partials = reinterpret_cast<float *>(scratch + STATIC_TABLE_BYTES);
