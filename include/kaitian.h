@@ -29,7 +29,12 @@
  *    throws across the boundary.  kt_last_error() returns a message for the last failing
  *    call made by the calling thread.
  *  - Kernel launches and copies are asynchronous with respect to the given stream.
- *    kt_schedule, kt_groups_init, kt_set_shares, kt_plan_query are pure host functions.
+ *    kt_schedule, kt_route, kt_adapt_*, kt_sampler_steps, kt_plan_buckets, kt_set_shares,
+ *    kt_set_coefficients and kt_plan_query are pure host functions; the first five need no
+ *    CUDA device at all.
+ *  - A kt_ctx (and a kt_adapt, a kt_graph) is not safe for concurrent use from several host
+ *    threads; different objects may be used from different threads.  kt_last_error() is per
+ *    thread.
  *  - Arithmetic is IEEE fp32 with a fixed order (ascending rank inside a group, ascending
  *    group): the first term of a sum is one rounded product, every later term one fused
  *    multiply-add.  bf16 gradients are widened exactly; bf16 outputs are rounded to
