@@ -29,9 +29,9 @@
  *    throws across the boundary.  kt_last_error() returns a message for the last failing
  *    call made by the calling thread.
  *  - Kernel launches and copies are asynchronous with respect to the given stream.
- *    kt_schedule, kt_route, kt_adapt_*, kt_sampler_steps, kt_plan_buckets, kt_set_shares,
- *    kt_set_coefficients and kt_plan_query are pure host functions; the first five need no
- *    CUDA device at all.
+ *    kt_scores, kt_schedule, kt_route, kt_adapt_*, kt_sampler_steps, kt_plan_buckets,
+ *    kt_set_shares, kt_set_coefficients and kt_plan_query are pure host functions; the first
+ *    six need no CUDA device at all.
  *  - A kt_ctx (and a kt_adapt, a kt_graph) is not safe for concurrent use from several host
  *    threads; different objects may be used from different threads.  kt_last_error() is per
  *    thread.
@@ -82,6 +82,12 @@ typedef enum { KT_D2H = 0, KT_H2D = 1 } kt_stage_dir;
  * then the higher rank).  Requires 1 <= K <= KT_MAX_RANKS and global_batch >= K.
  * Errors: KT_ERR_INVALID. */
 int kt_schedule(const double *step_times, int K, int global_batch, int32_t *shares_out);
+
+/* Section III-C, "Initial Benchmarking": the fastest device scores 1.0, every other device
+ * score_i = time_fastest / time_i.  step_times[K] (host): finite and > 0; scores_out[K] (host).
+ * This is the first half of kt_schedule, exposed for callers that share or log the scores
+ * (the paper publishes them to all ranks before training).  Errors: KT_ERR_INVALID. */
+int kt_scores(const double *step_times, int K, double *scores_out);
 
 /* Online adaptation of the scores (Section III-C, "Online Adaptation": monitor computation
  * times per batch during training and adjust the scores; the paper leaves the rule open).

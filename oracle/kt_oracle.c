@@ -39,6 +39,23 @@
 /* A rank never gets zero samples: a zero share is raised to one, taken from    */
 /* the currently largest share (tie: the slowest of them, then higher index).   */
 /* ------------------------------------------------------------------------- */
+/* The scores alone: score_i = time_fastest / time_i (Section III-C). */
+int kto_scores(const double *step_times, int K, double *scores)
+{
+    if (!step_times || !scores || K < 1)
+        return KTO_ERR_INVALID;
+    for (int i = 0; i < K; ++i)
+        if (!(step_times[i] > 0.0) || !isfinite(step_times[i]))
+            return KTO_ERR_INVALID;
+    double t_min = step_times[0];
+    for (int i = 1; i < K; ++i)
+        if (step_times[i] < t_min)
+            t_min = step_times[i];
+    for (int i = 0; i < K; ++i)
+        scores[i] = t_min / step_times[i];
+    return KTO_OK;
+}
+
 int kto_schedule(const double *step_times, int K, int global_batch, int32_t *shares)
 {
     if (!step_times || !shares || K < 1 || global_batch < K)

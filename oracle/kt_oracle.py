@@ -45,6 +45,8 @@ def lib() -> C.CDLL:
         i32p, i64p, f32p, f64p = (C.POINTER(C.c_int32), C.POINTER(C.c_int64),
                                   C.POINTER(C.c_float), C.POINTER(C.c_double))
         vpp = C.POINTER(C.c_void_p)
+        L.kto_scores.argtypes = [f64p, C.c_int, f64p]
+        L.kto_scores.restype = C.c_int
         L.kto_schedule.argtypes = [f64p, C.c_int, C.c_int, i32p]
         L.kto_schedule.restype = C.c_int
         L.kto_adapt_observe.argtypes = [f64p, i32p, i64p, C.c_int, C.c_int, C.c_double, C.c_int,
@@ -107,6 +109,14 @@ def _check_dtype(arrays, dtype):
 
 
 # --------------------------------------------------------------------------- schedule
+def scores(step_times) -> np.ndarray:
+    t = np.ascontiguousarray(step_times, dtype=np.float64)
+    out = np.zeros(t.size, dtype=np.float64)
+    if lib().kto_scores(_p(t, C.c_double), int(t.size), _p(out, C.c_double)) != 0:
+        raise OracleError("kto_scores: invalid arguments")
+    return out
+
+
 def schedule(step_times, global_batch: int) -> np.ndarray:
     t = np.ascontiguousarray(step_times, dtype=np.float64)
     out = np.zeros(t.size, dtype=np.int32)

@@ -24,7 +24,7 @@ KT_OK, KT_ERR_INVALID, KT_ERR_SHAPE, KT_ERR_ALIGN = 0, -1, -2, -3
 KT_ERR_CUDA, KT_ERR_TIMEOUT, KT_ERR_STATE, KT_ERR_NOMEM = -4, -5, -6, -7
 KT_MAX_RANKS, KT_MAX_GROUPS = 64, 16
 
-EXPORTS = ["kt_schedule", "kt_adapt_create", "kt_adapt_observe", "kt_adapt_state", "kt_adapt_destroy",
+EXPORTS = ["kt_schedule", "kt_scores", "kt_adapt_create", "kt_adapt_observe", "kt_adapt_state", "kt_adapt_destroy",
            "kt_sampler_steps", "kt_sampler_indices", "kt_graph_begin", "kt_graph_end", "kt_graph_launch",
            "kt_graph_nodes", "kt_graph_destroy", "kt_groups_init", "kt_set_shares", "kt_set_coefficients",
            "kt_get_coefficients", "kt_set_transport_dtype", "kt_route", "kt_bucket_pack", "kt_plan_buckets", "kt_plan_query", "kt_hier_reduce",
@@ -51,6 +51,7 @@ def _load() -> C.CDLL:
     vpp = C.POINTER(C.c_void_p)
     sigs = {
         "kt_schedule": ([C.POINTER(C.c_double), C.c_int, C.c_int, i32p], C.c_int),
+        "kt_scores": ([C.POINTER(C.c_double), C.c_int, C.POINTER(C.c_double)], C.c_int),
         "kt_adapt_create": ([i32p, C.c_int, C.c_int, C.c_double, C.c_int, C.c_double, vpp], C.c_int),
         "kt_adapt_observe": ([vp, C.POINTER(C.c_double), i32p, C.POINTER(C.c_int)], C.c_int),
         "kt_adapt_state": ([vp, C.POINTER(C.c_double), i32p, i64p], C.c_int),
@@ -249,6 +250,14 @@ def kt_sampler_indices(index_list: Optional[torch.Tensor], dataset_size: int, sh
     _check(_lib.kt_sampler_indices(C.c_void_p(index_list.data_ptr()) if index_list is not None else None,
                                    int(dataset_size), _i32(shares), K, int(bool(drop_last)), pa.array,
                                    _stream(stream)))
+
+
+def kt_scores(step_times: Sequence[float]) -> List[float]:
+    K = len(step_times)
+    t = (C.c_double * max(K, 1))(*[float(x) for x in step_times])
+    out = (C.c_double * max(K, 1))()
+    _check(_lib.kt_scores(t, K, out))
+    return [float(out[i]) for i in range(K)]
 
 
 def kt_groups_init(group_of: Sequence[int], shares: Sequence[int], G: Optional[int] = None) -> Ctx:

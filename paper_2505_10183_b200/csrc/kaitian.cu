@@ -407,6 +407,19 @@ int kt_schedule(const double *step_times, int K, int global_batch, int32_t *shar
     return KT_OK;
 }
 
+int kt_scores(const double *step_times, int K, double *scores_out) {
+    if (!step_times || !scores_out) return fail(KT_ERR_INVALID, "NULL argument");
+    if (K < 1 || K > KT_MAX_RANKS) return fail(KT_ERR_INVALID, "K = %d outside [1, %d]", K, KT_MAX_RANKS);
+    double fastest = INFINITY;
+    for (int i = 0; i < K; ++i) {
+        if (!(step_times[i] > 0.0) || !std::isfinite(step_times[i]))
+            return fail(KT_ERR_INVALID, "step_times[%d] must be finite and > 0", i);
+        fastest = std::min(fastest, step_times[i]);
+    }
+    for (int i = 0; i < K; ++i) scores_out[i] = fastest / step_times[i];
+    return KT_OK;
+}
+
 int kt_groups_init(const int32_t *group_of, const int32_t *shares, int K, int G, kt_ctx **out) {
     if (!out) return fail(KT_ERR_INVALID, "out is NULL");
     *out = nullptr;

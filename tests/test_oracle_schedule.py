@@ -50,6 +50,24 @@ def test_paper_example_scores_and_shares(oracle):
     assert [round(x) for x in q] == [151, 105]
     got = oracle.schedule([float(t) for t in times], B)
     assert got.tolist() == [151, 105]
+    # the score function on its own, oracle and library: the printed 1.0 and 0.7
+    from paper_2505_10183_b200 import binding as kt
+    for fn in (lambda t: oracle.scores(t).tolist(), kt.kt_scores):
+        sc = fn([float(t) for t in times])
+        assert sc[0] == 1.0 and abs(sc[1] - 0.7) < 1e-15
+    import random
+    rnd = random.Random(2)
+    for _ in range(300):
+        ts = [rnd.uniform(0.01, 50.0) for _ in range(rnd.randint(1, 64))]
+        want = [Fraction(min(ts)) / Fraction(t) for t in ts]          # exact quotient of the doubles
+        got_o, got_l = oracle.scores(ts).tolist(), kt.kt_scores(ts)
+        assert got_o == got_l == [float(w) for w in want]             # one correctly rounded division
+        assert max(got_o) == 1.0
+    for bad in ([], [1.0, 0.0], [float("nan")], [float("inf"), 1.0]):
+        with pytest.raises(oracle.OracleError):
+            oracle.scores(bad)
+        with pytest.raises(kt.KtError):
+            kt.kt_scores(bad)
 
 
 @pytest.mark.parametrize("times,B,expect", [
