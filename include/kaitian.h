@@ -287,6 +287,19 @@ int kt_route(const int32_t *group_of, int K, int G, const int32_t *participants,
 int kt_sync_direct(kt_ctx *ctx, void *const *out_grads, int R, int out_dtype, float scale,
                    int bucket, void *stream);
 
+/* One AllReduce of the registered gradients in one call: Section III-B, steps 1-3, as the
+ * meta process group performs them for every collective.  With one group the call is
+ * kt_sync_direct.  With several groups it queues, on main_stream and the two copy streams,
+ * kt_hier_reduce(KT_INTRA) over all buckets, kt_relay_through_host of the whole transport,
+ * the wait for the way up, and kt_unpack_scale from the receive buffers.
+ * transport, host_pinned, recv: as in kt_relay_through_host (ignored, may be NULL, with one
+ * group); out_grads, R, out_dtype, scale: as in kt_unpack_scale; chunk_bytes >= 256.
+ * Asynchronous like its parts; results are bit-identical to calling the parts.
+ * Errors: those of the parts. */
+int kt_allreduce(kt_ctx *ctx, float *const *transport, float *const *host_pinned, float *const *recv,
+                 void *const *out_grads, int R, int out_dtype, float scale, int64_t chunk_bytes,
+                 void *main_stream, void *d2h_stream, void *h2d_stream);
+
 /* Hierarchical Broadcast (model synchronisation).  The paper routes Broadcast through the
  * same hierarchy as AllReduce (Section III, "broadcast for model synchronization"; Section
  * III-A: inside a group directly, between groups through host RAM in the three copy steps).

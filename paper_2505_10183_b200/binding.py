@@ -28,7 +28,7 @@ EXPORTS = ["kt_schedule", "kt_scores", "kt_adapt_create", "kt_adapt_observe", "k
            "kt_sampler_steps", "kt_sampler_indices", "kt_graph_begin", "kt_graph_end", "kt_graph_launch",
            "kt_graph_nodes", "kt_graph_destroy", "kt_groups_init", "kt_set_shares", "kt_set_coefficients",
            "kt_get_coefficients", "kt_set_transport_dtype", "kt_route", "kt_bucket_pack", "kt_plan_buckets", "kt_plan_query", "kt_hier_reduce",
-           "kt_stage_to_host", "kt_relay_through_host", "kt_stage_wait", "kt_unpack_scale", "kt_sync_direct", "kt_bcast_send", "kt_bcast_relay", "kt_bcast_recv", "kt_cast", "kt_copy_tensors", "kt_sync_flat_static", "kt_launch_count",
+           "kt_stage_to_host", "kt_relay_through_host", "kt_stage_wait", "kt_unpack_scale", "kt_sync_direct", "kt_allreduce", "kt_bcast_send", "kt_bcast_relay", "kt_bcast_recv", "kt_cast", "kt_copy_tensors", "kt_sync_flat_static", "kt_launch_count",
            "kt_last_error", "kt_destroy"]
 
 _DTYPES = {torch.float32: KT_F32, torch.bfloat16: KT_BF16}
@@ -78,6 +78,7 @@ def _load() -> C.CDLL:
         "kt_stage_wait": ([vp, C.c_int, C.c_int, vp, C.c_int], C.c_int),
         "kt_unpack_scale": ([vp, vpp, C.c_int, vpp, C.c_int, C.c_int, C.c_float, C.c_int, vp], C.c_int),
         "kt_sync_direct": ([vp, vpp, C.c_int, C.c_int, C.c_float, C.c_int, vp], C.c_int),
+        "kt_allreduce": ([vp, vpp, vpp, vpp, vpp, C.c_int, C.c_int, C.c_float, C.c_int64, vp, vp, vp], C.c_int),
         "kt_bcast_send": ([vp, C.c_int, C.c_int, vp, vp], C.c_int),
         "kt_bcast_relay": ([vp, C.c_int, C.c_int, vp, vp, vpp, C.c_int64, vp, vp, vp], C.c_int),
         "kt_bcast_recv": ([vp, C.c_int, C.c_int, vpp, vp], C.c_int),
@@ -432,6 +433,27 @@ def kt_sync_direct(ctx: Ctx, out_grads: Union[PtrArray, Sequence[Sequence[torch.
     _check(_lib.kt_sync_direct(ctx.handle, op.array, R, out_dtype, C.c_float(scale), int(bucket),
                                _stream(stream)))
     ctx._keep["out"] = op
+
+
+def kt_allreduce(ctx: Ctx, out_grads, transport: Optional[Ptrs] = None, host_pinned: Optional[Ptrs] = None,
+                 recv: Optional[Ptrs] = None, d2h_stream=None, h2d_stream=None, scale: float = 1.0,
+                 chunk_bytes: int = 4 << 20, out_dtype: Optional[int] = None, R: Optional[int] = None,
+                 main_stream=None) -> None:
+    """One AllReduce of the registered gradients: the direct route with one group, else reduce,
+    relay through pinned host memory, combine + unpack.  The three buffer lists and the two copy
+    streams are needed only with more than one group."""
+    op, R, out_dtype = _out_args(ctx, out_grads, out_dtype, R)
+    lists = [kt_ptrs(x) if x is not None else None for x in (transport, host_pinned, recv)]
+    if ctx.G > 1 and (any(x is None or x.n != ctx.G for x in lists) or d2h_stream is None or h2d_stream is None):
+        raise KtError(KT_ERR_SHAPE, "with %d groups, %d transport, pinned and receive buffers and two copy streams "
+                                    "are required" % (ctx.G, ctx.G))
+    arrs = [x.array if x is not None else None for x in lists]
+    _check(_lib.kt_allreduce(ctx.handle, arrs[0], arrs[1], arrs[2], op.array, R, out_dtype, C.c_float(scale),
+                             int(chunk_bytes), _stream(main_stream),
+                             _stream(d2h_stream) if d2h_stream is not None else None,
+                             _stream(h2d_stream) if h2d_stream is not None else None))
+    ctx._keep["out"] = op
+    ctx._keep["allreduce"] = lists
 
 
 def _recv_array(ctx: Ctx, recv: Sequence[Optional[torch.Tensor]]) -> C.Array:

@@ -902,6 +902,20 @@ int kt_sync_direct(kt_ctx *c, void *const *out_grads, int R, int out_dtype, floa
     return KT_OK;
 }
 
+int kt_allreduce(kt_ctx *c, float *const *transport, float *const *host_pinned, float *const *recv,
+                 void *const *out_grads, int R, int out_dtype, float scale, int64_t chunk_bytes, void *main_stream,
+                 void *d2h_stream, void *h2d_stream) {
+    if (int rc = check_ctx(c, true)) return rc;
+    if (c->G == 1) return kt_sync_direct(c, out_grads, R, out_dtype, scale, -1, main_stream);
+    if (int rc = check_out_args(c, out_grads, R, out_dtype)) return rc;      // fail before anything is queued
+    if (int rc = kt_hier_reduce(c, KT_INTRA, -1, transport, nullptr, main_stream)) return rc;
+    if (int rc = kt_relay_through_host(c, -1, transport, host_pinned, recv, chunk_bytes, main_stream, d2h_stream,
+                                       h2d_stream))
+        return rc;
+    if (int rc = kt_stage_wait(c, KT_H2D, -1, main_stream, -1)) return rc;
+    return kt_unpack_scale(c, recv, 0, out_grads, R, out_dtype, scale, -1, main_stream);
+}
+
 int kt_cast(const void *in, int in_dtype, void *out, int out_dtype, int64_t n, void *stream) {
     if (n < 0) return fail(KT_ERR_INVALID, "n is negative");
     if (n == 0) return KT_OK;

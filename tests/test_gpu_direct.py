@@ -143,3 +143,37 @@ def test_error_codes(kt):
         kt.kt_sync_direct(ctx, kt.kt_ptrs(out[0]), R=wl.K + 1, out_dtype=kt.KT_F32)
     assert e.value.status == kt.KT_ERR_SHAPE
     kt.kt_destroy(ctx)
+
+
+def test_allreduce_in_one_call_takes_the_route_the_groups_call_for(kt, oracle):
+    """kt_allreduce: one group -> the direct kernel (1 launch, no buffers); several groups ->
+    reduce, relay through pinned host memory, combine + unpack (2 launches); both equal the
+    oracle bit for bit, twice in a row."""
+    for wl in (W.Workload("one_group", 9, W.tiny().shapes, "f32", [0, 0, 0], [3, 2, 1]), W.tiny(), W.mobilenet_v2(),
+               W.resnet18()):
+        shares = H.shares_of(wl, kt)
+        host, dev = H.device_gradients(wl)
+        ctx = kt.kt_groups_init(wl.group_of, shares, wl.G)
+        kt.kt_bucket_pack(ctx, dev, wl.bucket_cap_bytes)
+        n = kt.kt_plan_query(ctx).transport_numel
+        out = [[torch.full((m,), float("nan"), dtype=H.TORCH_DT[wl.dtype], device="cuda") for m in wl.numel]]
+        kw = {}
+        if wl.G > 1:
+            kw = dict(transport=list(torch.full((wl.G, n), float("nan"), device="cuda")),
+                      host_pinned=list(torch.zeros(wl.G, n).pin_memory()),
+                      recv=list(torch.full((wl.G, n), float("nan"), device="cuda")),
+                      d2h_stream=torch.cuda.Stream(), h2d_stream=torch.cuda.Stream())
+        before = kt.kt_launch_count(ctx)
+        kt.kt_allreduce(ctx, out, scale=0.5, **kw)
+        kt.kt_allreduce(ctx, out, scale=0.5, **kw)
+        torch.cuda.synchronize()
+        assert kt.kt_launch_count(ctx) - before == (2 if wl.G == 1 else 4)
+        want, parts, _, _ = H.run_oracle_path(oracle, wl, host, shares, scale=0.5)
+        for t in range(wl.T):
+            H.assert_bit_equal(out[0][t], want[t], "%s out[%d]" % (wl.name, t))
+        if wl.G > 1:
+            for g in range(wl.G):
+                H.assert_bit_equal(kw["recv"][g], parts[g], "recv[%d]" % g)
+            with pytest.raises(kt.KtError):
+                kt.kt_allreduce(ctx, out)             # buffers are required with several groups
+        kt.kt_destroy(ctx)
