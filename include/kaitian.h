@@ -32,6 +32,9 @@
  *    kt_scores, kt_schedule, kt_route, kt_adapt_*, kt_sampler_steps, kt_plan_buckets,
  *    kt_set_shares, kt_set_coefficients and kt_plan_query are pure host functions; the first
  *    six need no CUDA device at all.
+ *  - A context is bound to the CUDA device that was current in kt_groups_init.  Calls on it
+ *    make that device current for their own duration and leave the calling thread's current
+ *    device as they found it.
  *  - A kt_ctx (and a kt_adapt, a kt_graph) is not safe for concurrent use from several host
  *    threads; different objects may be used from different threads.  kt_last_error() is per
  *    thread.

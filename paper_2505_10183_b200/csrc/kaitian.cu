@@ -51,6 +51,28 @@ int fail(int code, const char *fmt, ...) {
             return fail(KT_ERR_CUDA, "%s: %s", #call, cudaGetErrorString(e_));              \
     } while (0)
 
+// Makes a context's device current for the length of a call and puts the caller's device back
+// afterwards: a library call must not change which device the calling thread works on.
+struct DeviceScope {
+    int prev = -1;
+    cudaError_t status = cudaSuccess;
+    explicit DeviceScope(int device) {
+        status = cudaGetDevice(&prev);
+        if (status == cudaSuccess && prev != device) status = cudaSetDevice(device);
+        else if (status == cudaSuccess) prev = -1;          // nothing to restore
+    }
+    ~DeviceScope() {
+        if (prev >= 0) cudaSetDevice(prev);
+    }
+    DeviceScope(const DeviceScope &) = delete;
+    DeviceScope &operator=(const DeviceScope &) = delete;
+};
+
+#define KT_ON_DEVICE(dev)                                                                   \
+    DeviceScope device_scope_(dev);                                                         \
+    if (device_scope_.status != cudaSuccess)                                                \
+        return fail(KT_ERR_CUDA, "selecting device %d: %s", (dev), cudaGetErrorString(device_scope_.status))
+
 // ------------------------------------------------------------------ host-side state
 struct StageSlot {
     cudaEvent_t done = nullptr;
@@ -567,7 +589,7 @@ int kt_bucket_pack(kt_ctx *c, const void *const *grads, const int64_t *numel, in
             ptrs[static_cast<size_t>(k) * T + u] = grads[static_cast<size_t>(c->order[k]) * T + (T - 1 - u)];
 
     // ---- upload (one allocation, three 256-byte aligned regions)
-    KT_CUDA(cudaSetDevice(c->device));
+    KT_ON_DEVICE(c->device);
     const size_t sz_prefix = round_up((T + 1) * sizeof(int), 256);
     const size_t sz_info = round_up(T * sizeof(TInfo), 256);
     const size_t sz_ptrs = round_up(ptrs.size() * sizeof(void *), 256);
@@ -681,7 +703,7 @@ int kt_hier_reduce(kt_ctx *c, int phase, int bucket, float *const *transport, fl
     }
     TilePlan tp{};
     if (int rc = make_tile_plan(c, bucket, &tp)) return rc;
-    KT_CUDA(cudaSetDevice(c->device));
+    KT_ON_DEVICE(c->device);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
 
     if ((phase & KT_INTRA) && tp.n_tiles > 0) {
@@ -724,7 +746,7 @@ int kt_stage_to_host(kt_ctx *c, int dir, int bucket, float *const *transport, fl
         if (!transport[g] || !host_pinned[g]) return fail(KT_ERR_INVALID, "buffer %d is NULL", g);
     int64_t lo, n;
     bucket_range(c, bucket, &lo, &n);
-    KT_CUDA(cudaSetDevice(c->device));
+    KT_ON_DEVICE(c->device);
     cudaStream_t ms = static_cast<cudaStream_t>(main_stream), ss = static_cast<cudaStream_t>(side_stream);
     KT_CUDA(cudaEventRecord(c->ev_main, ms));
     KT_CUDA(cudaStreamWaitEvent(ss, c->ev_main, 0));
@@ -784,7 +806,7 @@ int kt_relay_through_host(kt_ctx *c, int bucket, float *const *send, float *cons
     std::vector<int64_t> sizes;
     for (int64_t left = n; left > 0; left -= sizes.back()) sizes.push_back(left < chunk ? left : chunk);
     const int64_t n_chunks = static_cast<int64_t>(sizes.size());
-    KT_CUDA(cudaSetDevice(c->device));
+    KT_ON_DEVICE(c->device);
     while (static_cast<int64_t>(c->chunk_events.size()) < n_chunks) {
         cudaEvent_t e;
         KT_CUDA(cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
@@ -841,7 +863,7 @@ int kt_unpack_scale(kt_ctx *c, const float *const *src, int from_combined, void 
     if (int rc = check_buffers(c, src, nsrc, "src")) return rc;
     TilePlan tp{};
     if (int rc = make_tile_plan(c, bucket, &tp)) return rc;
-    KT_CUDA(cudaSetDevice(c->device));
+    KT_ON_DEVICE(c->device);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     size_t sz_ptrs = 0;
     if (int rc = upload_out_table(c, out_grads, R, out_dtype, s, &sz_ptrs)) return rc;
@@ -877,7 +899,7 @@ int kt_sync_direct(kt_ctx *c, void *const *out_grads, int R, int out_dtype, floa
     if (int rc = check_out_args(c, out_grads, R, out_dtype)) return rc;
     TilePlan tp{};
     if (int rc = make_tile_plan(c, bucket, &tp)) return rc;
-    KT_CUDA(cudaSetDevice(c->device));
+    KT_ON_DEVICE(c->device);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     size_t sz_ptrs = 0;
     if (int rc = upload_out_table(c, out_grads, R, out_dtype, s, &sz_ptrs)) return rc;
@@ -965,7 +987,7 @@ const char *kt_last_error(const kt_ctx *) { return g_err; }
 
 void kt_destroy(kt_ctx *c) {
     if (!c) return;
-    cudaSetDevice(c->device);
+    DeviceScope device_scope_(c->device);
     if (c->d_tables || c->d_out) cudaDeviceSynchronize();
     if (c->d_tables) cudaFree(c->d_tables);
     if (c->d_out) cudaFree(c->d_out);
@@ -991,7 +1013,7 @@ extern "C" {
 
 int kt_graph_begin(kt_ctx *c, void *stream) {
     if (int rc = check_ctx(c, true)) return rc;
-    KT_CUDA(cudaSetDevice(c->device));
+    KT_ON_DEVICE(c->device);
     // thread-local mode: other threads of the process may keep allocating while this one records
     KT_CUDA(cudaStreamBeginCapture(static_cast<cudaStream_t>(stream), cudaStreamCaptureModeThreadLocal));
     return KT_OK;
@@ -1196,7 +1218,7 @@ int kt_bcast_send(kt_ctx *c, int root, int bucket, void *send, void *stream) {
     if (int rc = make_tile_plan(c, bucket, &p.tp)) return rc;
     if (p.tp.n_tiles == 0) return KT_OK;
     p.flat[p.g_root] = send;
-    KT_CUDA(cudaSetDevice(c->device));
+    KT_ON_DEVICE(c->device);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     if (c->in_dtype == KT_F32) k_bcast_send<float><<<p.tp.n_tiles, NT, 0, s>>>(p);
     else k_bcast_send<unsigned short><<<p.tp.n_tiles, NT, 0, s>>>(p);
@@ -1218,7 +1240,7 @@ int kt_bcast_recv(kt_ctx *c, int root, int bucket, void *const *recv, void *stre
     }
     if (int rc = make_tile_plan(c, bucket, &p.tp)) return rc;
     if (p.tp.n_tiles == 0 || c->G == 1) return KT_OK;
-    KT_CUDA(cudaSetDevice(c->device));
+    KT_ON_DEVICE(c->device);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     if (c->in_dtype == KT_F32) k_bcast_recv<float><<<p.tp.n_tiles, NT, 0, s>>>(p);
     else k_bcast_recv<unsigned short><<<p.tp.n_tiles, NT, 0, s>>>(p);
@@ -1246,7 +1268,7 @@ int kt_bcast_relay(kt_ctx *c, int root, int bucket, const void *send, void *host
     std::vector<int64_t> sizes;
     for (int64_t left = n; left > 0; left -= sizes.back()) sizes.push_back(left < chunk ? left : chunk);
     const int64_t n_chunks = static_cast<int64_t>(sizes.size());
-    KT_CUDA(cudaSetDevice(c->device));
+    KT_ON_DEVICE(c->device);
     while (static_cast<int64_t>(c->chunk_events.size()) < n_chunks) {
         cudaEvent_t e;
         KT_CUDA(cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
