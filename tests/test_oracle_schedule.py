@@ -81,7 +81,7 @@ def test_closed_forms(oracle, times, B, expect):
     assert oracle.schedule(times, B).tolist() == expect
 
 
-def test_survey_configs_against_exact_rationals(oracle):
+def test_named_configs_against_exact_rationals(oracle):
     for times, B in (([1, 1, Fraction(8, 5), Fraction(8, 5)], 256),
                      ([1] * 4 + [Fraction(7, 5)] * 2 + [Fraction(21, 10)] * 2, 256),
                      ([1] * 4 + [Fraction(7, 5)] * 2 + [Fraction(21, 10)] * 2, 512)):
