@@ -372,6 +372,82 @@ int kto_bucket_plan(const int64_t *numel, int T, int64_t bucket_cap_bytes,
 }
 
 /* ------------------------------------------------------------------------- */
+/* One rank per device: which part of a bucket each member of a group reduces.  */
+/* The paper hands the intra-group collective to the vendor library (Section    */
+/* III-A, first bullet) and says nothing of how the work is split among the     */
+/* devices of a group.  Reading taken: the range of a collective (one bucket,   */
+/* or the whole transport when bucket < 0) is cut into work units of `unit`     */
+/* elements that never cross a tensor: tensor t, which occupies the transport   */
+/* from its offset up to the next tensor's offset (padding included), holds     */
+/* ceil(extent / unit) of them, the last one possibly short.  The units of the  */
+/* range are numbered in transport order; with U units and M members, member m  */
+/* owns units floor(m U / M) ... floor((m+1) U / M) - 1, a contiguous element    */
+/* range [lo_out[m], lo_out[m] + n_out[m]).  A member that owns no unit gets      */
+/* n_out = 0 (lo_out then marks where its empty range sits).                     */
+/* ------------------------------------------------------------------------- */
+int kto_shard_ranges(const int64_t *numel, int T, int64_t bucket_cap_bytes, int64_t unit,
+                     int bucket, int n_members, int64_t *lo_out, int64_t *n_out)
+{
+    if (!numel || T < 1 || unit < 1 || n_members < 1 || !lo_out || !n_out)
+        return KTO_ERR_INVALID;
+    int64_t *offset = (int64_t *)malloc(sizeof(int64_t) * (size_t)T);
+    int32_t *bucket_of = (int32_t *)malloc(sizeof(int32_t) * (size_t)T);
+    int64_t *bstart = (int64_t *)malloc(sizeof(int64_t) * (size_t)T);
+    int64_t *bnumel = (int64_t *)malloc(sizeof(int64_t) * (size_t)T);
+    int32_t nb = 0;
+    int64_t total = 0;
+    int rc = kto_bucket_plan(numel, T, bucket_cap_bytes, offset, bucket_of, bstart, bnumel, &nb, &total);
+    if (rc == KTO_OK && (bucket < -1 || bucket >= nb))
+        rc = KTO_ERR_INVALID;
+    if (rc != KTO_OK) {
+        free(offset); free(bucket_of); free(bstart); free(bnumel);
+        return rc;
+    }
+    const int64_t range_hi = bucket < 0 ? total : bstart[bucket] + bnumel[bucket];
+
+    /* pass 1 counts the units of the range, pass 2 hands them out */
+    int64_t U = 0;
+    for (int pass = 0; pass < 2; ++pass) {
+        int64_t index = 0;
+        if (pass == 1) {
+            for (int m = 0; m < n_members; ++m) {
+                n_out[m] = 0;
+                /* an empty share sits where its first unit would be */
+                lo_out[m] = range_hi;
+            }
+        }
+        for (int t = T - 1; t >= 0; --t) {              /* transport order */
+            if (bucket >= 0 && bucket_of[t] != bucket)
+                continue;
+            const int64_t end = t > 0 ? offset[t - 1] : total;   /* the next tensor in the transport is t-1 */
+            const int64_t extent = end - offset[t];
+            for (int64_t at = 0; at < extent; at += unit, ++index) {
+                if (pass == 0)
+                    continue;
+                const int64_t len = extent - at < unit ? extent - at : unit;
+                for (int m = 0; m < n_members; ++m) {
+                    const int64_t first = (int64_t)m * U / n_members;
+                    const int64_t past = (int64_t)(m + 1) * U / n_members;
+                    if (index >= first && index < past) {
+                        if (n_out[m] == 0)
+                            lo_out[m] = offset[t] + at;
+                        n_out[m] += len;
+                    }
+                }
+            }
+        }
+        if (pass == 0)
+            U = index;
+    }
+    /* empty shares: place them at the start of the next member's range */
+    for (int m = n_members - 1; m >= 0; --m)
+        if (n_out[m] == 0)
+            lo_out[m] = m + 1 < n_members ? lo_out[m + 1] : range_hi;
+    free(offset); free(bucket_of); free(bstart); free(bnumel);
+    return KTO_OK;
+}
+
+/* ------------------------------------------------------------------------- */
 /* Casts.  bf16 is the upper half of an IEEE-754 binary32 pattern.             */
 /* Widening is exact.  Narrowing rounds to nearest, ties to even, on the bit    */
 /* pattern; a NaN keeps its sign and upper payload and is made quiet.           */

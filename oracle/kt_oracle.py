@@ -62,6 +62,8 @@ def lib() -> C.CDLL:
         L.kto_coefficients.restype = C.c_int
         L.kto_bucket_plan.argtypes = [i64p, C.c_int, C.c_int64, i64p, i32p, i64p, i64p, i32p, i64p]
         L.kto_bucket_plan.restype = C.c_int
+        L.kto_shard_ranges.argtypes = [i64p, C.c_int, C.c_int64, C.c_int64, C.c_int, C.c_int, i64p, i64p]
+        L.kto_shard_ranges.restype = C.c_int
         L.kto_bf16_to_f32.argtypes = [C.c_void_p, C.c_void_p, C.c_int64]
         L.kto_bf16_to_f32.restype = None
         L.kto_f32_to_bf16.argtypes = [C.c_void_p, C.c_void_p, C.c_int64]
@@ -230,6 +232,20 @@ def bucket_plan(numel, bucket_cap_bytes: int) -> Plan:
     return Plan(n, off, bof, bstart[: nb.value].copy(), bnumel[: nb.value].copy(), total.value)
 
 
+def shard_ranges(numel, bucket_cap_bytes: int, unit: int, bucket: int, n_members: int):
+    """One rank per device: the element range of the transport that each of the n_members
+    devices of a group reduces, for one bucket (or the whole transport, bucket = -1).
+    Returns a list of (lo, n), one per member."""
+    n = np.ascontiguousarray(numel, dtype=np.int64)
+    lo = np.zeros(max(n_members, 1), np.int64)
+    cnt = np.zeros(max(n_members, 1), np.int64)
+    rc = lib().kto_shard_ranges(_p(n, C.c_int64), n.size, int(bucket_cap_bytes), int(unit), int(bucket),
+                                int(n_members), _p(lo, C.c_int64), _p(cnt, C.c_int64))
+    if rc != 0:
+        raise OracleError("kto_shard_ranges: invalid arguments")
+    return [(int(a), int(b)) for a, b in zip(lo[:n_members], cnt[:n_members])]
+
+
 # --------------------------------------------------------------------------- casts
 def bf16_to_f32(x: np.ndarray) -> np.ndarray:
     x = np.ascontiguousarray(x, dtype=np.uint16)
@@ -373,3 +389,50 @@ def sync_step_flat_threads(x, dtype: int, group_of, shares, G: int, scale: float
     with ThreadPoolExecutor(max_workers=threads) as ex:
         list(ex.map(work, bounds))
     return out
+
+
+def sharded_sync_step(grads, numel, dtype: int, group_of, shares, G: int, bucket_cap_bytes: int, unit: int,
+                      scale: float = 1.0, out_dtype: int | None = None, per_bucket: bool = False):
+    """The whole path with one rank per device, in the order the devices work (Section III-A:
+    collective inside the group, device -> host, exchange between groups in host memory, host ->
+    device), every device doing only its own share of each range (shard_ranges):
+
+      1. member m of group g forms the group partial over ITS element range from the tensors
+         of all members of g (ascending rank) and stores that range in host memory;
+      2. once every range of every group is there, it reads ITS range of every group's
+         partial, combines them (ascending group), scales, casts, and writes that range into
+         the tensors of every member of its group.
+
+    Returns (out[r][t] for every rank r, the G partials as they stand in host memory, plan).
+    Per element the operations are those of sync_step, so every rank must end up with
+    sync_step's result."""
+    out_dtype = dtype if out_dtype is None else out_dtype
+    K = len(grads)
+    plan = bucket_plan(numel, bucket_cap_bytes)
+    a, W, _ = coefficients(group_of, shares, G)
+    members = [[r for r in range(K) if group_of[r] == g] for g in range(G)]
+    flat = [pack(grads[r], plan, dtype) for r in range(K)]            # a rank's tensors at the plan's offsets
+    host = [np.full(plan.transport_numel, np.nan, np.float32) for _ in range(G)]
+    S = [np.full(plan.transport_numel, np.nan, np.float32) for _ in range(G)]   # what group g's members combined
+    ranges = [-1] if not per_bucket else list(range(plan.n_buckets))
+    for b in ranges:
+        for g in range(G):                                            # step 1, every device of every group
+            mine = shard_ranges(numel, bucket_cap_bytes, unit, b, len(members[g]))
+            for m, (lo, n) in enumerate(mine):
+                if n == 0:
+                    continue
+                sub = bucket_plan([n], 1 << 62)
+                part = intra_reduce([[flat[r][lo:lo + n]] for r in members[g]], sub, dtype, [0] * len(members[g]),
+                                    [a[r] for r in members[g]], 1)[0]
+                host[g][lo:lo + n] = part[:n]
+        for g in range(G):                                            # step 2, after the exchange
+            mine = shard_ranges(numel, bucket_cap_bytes, unit, b, len(members[g]))
+            for m, (lo, n) in enumerate(mine):
+                if n:
+                    S[g][lo:lo + n] = combine([np.ascontiguousarray(host[h][lo:lo + n]) for h in range(G)], W)
+    out = [None] * K
+    for g in range(G):
+        tensors = unpack_scale(S[g], plan, scale, out_dtype)
+        for r in members[g]:
+            out[r] = [t.copy() for t in tensors]
+    return out, host, plan
