@@ -375,6 +375,79 @@ def recorded_step(kt, prob, steps: int) -> dict:
     return out
 
 
+def free_port() -> int:
+    import socket
+    with socket.socket(socket.AF_INET, socket.SOCK_STREAM) as sock:
+        sock.bind(("127.0.0.1", 0))
+        return sock.getsockname()[1]
+
+
+def launch_ranks(n: int, script: str, script_args, need_devices: bool = True, capture: bool = False):
+    """Starts `n` ranks of `script` on this node, one process per GPU, the way a multi-GPU run
+    of this benchmark is launched from outside: `python -m torch.distributed.run --nnodes=1
+    --nproc-per-node n --master-addr 127.0.0.1 --master-port P script args...`.  Refuses when
+    fewer than `n` CUDA devices are visible (never fewer replicas than asked for).  Returns the
+    finished process (capture=True keeps its output instead of passing it through)."""
+    if need_devices:
+        have = torch.cuda.device_count()
+        if have < n:
+            raise SystemExit("bench.py: --gpus %d was asked for but %d CUDA device(s) are visible; refusing to "
+                             "run fewer replicas than requested" % (n, have))
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", str(n),
+           "--master-addr", "127.0.0.1", "--master-port", str(free_port()), script] + list(script_args)
+    kw = dict(stdout=subprocess.PIPE, stderr=subprocess.PIPE, text=True) if capture else {}
+    return subprocess.run(cmd, **kw)
+
+
+def init_ranks(backend: str):
+    """Reads the launcher's environment.  Returns (world, rank, local_rank, dist or None); with
+    more than one rank the process group is up when this returns.  NCCL's own start-up log is
+    kept (in a file per process, so that standard output stays one JSON line): it is the record
+    of how many ranks the communicator really has."""
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world == 1:
+        return world, rank, local, None
+    import torch.distributed as dist
+    os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+    if backend == "nccl":
+        os.environ.setdefault("NCCL_DEBUG", "INFO")
+        os.environ.setdefault("NCCL_DEBUG_SUBSYS", "INIT")
+        os.environ.setdefault("NCCL_DEBUG_FILE", os.path.join(tempfile.gettempdir(), "kt_bench_nccl_%h_%p.log"))
+        torch.cuda.set_device(local)
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    else:
+        dist.init_process_group(backend, rank=rank, world_size=world)
+    return world, rank, local, dist
+
+
+def nccl_log_summary() -> dict:
+    """What this process's NCCL start-up log says about the communicator (ranks, version, whether
+    in-switch reduction was set up); empty when NCCL wrote no log."""
+    import glob
+    import re
+    pattern = os.environ.get("NCCL_DEBUG_FILE", "")
+    if not pattern:
+        return {}
+    path = pattern.replace("%p", str(os.getpid()))
+    out = {}
+    for name in glob.glob(path.replace("%h", "*")):
+        try:
+            text = open(name, errors="replace").read()
+        except OSError:
+            continue
+        m = re.search(r"nranks (\d+)", text)
+        if m:
+            out["nranks"] = int(m.group(1))
+        m = re.search(r"NCCL version ([0-9.]+)", text)
+        if m:
+            out["version"] = m.group(1)
+        out["nvls"] = bool(re.search(r"NVLS", text))
+        out["log"] = name
+    return out
+
+
 def max_over_ranks(seconds, dist, device) -> list:
     """Every replica times its own steps; the job is as slow as its slowest replica."""
     if dist is None:
@@ -400,14 +473,8 @@ def run_ours(args) -> dict:
                 time.sleep(0.5)
     from paper_2505_10183_b200 import binding as kt
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
+    world, rank, local, dist = init_ranks("nccl")
     torch.cuda.set_device(local)
-    dist = None
-    if world > 1:
-        import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
 
     wl = W.by_name(args.workload)
     prob = Problem(wl, kt, chunk_bytes=args_chunk(args))
@@ -516,6 +583,8 @@ def run_ours(args) -> dict:
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         result["cpu_baseline"] = cpu_baseline(wl, prob.shares, budget_s=args.cpu_seconds)
     if dist is not None:
+        result["nccl"] = nccl_log_summary()
+        result["nccl"]["used_for"] = "the barriers around the timed region and the max over ranks; no data-path collective"
         dist.destroy_process_group()
     return result if rank == 0 else None
 
@@ -692,7 +761,8 @@ def run_reference(args) -> dict:
     sample = "full %s step on one host thread, host-resident inputs" % wl.name
     return {
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT,
-        "n_gpus": int(os.environ.get("WORLD_SIZE", "1")), "steps": args.steps, "warmup": args.warmup,
+        "n_gpus": max(int(os.environ.get("WORLD_SIZE", "1")), int(getattr(args, "gpus", 1))),
+        "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": round(total / args.steps * 1e3, 3), "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": wl.dtype, "data": "synthetic",
         "config": {"workload": "%s: %d tensors, %d elements per rank, K=%d ranks in %d groups, shares %s"
@@ -772,6 +842,14 @@ def main() -> None:
     if args.sweep:
         run_sweep(args)
         return
+    if args.gpus < 1:
+        raise SystemExit("bench.py: --gpus must be >= 1")
+    env_world = os.environ.get("WORLD_SIZE")
+    if env_world is not None and args.gpus not in (1, int(env_world)):
+        raise SystemExit("bench.py: --gpus %d disagrees with WORLD_SIZE=%s set by the launcher" % (args.gpus, env_world))
+    if args.impl == "ours" and env_world is None and args.gpus > 1:
+        # not started by a launcher: start the N ranks here, one process per GPU
+        sys.exit(launch_ranks(args.gpus, os.path.abspath(__file__), sys.argv[1:]).returncode)
     out = run_reference(args) if args.impl == "reference" else run_ours(args)
     if out is not None:
         print(json.dumps(out), flush=True)

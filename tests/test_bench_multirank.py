@@ -1,6 +1,9 @@
-"""The N > 1 path of the benchmark on CPU: independent replicas, max-over-ranks timing, no
-collective on the data path.  Two gloo ranks stand in for two GPUs."""
+"""The N > 1 path of the benchmark on CPU: the launcher that starts one process per GPU,
+independent replicas, max-over-ranks timing, no collective on the data path.  Two gloo ranks
+stand in for two GPUs."""
+import json
 import os
+import subprocess
 import sys
 
 import pytest
@@ -54,3 +57,35 @@ def test_reference_arm_runs_on_rank_zero_only(monkeypatch):
     assert line["impl"] == "reference" and line["n_gpus"] == 2 and line["gpu_launches"] == 0
     assert line["e2e"]["h2d_bytes_per_step"] == 0 and line["cpu_baseline"]["kind"] == "oracle"
     assert line["value"] > 0
+
+
+def test_launcher_starts_the_ranks_and_rank_zero_prints_one_line():
+    """bench.launch_ranks is what `bench.py --gpus N` calls when no launcher started it; here it
+    starts two CPU ranks of a stand-in script that uses the benchmark's rank set-up, its
+    max-over-ranks and its throughput formula."""
+    sys.path.insert(0, ROOT)
+    import bench
+    proc = bench.launch_ranks(2, os.path.join(ROOT, "tests", "_rank_standin.py"), ["--gpus", "2"],
+                              need_devices=False, capture=True)
+    assert proc.returncode == 0, proc.stderr[-2000:]
+    lines = [ln for ln in proc.stdout.splitlines() if ln.startswith("{")]
+    assert len(lines) == 1                                   # rank 0 alone reports
+    line = json.loads(lines[0])
+    assert line["n_gpus"] == 2 and line["args"] == ["--gpus", "2"]
+    assert line["slowest"] == [2.0, 5.0]
+    assert line["value"] == pytest.approx(2 * 1000 * 10 / 2.0 / 1e9)
+
+
+def test_asking_for_more_gpus_than_there_are_fails_loudly():
+    """`bench.py --gpus N` never runs fewer replicas than it was asked for."""
+    proc = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "1000", "--steps", "1"],
+                          stdout=subprocess.PIPE, stderr=subprocess.PIPE, text=True,
+                          env={k: v for k, v in os.environ.items() if k not in ("WORLD_SIZE", "RANK", "LOCAL_RANK")})
+    assert proc.returncode != 0
+    assert "--gpus 1000 was asked for" in proc.stderr and "refusing" in proc.stderr
+    assert not any(ln.startswith("{") for ln in proc.stdout.splitlines())
+    # a launcher's world size that disagrees with the flag is an error too, not a silent override
+    proc = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "4", "--steps", "1"],
+                          stdout=subprocess.PIPE, stderr=subprocess.PIPE, text=True,
+                          env=dict(os.environ, WORLD_SIZE="2", RANK="0", LOCAL_RANK="0"))
+    assert proc.returncode != 0 and "disagrees with WORLD_SIZE=2" in proc.stderr
