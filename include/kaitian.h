@@ -217,9 +217,10 @@ int kt_hier_reduce(kt_ctx *ctx, int phase, int bucket, float *const *transport, 
  * dir KT_D2H: side_stream waits for the work queued so far on main_stream, then copies the
  *        bucket's range of every transport[g] (device) to host_pinned[g] (host, pinned,
  *        same element offsets).
- * dir KT_H2D: side_stream waits for main_stream and for the last KT_D2H of the same
- *        bucket, then copies host_pinned[g] back into transport[g] (typically a second,
- *        "receive" set of device buffers).
+ * dir KT_H2D: side_stream waits for main_stream and for the last KT_D2H of every range that
+ *        overlaps this one (the same bucket, the whole transport, and with bucket == -1 each
+ *        single bucket, whichever stream those went down on), then copies host_pinned[g]
+ *        back into transport[g] (typically a second, "receive" set of device buffers).
  * Both record a completion event that kt_stage_wait consumes.  transport / host_pinned:
  * host arrays of G pointers.  bucket as in kt_hier_reduce.
  * Errors: KT_ERR_STATE, KT_ERR_SHAPE, KT_ERR_INVALID, KT_ERR_CUDA. */
@@ -256,6 +257,13 @@ int kt_stage_wait(kt_ctx *ctx, int dir, int bucket, void *main_stream, int timeo
  *        R = 1, or up to K to hand every rank its own copy; element type out_dtype;
  *        numel as registered.  16-byte aligned tensors take the vectorised path.
  * out[t][j] = cast(scale * S[tensor_offset[t] + j]); one rounded multiply; padding ignored.
+ * Destination tables: the R*T output pointers live in a small device table.  A context keeps
+ *        up to 8 such tables, one per set of output tensors it has seen (least recently used
+ *        replaced), so a caller that alternates between sets -- double-buffered gradients --
+ *        pays for each upload once.  A set seen for the first time allocates its table (device
+ *        and pinned host memory, once) and uploads it with an asynchronous copy on `stream`;
+ *        the host does not wait for the device.  A table that a recorded step uses is never
+ *        replaced (until kt_bucket_pack re-plans).
  * Errors: KT_ERR_STATE, KT_ERR_SHAPE, KT_ERR_INVALID, KT_ERR_ALIGN, KT_ERR_NOMEM, KT_ERR_CUDA. */
 int kt_unpack_scale(kt_ctx *ctx, const float *const *src, int from_combined,
                     void *const *out_grads, int R, int out_dtype, float scale, int bucket,
@@ -286,6 +294,11 @@ int kt_route(const int32_t *group_of, int K, int G, const int32_t *participants,
  * route.  out_grads, R, out_dtype, scale, bucket as in kt_unpack_scale; the gradients are
  * the ones registered by kt_bucket_pack.  May allocate the destination table like
  * kt_unpack_scale.
+ * In place: an output tensor may be one of the registered gradient tensors of the same index t
+ * and the same element type (out_grads[c*T + t] == grads[r*T + t] for any c, r: the usual
+ * all-reduce in place); the call detects exact pointer equality and reads the gradients
+ * with ordinary loads then.  Outputs that overlap registered gradients in any other way
+ * (shifted, another index, another type) are not allowed and not detected.
  * Errors: KT_ERR_STATE, KT_ERR_SHAPE, KT_ERR_INVALID, KT_ERR_ALIGN, KT_ERR_NOMEM, KT_ERR_CUDA. */
 int kt_sync_direct(kt_ctx *ctx, void *const *out_grads, int R, int out_dtype, float scale,
                    int bucket, void *stream);
@@ -372,7 +385,9 @@ int kt_copy_tensors(void *const *dst, const void *const *src, const int64_t *byt
  * streams, or different host threads without ordering) race on it: keep calls on one
  * stream, or order them with events.
  * Calls no cudaMalloc / cudaFree and no allocating library routine; host state is on the
- * stack.  Errors: KT_ERR_INVALID, KT_ERR_SHAPE, KT_ERR_ALIGN, KT_ERR_CUDA. */
+ * stack, and nothing queued on the stream refers to it after the call returns (the tables
+ * reach the scratch as the parameters of a small kernel, not through a copy from host memory).
+ * Three kernels on `stream`.  Errors: KT_ERR_INVALID, KT_ERR_SHAPE, KT_ERR_ALIGN, KT_ERR_CUDA. */
 #define KT_STATIC_MAX_ELEMS (1 << 20)
 int kt_sync_flat_static(const int32_t *group_of, const int32_t *shares, int K, int G,
                         const void *const *grads, int in_dtype, int64_t n, void *out, int out_dtype,
@@ -385,7 +400,9 @@ int kt_sync_flat_static(const int32_t *group_of, const int32_t *shares, int K, i
  * recorded instead of executed; kt_graph_launch then replays the whole sequence with one
  * submission, which removes the per-call host cost that dominates small tensor lists.
  * Rules while recording: the context must have run the same sequence once before (so that
- * its device tables are uploaded and its events exist); every copy stream must be waited
+ * its device tables are uploaded and its events exist; a call that would have to upload a
+ * destination table returns KT_ERR_STATE and kt_graph_end then drops the recording with
+ * KT_ERR_STATE); every copy stream must be waited
  * for with kt_stage_wait(..., timeout_ms < 0) before kt_graph_end; pointers, sizes, shares
  * and scale are frozen into the recording (record again after kt_set_shares).
  * kt_graph_nodes: number of recorded operations.  The graph owns no buffers.

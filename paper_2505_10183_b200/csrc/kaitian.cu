@@ -79,6 +79,23 @@ struct StageSlot {
     bool recorded = false;
 };
 
+// One destination table of kt_unpack_scale / kt_sync_direct: R*T output pointers in transport
+// tensor order, then one flag per tensor (all R destinations 16-byte aligned).  A context keeps
+// several, so that a caller that alternates between sets of output tensors (double-buffered
+// gradients) finds each set already on the device.
+constexpr int KT_OUT_SETS = 8;
+struct OutSet {
+    void *dev = nullptr;             // device table
+    char *staging = nullptr;         // pinned host image the upload reads
+    size_t cap = 0;                  // bytes of both
+    std::vector<void *> ptrs;        // what was uploaded (caller's order)
+    int R = 0, dtype = -1;
+    cudaEvent_t uploaded = nullptr;  // the upload has read the staging image
+    cudaEvent_t used = nullptr;      // the last kernel that reads the device table
+    uint64_t stamp = 0;              // last use, for replacement
+    bool in_recording = false;       // a recorded step reads this table whenever it is replayed: never replaced
+};
+
 }  // namespace
 
 struct kt_ctx {
@@ -110,10 +127,10 @@ struct kt_ctx {
     int *d_prefix = nullptr;
     TInfo *d_info = nullptr;
     const void **d_ptrs = nullptr;
-    void *d_out = nullptr;           // out pointer table + aligned flags
-    size_t d_out_cap = 0;
-    std::vector<void *> out_cached;  // host copy of the uploaded out pointers
-    int out_R = 0, out_dtype = -1;
+    std::vector<const void *> h_ptrs;   // the registered gradient pointers, [K][T] as the caller listed them
+    OutSet out_sets[KT_OUT_SETS];    // destination tables on the device, least recently used replaced
+    uint64_t out_clock = 0;
+    bool recording_broken = false;   // a call between kt_graph_begin and kt_graph_end could not be recorded
 
     cudaEvent_t ev_main = nullptr;
     std::vector<StageSlot> slots[2]; // per direction: index 0 = all buckets, 1 + b = bucket b
@@ -321,48 +338,113 @@ int check_out_args(const kt_ctx *c, void *const *out_grads, int R, int out_dtype
 }
 
 // Destination table on the device: R*T pointers in transport tensor order, then one flag per
-// tensor saying that all R destinations are 16-byte aligned.  Uploaded only when it changed.
-// *sz_ptrs receives the byte offset of the flags inside the table.
-int upload_out_table(kt_ctx *c, void *const *out_grads, int R, int out_dtype, cudaStream_t s, size_t *sz_ptrs_out) {
+// tensor saying that all R destinations are 16-byte aligned.  Looked up among the context's
+// sets; on a miss the least recently used set is replaced: its image is written into pinned
+// host memory and uploaded with an asynchronous copy on the call's stream, after a stream-side
+// wait for the last kernel that read the table it replaces.  Nothing here waits for the device
+// unless a set has to grow or is replaced again while its own upload is still in flight.
+// *set_out receives the set; the caller records set->used after its launch.
+int upload_out_table(kt_ctx *c, void *const *out_grads, int R, int out_dtype, cudaStream_t s, bool capturing,
+                     OutSet **set_out, size_t *sz_ptrs_out) {
     const int T = c->T;
     const size_t np = static_cast<size_t>(R) * T;
-    const bool same = c->out_R == R && c->out_dtype == out_dtype && c->out_cached.size() == np &&
-                      std::memcmp(c->out_cached.data(), out_grads, np * sizeof(void *)) == 0;
     const size_t sz_ptrs = round_up(np * sizeof(void *), 256);
     *sz_ptrs_out = sz_ptrs;
-    if (same) return KT_OK;
-    const size_t need = sz_ptrs + round_up(T, 256);
-    if (need > c->d_out_cap) {
-        // the previous table may still be in use by queued kernels: release it once they are done
-        if (c->d_out) {
-            KT_CUDA(cudaDeviceSynchronize());
-            cudaFree(c->d_out);
-            c->d_out = nullptr;
-            c->d_out_cap = 0;
+    OutSet *victim = nullptr;
+    for (OutSet &o : c->out_sets) {
+        if (o.dev && o.R == R && o.dtype == out_dtype && o.ptrs.size() == np &&
+            std::memcmp(o.ptrs.data(), out_grads, np * sizeof(void *)) == 0) {
+            o.stamp = ++c->out_clock;
+            o.in_recording = o.in_recording || capturing;
+            *set_out = &o;
+            return KT_OK;
         }
-        if (cudaMalloc(&c->d_out, need) != cudaSuccess) {
+        if (!o.in_recording && (!victim || o.stamp < victim->stamp)) victim = &o;
+    }
+    if (capturing) {
+        // an upload cannot be part of a recording: a replay would copy whatever the staging
+        // image holds by then
+        c->recording_broken = true;
+        return fail(KT_ERR_STATE, "this set of output tensors is not on the device yet: run the step once "
+                                  "with it before kt_graph_begin");
+    }
+    if (!victim)
+        return fail(KT_ERR_STATE, "all %d destination tables of this context are held by recorded steps; "
+                                  "kt_bucket_pack releases them", KT_OUT_SETS);
+    OutSet &o = *victim;
+    if (!o.uploaded) {
+        KT_CUDA(cudaEventCreateWithFlags(&o.uploaded, cudaEventDisableTiming));
+        KT_CUDA(cudaEventCreateWithFlags(&o.used, cudaEventDisableTiming));
+    }
+    const size_t need = sz_ptrs + round_up(T, 256);
+    if (need > o.cap) {
+        // kernels queued earlier may still read the old table: wait for the last of them, no more
+        if (o.dev) {
+            KT_CUDA(cudaEventSynchronize(o.used));
+            KT_CUDA(cudaEventSynchronize(o.uploaded));
+            cudaFree(o.dev);
+            cudaFreeHost(o.staging);
+            o.dev = nullptr;
+            o.staging = nullptr;
+            o.cap = 0;
+            o.ptrs.clear();
+        }
+        if (cudaMalloc(&o.dev, need) != cudaSuccess) {
             cudaGetLastError();
+            o.dev = nullptr;
             return fail(KT_ERR_NOMEM, "device allocation of %zu bytes failed", need);
         }
-        c->d_out_cap = need;
+        if (cudaMallocHost(reinterpret_cast<void **>(&o.staging), need) != cudaSuccess) {
+            cudaGetLastError();
+            cudaFree(o.dev);
+            o.dev = nullptr;
+            o.staging = nullptr;
+            return fail(KT_ERR_NOMEM, "pinned host allocation of %zu bytes failed", need);
+        }
+        o.cap = need;
     } else {
-        KT_CUDA(cudaStreamSynchronize(s));   // queued kernels may still read the old table
+        KT_CUDA(cudaEventSynchronize(o.uploaded));       // the image may be rewritten only once it was read
+        KT_CUDA(cudaStreamWaitEvent(s, o.used, 0));      // the table only once its last reader is done
     }
-    std::vector<char> staging(sz_ptrs + T, 0);
+    o.ptrs.clear();                                      // not a valid set until the copy is queued
+    std::memset(o.staging, 0, need);
     for (int cpy = 0; cpy < R; ++cpy)
         for (int u = 0; u < T; ++u)
-            reinterpret_cast<void **>(staging.data())[static_cast<size_t>(cpy) * T + u] =
+            reinterpret_cast<void **>(o.staging)[static_cast<size_t>(cpy) * T + u] =
                 out_grads[static_cast<size_t>(cpy) * T + (T - 1 - u)];
     for (int u = 0; u < T; ++u) {
         bool al = true;
         for (int cpy = 0; cpy < R; ++cpy) al = al && aligned16(out_grads[static_cast<size_t>(cpy) * T + (T - 1 - u)]);
-        staging[sz_ptrs + u] = al ? 1 : 0;
+        o.staging[sz_ptrs + u] = al ? 1 : 0;
     }
-    KT_CUDA(cudaMemcpy(c->d_out, staging.data(), staging.size(), cudaMemcpyHostToDevice));
-    c->out_cached.assign(out_grads, out_grads + np);
-    c->out_R = R;
-    c->out_dtype = out_dtype;
+    KT_CUDA(cudaMemcpyAsync(o.dev, o.staging, need, cudaMemcpyHostToDevice, s));
+    KT_CUDA(cudaEventRecord(o.uploaded, s));
+    KT_CUDA(cudaEventRecord(o.used, s));
+    o.ptrs.assign(out_grads, out_grads + np);
+    o.R = R;
+    o.dtype = out_dtype;
+    o.stamp = ++c->out_clock;
+    *set_out = &o;
     return KT_OK;
+}
+
+void forget_out_sets(kt_ctx *c) {
+    // a new plan changes T and the tensor order: no uploaded table stays valid
+    for (OutSet &o : c->out_sets) {
+        o.ptrs.clear();
+        o.R = 0;
+        o.dtype = -1;
+        o.in_recording = false;
+    }
+}
+
+bool is_capturing(cudaStream_t s) {
+    cudaStreamCaptureStatus st = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing(s, &st) != cudaSuccess) {
+        cudaGetLastError();
+        return false;
+    }
+    return st != cudaStreamCaptureStatusNone;
 }
 
 }  // namespace
@@ -629,7 +711,8 @@ int kt_bucket_pack(kt_ctx *c, const void *const *grads, const int64_t *numel, in
     c->prefix = prefix;
     c->info = info;
     c->planned = true;
-    c->out_cached.clear();
+    c->h_ptrs.assign(grads, grads + static_cast<size_t>(c->K) * T);
+    forget_out_sets(c);
     for (int dir = 0; dir < 2; ++dir) {
         for (auto &s : c->slots[dir]) s.recorded = false;
         while (static_cast<int>(c->slots[dir].size()) < nb + 1) {
@@ -751,10 +834,13 @@ int kt_stage_to_host(kt_ctx *c, int dir, int bucket, float *const *transport, fl
     KT_CUDA(cudaEventRecord(c->ev_main, ms));
     KT_CUDA(cudaStreamWaitEvent(ss, c->ev_main, 0));
     if (dir == KT_H2D) {
-        StageSlot &d2h = c->slots[KT_D2H][bucket + 1];
-        if (d2h.recorded) KT_CUDA(cudaStreamWaitEvent(ss, d2h.done, 0));
-        StageSlot &all = c->slots[KT_D2H][0];
-        if (bucket >= 0 && all.recorded) KT_CUDA(cudaStreamWaitEvent(ss, all.done, 0));
+        // the way up reads what the way down wrote: wait for every copy down that covered any part
+        // of this range -- the same bucket, the whole transport, and, when this call covers the
+        // whole transport, every single bucket (they may have gone down on other streams)
+        std::vector<StageSlot> &down = c->slots[KT_D2H];
+        for (int i = 0; i < static_cast<int>(down.size()); ++i)
+            if (down[i].recorded && (bucket < 0 || i == 0 || i == bucket + 1))
+                KT_CUDA(cudaStreamWaitEvent(ss, down[i].done, 0));
     }
     const size_t es = transport_elem_size(c);
     for (int g = 0; g < c->G && n > 0; ++g) {
@@ -866,7 +952,9 @@ int kt_unpack_scale(kt_ctx *c, const float *const *src, int from_combined, void 
     KT_ON_DEVICE(c->device);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     size_t sz_ptrs = 0;
-    if (int rc = upload_out_table(c, out_grads, R, out_dtype, s, &sz_ptrs)) return rc;
+    OutSet *set = nullptr;
+    const bool capturing = is_capturing(s);
+    if (int rc = upload_out_table(c, out_grads, R, out_dtype, s, capturing, &set, &sz_ptrs)) return rc;
     if (tp.n_tiles == 0) return KT_OK;
 
     K2Params p{};
@@ -880,8 +968,8 @@ int kt_unpack_scale(kt_ctx *c, const float *const *src, int from_combined, void 
         for (int g = 0; g < c->G; ++g) p.src[g] = src[g];
     }
     p.wide = all_aligned32(src, nsrc);
-    p.out_ptrs = static_cast<void *const *>(c->d_out);
-    p.out_aligned = static_cast<const unsigned char *>(c->d_out) + sz_ptrs;
+    p.out_ptrs = static_cast<void *const *>(set->dev);
+    p.out_aligned = static_cast<const unsigned char *>(set->dev) + sz_ptrs;
     p.R = R;
     p.scale = scale;
     const int src_dtype = from_combined ? KT_F32 : c->transport_dtype;
@@ -891,6 +979,7 @@ int kt_unpack_scale(kt_ctx *c, const float *const *src, int from_combined, void 
         launch_k2<unsigned short>(tp.tile, tp.n_tiles, s, p, src_dtype);
     c->launches += 1;
     KT_CUDA(cudaGetLastError());
+    if (!capturing) KT_CUDA(cudaEventRecord(set->used, s));
     return KT_OK;
 }
 
@@ -902,7 +991,9 @@ int kt_sync_direct(kt_ctx *c, void *const *out_grads, int R, int out_dtype, floa
     KT_ON_DEVICE(c->device);
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     size_t sz_ptrs = 0;
-    if (int rc = upload_out_table(c, out_grads, R, out_dtype, s, &sz_ptrs)) return rc;
+    OutSet *set = nullptr;
+    const bool capturing = is_capturing(s);
+    if (int rc = upload_out_table(c, out_grads, R, out_dtype, s, capturing, &set, &sz_ptrs)) return rc;
     if (tp.n_tiles == 0) return KT_OK;
 
     DirectParams p{};
@@ -910,17 +1001,34 @@ int kt_sync_direct(kt_ctx *c, void *const *out_grads, int R, int out_dtype, floa
     p.ptrs = c->d_ptrs;
     p.rt = c->rt;
     p.gt = c->gt;
-    p.out_ptrs = static_cast<void *const *>(c->d_out);
-    p.out_aligned = static_cast<const unsigned char *>(c->d_out) + sz_ptrs;
+    p.out_ptrs = static_cast<void *const *>(set->dev);
+    p.out_aligned = static_cast<const unsigned char *>(set->dev) + sz_ptrs;
     p.R = R;
     p.scale = scale;
+    // an output that is one of the registered gradient tensors (all-reduce in place, same element
+    // type) is legal; the kernel then reads the gradients with ordinary loads
+    bool inplace = false;
+    if (c->in_dtype == out_dtype)
+        for (int cpy = 0; cpy < R && !inplace; ++cpy)
+            for (int t = 0; t < c->T && !inplace; ++t)
+                for (int r = 0; r < c->K && !inplace; ++r)
+                    inplace = c->numel[t] > 0 && out_grads[static_cast<size_t>(cpy) * c->T + t] ==
+                                                     c->h_ptrs[static_cast<size_t>(r) * c->T + t];
     const bool in32 = c->in_dtype == KT_F32, out32 = out_dtype == KT_F32;
-    if (in32 && out32) k_direct_sync<float, float, KT_KB><<<tp.n_tiles, NT, 0, s>>>(p);
-    else if (in32) k_direct_sync<float, unsigned short, KT_KB><<<tp.n_tiles, NT, 0, s>>>(p);
-    else if (out32) k_direct_sync<unsigned short, float, KT_KB_DIRECT_BF16><<<tp.n_tiles, NT, 0, s>>>(p);
-    else k_direct_sync<unsigned short, unsigned short, KT_KB_DIRECT_BF16><<<tp.n_tiles, NT, 0, s>>>(p);
+    if (in32 && out32) {
+        if (inplace) k_direct_sync<float, float, KT_KB, true><<<tp.n_tiles, NT, 0, s>>>(p);
+        else k_direct_sync<float, float, KT_KB, false><<<tp.n_tiles, NT, 0, s>>>(p);
+    } else if (in32) {
+        k_direct_sync<float, unsigned short, KT_KB, false><<<tp.n_tiles, NT, 0, s>>>(p);
+    } else if (out32) {
+        k_direct_sync<unsigned short, float, KT_KB_DIRECT_BF16, false><<<tp.n_tiles, NT, 0, s>>>(p);
+    } else {
+        if (inplace) k_direct_sync<unsigned short, unsigned short, KT_KB_DIRECT_BF16, true><<<tp.n_tiles, NT, 0, s>>>(p);
+        else k_direct_sync<unsigned short, unsigned short, KT_KB_DIRECT_BF16, false><<<tp.n_tiles, NT, 0, s>>>(p);
+    }
     c->launches += 1;
     KT_CUDA(cudaGetLastError());
+    if (!capturing) KT_CUDA(cudaEventRecord(set->used, s));
     return KT_OK;
 }
 
@@ -988,9 +1096,16 @@ const char *kt_last_error(const kt_ctx *) { return g_err; }
 void kt_destroy(kt_ctx *c) {
     if (!c) return;
     DeviceScope device_scope_(c->device);
-    if (c->d_tables || c->d_out) cudaDeviceSynchronize();
+    bool tables = c->d_tables != nullptr;
+    for (const OutSet &o : c->out_sets) tables = tables || o.dev;
+    if (tables) cudaDeviceSynchronize();
     if (c->d_tables) cudaFree(c->d_tables);
-    if (c->d_out) cudaFree(c->d_out);
+    for (OutSet &o : c->out_sets) {
+        if (o.dev) cudaFree(o.dev);
+        if (o.staging) cudaFreeHost(o.staging);
+        if (o.uploaded) cudaEventDestroy(o.uploaded);
+        if (o.used) cudaEventDestroy(o.used);
+    }
     if (c->ev_main) cudaEventDestroy(c->ev_main);
     for (int dir = 0; dir < 2; ++dir)
         for (auto &s : c->slots[dir])
@@ -1016,6 +1131,7 @@ int kt_graph_begin(kt_ctx *c, void *stream) {
     KT_ON_DEVICE(c->device);
     // thread-local mode: other threads of the process may keep allocating while this one records
     KT_CUDA(cudaStreamBeginCapture(static_cast<cudaStream_t>(stream), cudaStreamCaptureModeThreadLocal));
+    c->recording_broken = false;
     return KT_OK;
 }
 
@@ -1029,6 +1145,12 @@ int kt_graph_end(kt_ctx *c, void *stream, kt_graph **out) {
         cudaGetLastError();
         return fail(KT_ERR_CUDA, "cudaStreamEndCapture: %s (a copy stream that was not waited for, or a call "
                                  "that cannot be recorded, ends a recording this way)", cudaGetErrorString(e));
+    }
+    if (c->recording_broken) {
+        c->recording_broken = false;
+        if (g) cudaGraphDestroy(g);
+        return fail(KT_ERR_STATE, "a call made while recording was refused (it needed an upload or an allocation): "
+                                  "the recording is incomplete and was dropped");
     }
     kt_graph *h = new (std::nothrow) kt_graph();
     if (!h) {
@@ -1311,18 +1433,28 @@ namespace {
 
 constexpr size_t STATIC_TABLE_BYTES = 4096;
 
-struct alignas(256) StaticTables {      // image of the first STATIC_TABLE_BYTES of the scratch
+struct StaticTables {                   // image of the first bytes of the scratch
     int prefix[8];                      // tiles before tensor 0 and 1
-    alignas(32) TInfo info;             // the one tensor
-    alignas(8) const void *in_ptrs[KT_MAX_RANKS];
+    TInfo info;                         // the one tensor
+    const void *in_ptrs[KT_MAX_RANKS];
     void *out_ptr[1];
     unsigned char out_aligned[8];
 };
 static_assert(sizeof(StaticTables) <= STATIC_TABLE_BYTES, "tables outgrew their slot");
+static_assert(sizeof(StaticTables) % 16 == 0 && offsetof(StaticTables, info) % 16 == 0,
+              "the tables are written, and the tensor record read, in 16-byte words");
 
 // Held by every GPU that loads the library, until the process exits.
 static __device__ __align__(256) unsigned char
     g_static_scratch[STATIC_TABLE_BYTES + static_cast<size_t>(KT_STATIC_MAX_ELEMS) * sizeof(float)];
+
+// Writes the tables into the scratch.  They travel as kernel parameters, which the runtime
+// copies when the launch is queued: the call depends on no host memory after it returns.
+__global__ void k_static_tables(const __grid_constant__ StaticTables tab, unsigned char *scratch) {
+    const uint4 *src = reinterpret_cast<const uint4 *>(&tab);
+    uint4 *dst = reinterpret_cast<uint4 *>(scratch);
+    for (unsigned i = threadIdx.x; i < sizeof(StaticTables) / sizeof(uint4); i += blockDim.x) dst[i] = src[i];
+}
 
 constexpr int STATIC_MAX_DEVICES = 64;
 std::mutex g_static_mutex;
@@ -1414,8 +1546,8 @@ extern "C" int kt_sync_flat_static(const int32_t *group_of, const int32_t *share
     }
 
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    // tables: the source is ordinary stack memory, which the runtime stages before returning
-    KT_CUDA(cudaMemcpyAsync(scratch, &tab, sizeof(tab), cudaMemcpyHostToDevice, s));
+    k_static_tables<<<1, 64, 0, s>>>(tab, scratch);
+    KT_CUDA(cudaGetLastError());
 
     TilePlan tp{};
     tp.prefix = reinterpret_cast<const int *>(scratch + offsetof(StaticTables, prefix));

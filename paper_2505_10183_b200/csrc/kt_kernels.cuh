@@ -135,6 +135,16 @@ __device__ __forceinline__ uint4 ld_stream(const void *p) {
     return v;
 }
 
+__device__ __forceinline__ uint4 ld_plain(const void *p) {
+    // for data the same launch also writes (in-place outputs): an ordinary, coherent load
+    uint4 v;
+    asm volatile("ld.global.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                 : "l"(p)
+                 : "memory");
+    return v;
+}
+
 template <typename P>
 __device__ __forceinline__ P *ldg_ptr(P *const *slot) {
     // pointer tables are read-only for the lifetime of a launch
@@ -476,7 +486,10 @@ __device__ __forceinline__ void store_out(Tout *d, const float (&y)[VEC]) {
     }
 }
 
-template <typename Tin, typename Tout, int KB, bool EDGE>
+// INPLACE: some output tensor is one of the registered gradient tensors (an all-reduce in
+// place).  Every thread reads all ranks' values of its elements before it writes them, so the
+// result is the same; only the loads must not take the read-only path.
+template <typename Tin, typename Tout, int KB, bool EDGE, bool INPLACE>
 __device__ __forceinline__ void direct_tile(const DirectParams &p, const TileRef &t) {
     constexpr int VEC = Elem<Tin>::VEC;
     constexpr int TILE = Elem<Tin>::TILE;
@@ -498,7 +511,7 @@ __device__ __forceinline__ void direct_tile(const DirectParams &p, const TileRef
 #pragma unroll
                 for (int it = 0; it < ITERS; ++it) {
                     if (!EDGE || (aligned && e[it] + VEC <= t.ti.numel))
-                        raw[j][it] = ld_stream(s + e[it]);
+                        raw[j][it] = INPLACE ? ld_plain(s + e[it]) : ld_stream(s + e[it]);
                     else
                         raw[j][it] = Elem<Tin>::gather(s, e[it], t.ti.numel);
                 }
@@ -549,13 +562,13 @@ __device__ __forceinline__ void direct_tile(const DirectParams &p, const TileRef
     }
 }
 
-template <typename Tin, typename Tout, int KB>
+template <typename Tin, typename Tout, int KB, bool INPLACE>
 __global__ void __launch_bounds__(NT) k_direct_sync(const __grid_constant__ DirectParams p) {
     const TileRef t = locate_tile(p.tp);
     if ((t.ti.flags & FLAG_ALIGNED) && p.out_aligned[t.u] && t.e0 + Elem<Tin>::TILE <= t.ti.numel)
-        direct_tile<Tin, Tout, KB, false>(p, t);
+        direct_tile<Tin, Tout, KB, false, INPLACE>(p, t);
     else
-        direct_tile<Tin, Tout, KB, true>(p, t);
+        direct_tile<Tin, Tout, KB, true, INPLACE>(p, t);
 }
 
 // ------------------------------------------------------------------ flat inter-group combine into a combined buffer

@@ -40,8 +40,11 @@ def shares_of(wl, kt=None):
 
 
 def run_gpu_path(kt, wl, dev_grads, shares, out_dtype=None, R=1, scale=1.0, per_bucket=False,
-                 use_combined=False, staged=False, relay_chunk=4 << 20, rows=False, transport_dtype=torch.float32):
-    """Returns (out[c][t] tensors, transport list, plan, ctx)."""
+                 use_combined=False, staged=False, relay_chunk=4 << 20, rows=False, transport_dtype=torch.float32,
+                 skew16=False):
+    """Returns (out[c][t] tensors, transport list, plan, ctx).  skew16: every transport, pinned
+    and receive buffer starts 16 bytes past a 32-byte boundary (the least alignment the library
+    accepts), so that 8-float accesses cannot be single 256-bit instructions."""
     ctx = kt.kt_groups_init(wl.group_of, shares, wl.G)
     if transport_dtype != torch.float32:
         kt.kt_set_transport_dtype(ctx, kt.KT_BF16)
@@ -52,6 +55,15 @@ def run_gpu_path(kt, wl, dev_grads, shares, out_dtype=None, R=1, scale=1.0, per_
     # chunk of all groups in one copy)
     def buffers(pinned=False):
         tdt = transport_dtype
+        if skew16:
+            shift = 16 // torch.empty(0, dtype=tdt).element_size()
+            out = []
+            for _ in range(wl.G):
+                whole = torch.full((n + 64,), float("nan"), dtype=tdt, device=None if pinned else "cuda")
+                whole = whole.pin_memory() if pinned else whole
+                assert whole.data_ptr() % 32 == 0
+                out.append(whole[shift:shift + n])
+            return out
         if rows:
             whole = torch.full((wl.G, n), float("nan"), dtype=tdt, device=None if pinned else "cuda")
             return list(whole.pin_memory() if pinned else whole)

@@ -127,6 +127,31 @@ def test_random_problems_misaligned_inputs_and_outputs(kt, oracle, seed):
                    out_shift=lambda c, t: shifts.setdefault((c, t), rnd.choice([0, 0, 1, 2, 3, 4])))
 
 
+@pytest.mark.parametrize("name,dtype", [("tiny", "f32"), ("mobilenet_v2", "f32"), ("resnet50", "bf16"), ("tiny", "bf16")])
+def test_all_reduce_in_place(kt, oracle, name, dtype):
+    """The outputs are the registered gradient tensors themselves: every rank's tensors are
+    overwritten with the reduced gradient (R = K), and, in a second problem, only rank 1's
+    (R = 1), the other ranks keeping their inputs.  Misaligned tensors included."""
+    for R_all in (True, False):
+        wl = W.by_name(name)
+        wl.dtype = dtype
+        shares = H.shares_of(wl, kt)
+        host, dev = H.device_gradients(wl, misalign=0 if R_all else 3)
+        ctx = kt.kt_groups_init(wl.group_of, shares, wl.G)
+        kt.kt_bucket_pack(ctx, dev, wl.bucket_cap_bytes)
+        out = dev if R_all else [dev[1]]
+        kt.kt_sync_direct(ctx, out, scale=0.5)
+        torch.cuda.synchronize()
+        want, _, _, _ = H.run_oracle_path(oracle, wl, host, shares, scale=0.5)
+        for r in range(wl.K):
+            for t in range(wl.T):
+                if R_all or r == 1:
+                    H.assert_bit_equal(dev[r][t], want[t], "rank %d tensor %d" % (r, t))
+                else:
+                    H.assert_bit_equal(dev[r][t], host[r][t], "untouched rank %d tensor %d" % (r, t))
+        kt.kt_destroy(ctx)
+
+
 def test_error_codes(kt):
     wl = W.tiny()
     _, dev = H.device_gradients(wl)

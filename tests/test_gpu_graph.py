@@ -71,13 +71,91 @@ def test_recording_a_sequence_that_cannot_be_recorded_reports_an_error(kt):
         kt.kt_hier_reduce(prob.ctx, kt.KT_INTRA, prob.transport, stream=prob.main)
         torch.cuda.synchronize()
         kt.kt_graph_begin(prob.ctx, prob.main)
-        with pytest.raises(kt.KtError):
+        with pytest.raises(kt.KtError) as e:
             prob.step()
+        assert e.value.status == kt.KT_ERR_STATE
         with pytest.raises(kt.KtError) as e:
             kt.kt_graph_end(prob.ctx, prob.main)
-        assert e.value.status == kt.KT_ERR_CUDA
+        assert e.value.status == kt.KT_ERR_STATE
         torch.cuda.synchronize()
         prob.step()                                   # eager execution still works
         torch.cuda.synchronize()
     assert bool(torch.isfinite(prob.out[0][0]).all())
     kt.kt_destroy(prob.ctx)
+
+
+@pytest.mark.parametrize("name", ["tiny", "mobilenet_v2"])
+def test_alternating_output_sets_eager_and_recorded(kt, oracle, name):
+    """Double-buffered gradients: the caller alternates between two sets of output tensors (and
+    a third route, the one-pass kernel, between two more).  Each set's destination table stays
+    on the device, so alternating needs no new upload, each set can be part of a recording,
+    and every result equals the oracle's bit for bit."""
+    wl = W.by_name(name)
+    shares = H.shares_of(wl, kt)
+    host, dev = H.device_gradients(wl)
+    ctx = kt.kt_groups_init(wl.group_of, shares, wl.G)
+    kt.kt_bucket_pack(ctx, dev, wl.bucket_cap_bytes)
+    n = kt.kt_plan_query(ctx).transport_numel
+    transport = [torch.full((n,), float("nan"), device="cuda") for _ in range(wl.G)]
+    sets = [[[torch.full((m,), float("nan"), device="cuda") for m in wl.numel]] for _ in range(4)]
+    want, _, _, _ = H.run_oracle_path(oracle, wl, host, shares)
+    main = torch.cuda.Stream()
+
+    def run(i):
+        if i < 2:
+            kt.kt_hier_reduce(ctx, kt.KT_INTRA, transport, stream=main)
+            kt.kt_unpack_scale(ctx, transport, sets[i], stream=main)
+        else:
+            kt.kt_sync_direct(ctx, sets[i], stream=main)
+
+    def check(i, what):
+        torch.cuda.synchronize()
+        for t in range(wl.T):
+            H.assert_bit_equal(sets[i][0][t], want[t], "%s: set %d out[%d]" % (what, i, t))
+            sets[i][0][t].fill_(float("nan"))
+        torch.cuda.synchronize()
+
+    with torch.cuda.stream(main):
+        for step in range(12):                       # back to back, no synchronisation between
+            run(step % 4)
+        for i in range(4):
+            check(i, "eager")
+        graphs = []
+        for i in range(4):                           # every set is already on the device: recordable
+            kt.kt_graph_begin(ctx, main)
+            run(i)
+            graphs.append(kt.kt_graph_end(ctx, main))
+        for step in range(8):
+            kt.kt_graph_launch(graphs[step % 4], main)
+        for i in range(4):
+            check(i, "recorded")
+        # tables held by recordings are never replaced: five more sets share the remaining
+        # tables in turn, and the recorded ones still replay correctly afterwards
+        extra = [[[torch.full((m,), float("nan"), device="cuda") for m in wl.numel]] for _ in range(5)]
+        for step in range(15):
+            kt.kt_sync_direct(ctx, extra[step % 5], stream=main)
+        torch.cuda.synchronize()
+        for x in extra:
+            for t in range(wl.T):
+                H.assert_bit_equal(x[0][t], want[t], "churned set out[%d]" % t)
+        kt.kt_graph_launch(graphs[0], main)
+        kt.kt_graph_launch(graphs[3], main)
+        check(0, "recorded, after other sets came and went")
+        check(3, "recorded, after other sets came and went")
+        # once every table is held by a recording, a new set is refused with a clear status
+        for i in range(4):
+            kt.kt_sync_direct(ctx, extra[i], stream=main)
+            kt.kt_graph_begin(ctx, main)
+            kt.kt_sync_direct(ctx, extra[i], stream=main)
+            graphs.append(kt.kt_graph_end(ctx, main))
+        with pytest.raises(kt.KtError) as e:
+            kt.kt_sync_direct(ctx, extra[4], stream=main)
+        assert e.value.status == kt.KT_ERR_STATE and "held by recorded steps" in str(e.value)
+        kt.kt_bucket_pack(ctx, dev, wl.bucket_cap_bytes)      # a new plan releases them
+        kt.kt_sync_direct(ctx, extra[4], stream=main)
+        torch.cuda.synchronize()
+        for t in range(wl.T):
+            H.assert_bit_equal(extra[4][0][t], want[t], "after re-planning out[%d]" % t)
+    for g in graphs:
+        kt.kt_graph_destroy(g)
+    kt.kt_destroy(ctx)

@@ -163,39 +163,61 @@ def test_mobilenet_v2_ragged(kt, oracle):
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
 @pytest.mark.parametrize("nbytes", [4 << 10, 64 << 10, 1 << 20, 16 << 20])
 def test_sweep_small_points(kt, oracle, K, dtype, nbytes):
-    if nbytes == 16 << 20 and K == 16 and dtype == "bf16":
-        pytest.skip("covered by the fp32 point of the same size")
     compare_all(kt, oracle, W.sweep_point(K, nbytes, dtype))
 
 
-def test_sweep_large_point_sampled_windows(kt, oracle):
-    """1 GiB per rank, K = 4: device-generated values; 2^20-element windows are copied to
-    the host and checked element by element (the path is element-wise, so a window's
-    result depends on that window's inputs only)."""
-    wl = W.sweep_point(4, 1 << 30, "f32")
+def check_sampled_windows(kt, oracle, K, nbytes, dtype, n_random=6):
+    """A flat sweep point too large for the oracle to walk in full: device-generated values;
+    2^20-element windows (the first, the last, and random ones at odd offsets) are copied to
+    the host and checked element by element.  The path is element-wise, so a window's result
+    depends on that window's inputs only."""
+    wl = W.sweep_point(K, nbytes, dtype)
     shares = wl.shares
     n = wl.N
+    dt = H.ORACLE_DT[dtype]
     dev = [[W.rank_gradients(wl, r, "cuda")] for r in range(wl.K)]
     ctx = kt.kt_groups_init(wl.group_of, shares, wl.G)
     kt.kt_bucket_pack(ctx, dev, wl.bucket_cap_bytes)
     plan = kt.kt_plan_query(ctx)
     assert plan.transport_numel == n and plan.n_buckets == 1
-    transport = [torch.empty(n, device="cuda") for _ in range(wl.G)]
-    out = [[torch.empty(n, device="cuda")]]
+    transport = [torch.full((n,), float("nan"), device="cuda") for _ in range(wl.G)]
+    out = [[torch.full((n,), float("nan"), dtype=H.TORCH_DT[dtype], device="cuda")]]
+    direct = [[torch.full((n,), float("nan"), dtype=H.TORCH_DT[dtype], device="cuda")]]
     kt.kt_hier_reduce(ctx, kt.KT_INTRA, transport)
     kt.kt_unpack_scale(ctx, transport, out)
+    kt.kt_sync_direct(ctx, direct)
     torch.cuda.synchronize()
     win = 1 << 20
-    rng = np.random.default_rng(5)
-    starts = [0, n - win] + (rng.integers(0, n // win - 1, size=6) * win + 12345).tolist()
+    rng = np.random.default_rng(5 + K)
+    starts = [0, n - win] + (rng.integers(0, n // win - 1, size=n_random) * win + 12344).tolist()
     for s in starts:
         s = int(min(max(s, 0), n - win))
         hx = [[W.as_numpy(dev[r][0][s:s + win])] for r in range(wl.K)]
-        o_out, o_parts, _, _ = oracle.sync_step(hx, [win], F32, wl.group_of, shares, wl.G, 1 << 62)
+        o_out, o_parts, _, _ = oracle.sync_step(hx, [win], dt, wl.group_of, shares, wl.G, 1 << 62)
         for g in range(wl.G):
             H.assert_bit_equal(transport[g][s:s + win], o_parts[g], "window %d transport[%d]" % (s, g))
         H.assert_bit_equal(out[0][0][s:s + win], o_out[0], "window %d out" % s)
+        H.assert_bit_equal(direct[0][0][s:s + win], o_out[0], "window %d one-pass out" % s)
+    # no window was skipped by the kernels: nothing of the NaN fill is left anywhere
+    for t in transport + out[0] + direct[0]:
+        assert not bool(torch.isnan(t).any())
     kt.kt_destroy(ctx)
+    del dev, transport, out, direct
+    torch.cuda.empty_cache()
+
+
+def test_sweep_large_point_sampled_windows(kt, oracle):
+    """1 GiB per rank, K = 4, fp32."""
+    check_sampled_windows(kt, oracle, 4, 1 << 30, "f32")
+
+
+@pytest.mark.parametrize("K", [8, 16])
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("nbytes", [64 << 20, 256 << 20, 1 << 30])
+def test_sweep_large_points_sampled_windows(kt, oracle, K, dtype, nbytes):
+    """The bucket sizes the bandwidth target is stated for (64 MiB and up per rank), with
+    8 and 16 ranks, fp32 and bf16 gradients."""
+    check_sampled_windows(kt, oracle, K, nbytes, dtype)
 
 
 # ------------------------------------------------------------------ variants and edge cases
@@ -356,6 +378,42 @@ def test_staging_bytes_and_ordering(kt, oracle):
     _, o_parts, _, _ = H.run_oracle_path(oracle, wl, host_g, shares)
     for g in range(wl.G):
         H.assert_bit_equal(pinned[g], o_parts[g])
+    kt.kt_destroy(ctx)
+
+
+def test_whole_transport_goes_up_only_after_every_bucket_came_down(kt, oracle):
+    """Mixed granularity on different copy streams: the partials go down bucket by bucket on one
+    stream, the whole transport comes back up in one call on another.  The way up must wait
+    for every bucket's way down (the pinned buffers are poisoned first)."""
+    wl = W.resnet18()
+    shares = H.shares_of(wl, kt)
+    host_g, dev = H.device_gradients(wl)
+    ctx = kt.kt_groups_init(wl.group_of, shares, wl.G)
+    kt.kt_bucket_pack(ctx, dev, wl.bucket_cap_bytes)
+    plan = kt.kt_plan_query(ctx)
+    n = plan.transport_numel
+    assert plan.n_buckets >= 2
+    tr = [torch.empty(n, device="cuda") for _ in range(wl.G)]
+    recv = [torch.empty(n, device="cuda") for _ in range(wl.G)]
+    pinned = [torch.zeros(n).pin_memory() for _ in range(wl.G)]
+    down, up = torch.cuda.Stream(), torch.cuda.Stream()
+    poison = float(np.float32(-7.25e33))
+    for _ in range(3):
+        for p, r in zip(pinned, recv):
+            p.fill_(poison)
+            r.fill_(float("nan"))
+        torch.cuda.synchronize()
+        kt.kt_hier_reduce(ctx, kt.KT_INTRA, tr)
+        for b in range(plan.n_buckets):
+            kt.kt_stage_to_host(ctx, kt.KT_D2H, tr, pinned, bucket=b, side_stream=down)
+        kt.kt_stage_to_host(ctx, kt.KT_H2D, recv, pinned, bucket=-1, side_stream=up)
+        kt.kt_stage_wait(ctx, kt.KT_H2D, bucket=-1, timeout_ms=20000)
+        torch.cuda.synchronize()
+        for g in range(wl.G):
+            assert not bool((recv[g] == poison).any())
+    _, o_parts, _, _ = H.run_oracle_path(oracle, wl, host_g, shares)
+    for g in range(wl.G):
+        H.assert_bit_equal(recv[g], o_parts[g], "receive buffer %d" % g)
     kt.kt_destroy(ctx)
 
 

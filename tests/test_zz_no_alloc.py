@@ -6,12 +6,18 @@ memory pool, processes whose device memory is planned up front.  For them the li
 the scratch of the flat path in a fixed device array.  This test calls that entry point
 through the C ABI twice in a row -- the second call with other sizes, groups and dtypes, so
 that whatever the first call left in the shared array would show -- and checks each result
-bit for bit against the existing route (kt_groups_init + kt_bucket_pack + kt_hier_reduce +
-kt_unpack_scale), the same bar as the other GPU tests.  The file sorts last on purpose:
-a run that stops at the first failure has then already run every other test.
+bit for bit against the CPU oracle on host copies of the same bytes and against the existing
+route (kt_groups_init + kt_bucket_pack + kt_hier_reduce + kt_unpack_scale), the same bar as
+the other GPU tests.  It also checks the property the entry point exists for: the device's
+free memory is the same before and after the calls.  The file sorts last on purpose: a run
+that stops at the first failure has then already run every other test.
 """
 import pytest
 import torch
+
+from paper_2505_10183_b200 import workloads as W
+
+import _harness as H
 
 pytestmark = pytest.mark.gpu
 
@@ -53,7 +59,16 @@ def same_bits(a, b):
     return torch.equal(a.view(view), b.view(view))
 
 
-def test_static_scratch_entry_matches_existing_route_twice_in_a_row(kt):
+def oracle_result(oracle, c, grads):
+    """The oracle's whole step on host copies of the very bytes the device holds."""
+    dt = {torch.float32: 0, torch.bfloat16: 1}
+    host = [[W.as_numpy(g)] for g in grads]
+    out, _, _, _ = oracle.sync_step(host, [c["n"]], dt[c["dtype"]], c["group_of"], c["shares"],
+                                    max(c["group_of"]) + 1, 1 << 62, c["scale"], dt[c["out_dtype"]])
+    return out[0]
+
+
+def test_static_scratch_entry_matches_oracle_and_existing_route_twice_in_a_row(kt, oracle):
     cases = [
         # first call: uneven shares, three groups, ragged length, fp32
         dict(group_of=[0, 0, 0, 1, 1, 2], shares=[40, 40, 29, 29, 19, 19], n=100_003, dtype=torch.float32,
@@ -64,17 +79,27 @@ def test_static_scratch_entry_matches_existing_route_twice_in_a_row(kt):
     ]
     inputs = [make_grads(len(c["group_of"]), c["n"], c["dtype"], 900 + i, c["misalign"]) for i, c in enumerate(cases)]
     outs = [torch.full((c["n"],), float("nan"), dtype=c["out_dtype"], device="cuda") for c in cases]
-    for c, g, o in zip(cases, inputs, outs):          # back to back, no synchronisation between
+    third = torch.full((cases[0]["n"],), float("nan"), device="cuda")
+    # One warm-up call per case before the free-memory reading: the first call on a device looks
+    # up the scratch address, and the driver loads a kernel's code when it is first launched.
+    for c, g, o in zip(cases, inputs, outs):
         kt.kt_sync_flat_static(c["group_of"], c["shares"], g, o, scale=c["scale"])
     torch.cuda.synchronize()
-    for c, g, o in zip(cases, inputs, outs):
-        want = existing_route(kt, c["group_of"], c["shares"], g, c["out_dtype"], c["scale"])
-        assert same_bits(o, want)
-    # and once more with the first case: the array now holds the second call's leftovers
-    o = torch.full((cases[0]["n"],), float("nan"), device="cuda")
-    kt.kt_sync_flat_static(cases[0]["group_of"], cases[0]["shares"], inputs[0], o, scale=1.0)
+    for o in outs:
+        o.fill_(float("nan"))
     torch.cuda.synchronize()
-    assert same_bits(o, outs[0])
+    free_before = torch.cuda.mem_get_info()[0]
+    for c, g, o in zip(cases, inputs, outs):          # back to back, no synchronisation between
+        kt.kt_sync_flat_static(c["group_of"], c["shares"], g, o, scale=c["scale"])
+    # and once more with the first case: the array now holds the second call's leftovers
+    kt.kt_sync_flat_static(cases[0]["group_of"], cases[0]["shares"], inputs[0], third, scale=1.0)
+    torch.cuda.synchronize()
+    assert torch.cuda.mem_get_info()[0] == free_before, "the calls changed the device's free memory"
+    for c, g, o in zip(cases, inputs, outs):
+        want = oracle_result(oracle, c, g)
+        H.assert_bit_equal(o, want, "kt_sync_flat_static against the oracle")
+        assert same_bits(o, existing_route(kt, c["group_of"], c["shares"], g, c["out_dtype"], c["scale"]))
+    assert same_bits(third, outs[0])
 
 
 def test_static_scratch_entry_rejects_what_does_not_fit(kt):
