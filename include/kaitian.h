@@ -198,6 +198,77 @@ int kt_plan_query(const kt_ctx *ctx, int32_t *n_buckets, int64_t *bucket_start,
                   int64_t *bucket_numel, int64_t *tensor_offset, int32_t *bucket_of,
                   int64_t *transport_numel);
 
+/* One rank per device (Section III-A: the devices of a group run the group's collective among
+ * themselves, device to device; Section III-B, steps 2-3).  The calls above and below treat
+ * all K ranks' tensors as resident in one device's memory.  When every rank is a process with
+ * a device of its own, each device does a share of every collective: the range of a call (one
+ * bucket, or the whole transport with bucket == -1) is cut into work units of
+ * kt_work_unit(in_dtype) transport elements that never cross a tensor (a tensor owns the
+ * transport from its offset to the next tensor's offset, padding included, and holds
+ * ceil(extent / unit) units); with U units in the range and M members in the group, member m
+ * (ranks of the group in ascending order) owns units floor(m*U/M) ... floor((m+1)*U/M) - 1,
+ * one contiguous element range.
+ *
+ * kt_work_unit:    elements per work unit for gradients of in_dtype (negative status if unknown).
+ * kt_shard_ranges: the members' element ranges as a pure host function (no context, no
+ *        device): numel, T, bucket_cap_bytes as in kt_plan_buckets; lo_out[n_members],
+ *        n_out[n_members] (host) receive start and length of every member's range; a member
+ *        without a unit gets length 0.  Errors: KT_ERR_INVALID, KT_ERR_SHAPE.
+ * kt_shard_bind:   declares that the context belongs to rank `rank` of the map given to
+ *        kt_groups_init.  Call it before kt_bucket_pack.  From then on
+ *          - kt_bucket_pack takes the tensors of the M members of the rank's group only:
+ *            grads[m*T + t], members in ascending rank order, the rank's own tensors by their
+ *            ordinary addresses and its group mates' tensors by addresses under which this
+ *            device can read them (peer-mapped: kt_ipc_open, or peer access inside one
+ *            process).  They are read with ordinary loads.
+ *          - kt_hier_reduce(KT_INTRA) forms the group partial over this member's share of
+ *            the range, from all M members' tensors, into transport[own group] (the other
+ *            entries of `transport` are not looked at);
+ *          - kt_stage_to_host(KT_D2H) copies that share of transport[own group] down;
+ *            kt_stage_to_host(KT_H2D) copies the same element range of every OTHER group's
+ *            partial up (host_pinned is memory that all processes share; between the two
+ *            the caller needs a barrier across processes, after its own copy down has
+ *            finished, because other processes write what the way up reads);
+ *          - kt_hier_reduce(KT_INTER), kt_unpack_scale and kt_sync_direct work on the share
+ *            only; with R = M and out_grads[m*T + t] addressing member m's output tensors
+ *            (peer-mapped again) every member receives this member's share of the result,
+ *            so that after all members have run, and a barrier, every rank holds the whole
+ *            reduced gradient.  kt_sync_direct needs G == 1 (it reads all ranks).
+ *          - kt_relay_through_host, kt_allreduce across groups, the broadcast calls and the
+ *            standalone pack return KT_ERR_STATE.
+ *        Per element the arithmetic and its order are unchanged: results are bit-identical to
+ *        the unsharded calls.  Ranks synchronise on the host (barriers); no kernel waits for
+ *        another device.  Errors: KT_ERR_INVALID.
+ * kt_shard_query:  the element range of `member` (-1: this context's own) for `bucket` under
+ *        the registered plan, and the number of members (each output may be NULL).
+ *        Errors: KT_ERR_STATE, KT_ERR_SHAPE, KT_ERR_INVALID. */
+int kt_work_unit(int in_dtype);
+int kt_shard_ranges(const int64_t *numel, int T, int64_t bucket_cap_bytes, int64_t unit, int bucket,
+                    int n_members, int64_t *lo_out, int64_t *n_out);
+int kt_shard_bind(kt_ctx *ctx, int rank);
+int kt_shard_query(const kt_ctx *ctx, int bucket, int member, int *n_members, int64_t *lo, int64_t *n);
+
+/* Memory shared between the processes of one node, for one rank per device.
+ * kt_ipc_export: dev_ptr (device, anywhere inside an allocation made with cudaMalloc, e.g. by a
+ *        framework's allocator) -> a handle of KT_IPC_HANDLE_BYTES bytes (host) naming the
+ *        allocation, and the pointer's byte offset inside it.  Both are plain bytes that can be
+ *        sent to another process of the node.
+ * kt_ipc_open:   in another process, with the device current that shall read or write the
+ *        memory: handle + offset -> *dev_ptr_out, an address valid in this process.  A handle is
+ *        mapped once per process and device and counted; the exporting process must keep the
+ *        allocation alive while it is open elsewhere.
+ * kt_ipc_close:  gives one reference back; the last one unmaps.
+ * kt_host_register / kt_host_unregister: page-locks `bytes` bytes of host memory at `host`
+ *        (for instance a POSIX shared-memory segment mapped by every process) so that
+ *        kt_stage_to_host can copy to and from it asynchronously.
+ * Errors: KT_ERR_INVALID, KT_ERR_STATE, KT_ERR_CUDA. */
+#define KT_IPC_HANDLE_BYTES 64
+int kt_ipc_export(const void *dev_ptr, void *handle_out, int64_t *offset_out);
+int kt_ipc_open(const void *handle, int64_t offset, void **dev_ptr_out);
+int kt_ipc_close(const void *handle);
+int kt_host_register(void *host, int64_t bytes);
+int kt_host_unregister(void *host);
+
 /* The two reductions of Section III-A.
  * transport: host array of G device pointers, fp32, transport_numel elements each,
  *        16-byte aligned.

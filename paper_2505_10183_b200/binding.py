@@ -29,7 +29,8 @@ EXPORTS = ["kt_schedule", "kt_scores", "kt_adapt_create", "kt_adapt_observe", "k
            "kt_graph_nodes", "kt_graph_destroy", "kt_groups_init", "kt_set_shares", "kt_set_coefficients",
            "kt_get_coefficients", "kt_set_transport_dtype", "kt_route", "kt_bucket_pack", "kt_plan_buckets", "kt_plan_query", "kt_hier_reduce",
            "kt_stage_to_host", "kt_relay_through_host", "kt_stage_wait", "kt_unpack_scale", "kt_sync_direct", "kt_allreduce", "kt_bcast_send", "kt_bcast_relay", "kt_bcast_recv", "kt_cast", "kt_copy_tensors", "kt_sync_flat_static", "kt_launch_count",
-           "kt_last_error", "kt_destroy"]
+           "kt_last_error", "kt_destroy", "kt_work_unit", "kt_shard_ranges", "kt_shard_bind", "kt_shard_query",
+           "kt_ipc_export", "kt_ipc_open", "kt_ipc_close", "kt_host_register", "kt_host_unregister"]
 
 _DTYPES = {torch.float32: KT_F32, torch.bfloat16: KT_BF16}
 
@@ -86,6 +87,15 @@ def _load() -> C.CDLL:
         "kt_copy_tensors": ([vpp, vpp, i64p, C.c_int, C.c_int, vp], C.c_int),
         "kt_sync_flat_static": ([i32p, i32p, C.c_int, C.c_int, vpp, C.c_int, C.c_int64, vp, C.c_int,
                                  C.c_float, vp], C.c_int),
+        "kt_work_unit": ([C.c_int], C.c_int),
+        "kt_shard_ranges": ([i64p, C.c_int, C.c_int64, C.c_int64, C.c_int, C.c_int, i64p, i64p], C.c_int),
+        "kt_shard_bind": ([vp, C.c_int], C.c_int),
+        "kt_shard_query": ([vp, C.c_int, C.c_int, C.POINTER(C.c_int), i64p, i64p], C.c_int),
+        "kt_ipc_export": ([vp, vp, i64p], C.c_int),
+        "kt_ipc_open": ([vp, C.c_int64, vpp], C.c_int),
+        "kt_ipc_close": ([vp], C.c_int),
+        "kt_host_register": ([vp, C.c_int64], C.c_int),
+        "kt_host_unregister": ([vp], C.c_int),
         "kt_launch_count": ([vp], C.c_int64),
         "kt_last_error": ([vp], C.c_char_p),
         "kt_destroy": ([vp], None),
@@ -160,6 +170,7 @@ class Ctx:
     def __init__(self, handle: int, K: int, G: int):
         self.handle = C.c_void_p(handle)
         self.K, self.G, self.T = K, G, 0
+        self.sources = K              # rank lists kt_bucket_pack expects (the group's members once bound to a rank)
         self._keep = {}
 
     def __del__(self):
@@ -309,11 +320,11 @@ def kt_get_coefficients(ctx: Ctx):
 def kt_bucket_pack(ctx: Ctx, grads: Sequence[Sequence[torch.Tensor]], bucket_cap_bytes: int,
                    flat_out: Optional[Ptrs] = None, stream=None) -> None:
     """grads[r][t]: tensor t of rank r (contiguous, all of one dtype, same shapes per rank)."""
-    if len(grads) != ctx.K:
-        raise KtError(KT_ERR_SHAPE, "expected gradient lists of %d ranks" % ctx.K)
+    if len(grads) != ctx.sources:
+        raise KtError(KT_ERR_SHAPE, "expected gradient lists of %d ranks" % ctx.sources)
     T = len(grads[0])
     flat = []
-    for r in range(ctx.K):
+    for r in range(ctx.sources):
         if len(grads[r]) != T:
             raise KtError(KT_ERR_SHAPE, "rank %d holds %d tensors, rank 0 holds %d" % (r, len(grads[r]), T))
         for t in range(T):
@@ -331,6 +342,83 @@ def kt_bucket_pack(ctx: Ctx, grads: Sequence[Sequence[torch.Tensor]], bucket_cap
                                fo.array if fo is not None else None, _stream(stream)))
     ctx.T = T
     ctx._keep["grads"] = pa
+
+
+def kt_bucket_pack_ptrs(ctx: Ctx, grads: PtrArray, numel: Sequence[int], dtype: int, bucket_cap_bytes: int,
+                        stream=None) -> None:
+    """kt_bucket_pack from raw device addresses (grads: rank-major, ctx.sources * len(numel)
+    pointers), for tensors that are not torch tensors of this process: memory of other
+    processes mapped with kt_ipc_open."""
+    T = len(numel)
+    if grads.n != ctx.sources * T:
+        raise KtError(KT_ERR_SHAPE, "expected %d gradient pointers" % (ctx.sources * T))
+    n = (C.c_int64 * max(T, 1))(*[int(v) for v in numel])
+    _check(_lib.kt_bucket_pack(ctx.handle, grads.array, n, T, int(dtype), int(bucket_cap_bytes), None, _stream(stream)))
+    ctx.T = T
+    ctx._keep["grads"] = grads
+
+
+def kt_work_unit(dtype: int) -> int:
+    u = int(_lib.kt_work_unit(int(dtype)))
+    _check(u if u < 0 else 0)
+    return u
+
+
+def kt_shard_ranges(numel: Sequence[int], bucket_cap_bytes: int, unit: int, bucket: int, n_members: int):
+    """Pure host: [(lo, n)] per member, the element range of the transport each of the
+    n_members devices of a group works on."""
+    T = len(numel)
+    n = (C.c_int64 * max(T, 1))(*[int(v) for v in numel])
+    lo = (C.c_int64 * max(n_members, 1))()
+    cnt = (C.c_int64 * max(n_members, 1))()
+    _check(_lib.kt_shard_ranges(n, T, int(bucket_cap_bytes), int(unit), int(bucket), int(n_members), lo, cnt))
+    return [(int(lo[m]), int(cnt[m])) for m in range(n_members)]
+
+
+def kt_shard_bind(ctx: Ctx, rank: int, group_of: Sequence[int]) -> None:
+    """Binds the context to one rank (one rank per device); group_of is the map given to
+    kt_groups_init, used here only to know how many rank lists kt_bucket_pack will expect."""
+    _check(_lib.kt_shard_bind(ctx.handle, int(rank)))
+    ctx.sources = sum(1 for g in group_of if g == group_of[rank])
+
+
+def kt_shard_query(ctx: Ctx, bucket: int = -1, member: int = -1):
+    """Returns (lo, n, members): this context's (or `member`'s) element range for `bucket`."""
+    M, lo, n = C.c_int(0), C.c_int64(0), C.c_int64(0)
+    _check(_lib.kt_shard_query(ctx.handle, int(bucket), int(member), C.byref(M), C.byref(lo), C.byref(n)))
+    return int(lo.value), int(n.value), int(M.value)
+
+
+KT_IPC_HANDLE_BYTES = 64
+
+
+def kt_ipc_export(address: int):
+    """Returns (handle bytes, offset) for a device address inside a cudaMalloc allocation."""
+    h = (C.c_ubyte * KT_IPC_HANDLE_BYTES)()
+    off = C.c_int64(0)
+    _check(_lib.kt_ipc_export(C.c_void_p(int(address)), h, C.byref(off)))
+    return bytes(h), int(off.value)
+
+
+def kt_ipc_open(handle: bytes, offset: int) -> int:
+    """Maps another process's allocation on the current device; returns the address."""
+    out = C.c_void_p()
+    buf = (C.c_ubyte * KT_IPC_HANDLE_BYTES).from_buffer_copy(handle)
+    _check(_lib.kt_ipc_open(buf, int(offset), C.byref(out)))
+    return int(out.value)
+
+
+def kt_ipc_close(handle: bytes) -> None:
+    buf = (C.c_ubyte * KT_IPC_HANDLE_BYTES).from_buffer_copy(handle)
+    _check(_lib.kt_ipc_close(buf))
+
+
+def kt_host_register(address: int, nbytes: int) -> None:
+    _check(_lib.kt_host_register(C.c_void_p(int(address)), int(nbytes)))
+
+
+def kt_host_unregister(address: int) -> None:
+    _check(_lib.kt_host_unregister(C.c_void_p(int(address))))
 
 
 def kt_plan_buckets(numel: Sequence[int], bucket_cap_bytes: int) -> Plan:

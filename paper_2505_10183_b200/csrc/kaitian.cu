@@ -132,6 +132,12 @@ struct kt_ctx {
     uint64_t out_clock = 0;
     bool recording_broken = false;   // a call between kt_graph_begin and kt_graph_end could not be recorded
 
+    // one rank per device (kt_shard_bind): this context belongs to rank `shard_rank`, member
+    // `shard_member` of the `shard_M` ranks of group `shard_g`; it works on that member's share
+    // of every range and reads the gradients of its group's members only
+    int shard_rank = -1, shard_g = 0, shard_member = 0, shard_M = 0;
+    RankTab shard_rt{};              // the group's members alone, in ascending rank order
+
     cudaEvent_t ev_main = nullptr;
     std::vector<StageSlot> slots[2]; // per direction: index 0 = all buckets, 1 + b = bucket b
     std::vector<cudaEvent_t> chunk_events;   // chunk k went down: its way up may start
@@ -142,6 +148,35 @@ struct kt_ctx {
 namespace {
 
 int64_t round_up(int64_t x, int64_t m) { return (x + m - 1) / m * m; }
+
+bool sharded(const kt_ctx *c) { return c->shard_rank >= 0; }
+// how many ranks' gradient tensors a context reads: all of them, or its own group's
+int n_sources(const kt_ctx *c) { return sharded(c) ? c->shard_M : c->K; }
+// which of the caller's rank lists feeds position k of the device pointer table
+int source_of(const kt_ctx *c, int k) { return sharded(c) ? k : c->order[k]; }
+const RankTab &reduce_table(const kt_ctx *c) { return sharded(c) ? c->shard_rt : c->rt; }
+
+// The group's own rows of the rank table, for a context bound to one rank.
+void refresh_shard(kt_ctx *c) {
+    if (!sharded(c)) return;
+    std::memset(&c->shard_rt, 0, sizeof(c->shard_rt));
+    int m = 0;
+    for (int k = 0; k < c->K; ++k) {
+        if (c->rt.gid[k] != c->shard_g) continue;
+        c->shard_rt.coef[m] = c->rt.coef[k];
+        c->shard_rt.gid[m] = static_cast<signed char>(c->shard_g);
+        ++m;
+    }
+    c->shard_rt.first[0] = 1;
+    c->shard_rt.last[m - 1] = 1;
+    c->shard_rt.K = m;
+}
+
+// Member m of M owns units [floor(m U / M), floor((m + 1) U / M)) of a range of U work units.
+void member_units(int64_t U, int member, int M, int64_t *first, int64_t *past) {
+    *first = static_cast<int64_t>(member) * U / M;
+    *past = static_cast<int64_t>(member + 1) * U / M;
+}
 
 // Bucket plan: tensors in reverse list order, greedy fill up to cap elements, tensors never
 // split, every tensor at a multiple of 8 elements, every bucket at a multiple of 64.
@@ -206,6 +241,7 @@ int compute_coefficients(kt_ctx *c) {
     c->gt.G = c->G;
     for (int g = 0; g < c->G; ++g)
         c->gt.W[g] = static_cast<float>(static_cast<double>(Bg[g]) / static_cast<double>(B));
+    refresh_shard(c);
     return KT_OK;
 }
 
@@ -245,20 +281,60 @@ int grid_for(kt_ctx *c, Kern kernel, size_t smem, long long units) {
     return static_cast<int>(g < 1 ? 1 : g);
 }
 
+// Work units [*t0, *t1) of a call's range (one bucket, or everything for bucket == -1) that the
+// context works on: all of them, or, bound to one rank, that member's share.
+void unit_range(const kt_ctx *c, int bucket, int member, int *t0, int *t1) {
+    const int u_lo = bucket < 0 ? 0 : c->bucket_u_lo[bucket];
+    const int u_hi = bucket < 0 ? c->T : c->bucket_u_hi[bucket];
+    *t0 = c->prefix[u_lo];
+    *t1 = c->prefix[u_hi];
+    if (member >= 0) {
+        int64_t first, past;
+        member_units(*t1 - *t0, member, c->shard_M, &first, &past);
+        *t1 = *t0 + static_cast<int>(past);
+        *t0 = *t0 + static_cast<int>(first);
+    }
+}
+
+// The tensor (transport order) that holds work unit `tile`; T for the index past the last unit.
+int tensor_of_unit(const kt_ctx *c, int tile) {
+    return static_cast<int>(std::upper_bound(c->prefix.begin(), c->prefix.end(), tile) - c->prefix.begin()) - 1;
+}
+
+// First transport element of a work unit; transport_numel for the index past the last unit.
+// Tensors follow one another without gaps (a tensor's extent includes the padding behind it),
+// so a run of units is one contiguous element range.
+int64_t unit_start(const kt_ctx *c, int tile) {
+    const int u = tensor_of_unit(c, tile);
+    if (u >= c->T) return c->transport_numel;
+    return c->info[u].dst_off + static_cast<int64_t>(tile - c->prefix[u]) * c->tile;
+}
+
 // tile range of a bucket (or of everything for bucket == -1)
 int make_tile_plan(const kt_ctx *c, int bucket, TilePlan *tp) {
     if (bucket < -1 || bucket >= static_cast<int>(c->bucket_start.size()))
         return fail(KT_ERR_SHAPE, "bucket %d out of range [-1, %d)", bucket, (int)c->bucket_start.size());
+    int t0, t1;
+    unit_range(c, bucket, sharded(c) ? c->shard_member : -1, &t0, &t1);
     tp->prefix = c->d_prefix;
     tp->info = c->d_info;
     tp->T = c->T;
-    tp->u_lo = bucket < 0 ? 0 : c->bucket_u_lo[bucket];
-    tp->u_hi = bucket < 0 ? c->T : c->bucket_u_hi[bucket];
-    tp->tile_lo = c->prefix[tp->u_lo];
-    tp->n_tiles = c->prefix[tp->u_hi] - tp->tile_lo;
+    if (sharded(c)) {            // the tensors that hold the share's first and last unit
+        tp->u_lo = t1 > t0 ? tensor_of_unit(c, t0) : 0;
+        tp->u_hi = t1 > t0 ? tensor_of_unit(c, t1 - 1) + 1 : 0;
+    } else {
+        tp->u_lo = bucket < 0 ? 0 : c->bucket_u_lo[bucket];
+        tp->u_hi = bucket < 0 ? c->T : c->bucket_u_hi[bucket];
+    }
+    tp->tile_lo = t0;
+    tp->n_tiles = t1 - t0;
     tp->tile = c->tile;
     tp->single = tp->u_hi - tp->u_lo == 1;
-    if (tp->single) tp->one = c->info[tp->u_lo];
+    tp->single_skip = 0;
+    if (tp->single) {
+        tp->one = c->info[tp->u_lo];
+        tp->single_skip = t0 - c->prefix[tp->u_lo];
+    }
     tp->tables = c->d_tables;
     tp->table_bytes = static_cast<int>(c->d_tables_bytes < static_cast<size_t>(NT) * 128 ? c->d_tables_bytes
                                                                                           : static_cast<size_t>(NT) * 128);
@@ -266,6 +342,13 @@ int make_tile_plan(const kt_ctx *c, int bucket, TilePlan *tp) {
 }
 
 void bucket_range(const kt_ctx *c, int bucket, int64_t *lo, int64_t *n) {
+    if (sharded(c)) {
+        int t0, t1;
+        unit_range(c, bucket, c->shard_member, &t0, &t1);
+        *lo = unit_start(c, t0);
+        *n = unit_start(c, t1) - *lo;
+        return;
+    }
     if (bucket < 0) {
         *lo = 0;
         *n = c->transport_numel;
@@ -569,6 +652,7 @@ int kt_set_coefficients(kt_ctx *c, const float *a, const float *W) {
     if (!a || !W) return fail(KT_ERR_INVALID, "NULL argument");
     for (int k = 0; k < c->K; ++k) c->rt.coef[k] = a[c->order[k]];
     for (int g = 0; g < c->G; ++g) c->gt.W[g] = W[g];
+    refresh_shard(c);
     return KT_OK;
 }
 
@@ -623,9 +707,12 @@ int kt_bucket_pack(kt_ctx *c, const void *const *grads, const int64_t *numel, in
     if (in_dtype != KT_F32 && in_dtype != KT_BF16) return fail(KT_ERR_INVALID, "unknown in_dtype %d", in_dtype);
     if (bucket_cap_bytes < 4) return fail(KT_ERR_INVALID, "bucket_cap_bytes must be >= 4");
     const size_t es = in_dtype == KT_F32 ? 4 : 2;
+    const int n_src = n_sources(c);
+    if (flat_out && sharded(c))
+        return fail(KT_ERR_STATE, "the standalone pack is not available on a context bound to one rank");
     for (int t = 0; t < T; ++t) {
         if (numel[t] < 0) return fail(KT_ERR_INVALID, "numel[%d] is negative", t);
-        for (int r = 0; r < c->K; ++r) {
+        for (int r = 0; r < n_src; ++r) {
             const void *p = grads[static_cast<size_t>(r) * T + t];
             if (numel[t] > 0 && !p) return fail(KT_ERR_INVALID, "grads[%d][%d] is NULL", r, t);
             if (reinterpret_cast<uintptr_t>(p) % es) return fail(KT_ERR_ALIGN, "grads[%d][%d] is not element aligned", r, t);
@@ -659,16 +746,16 @@ int kt_bucket_pack(kt_ctx *c, const void *const *grads, const int64_t *numel, in
         ti.ext = end - offset[t];
         ti.flags = FLAG_ALIGNED;
         ti.pad_ = 0;
-        for (int r = 0; r < c->K; ++r)
+        for (int r = 0; r < n_src; ++r)
             if (!aligned16(grads[static_cast<size_t>(r) * T + t])) ti.flags = 0;
         const int64_t tiles = (ti.ext + tile - 1) / tile;
         if (prefix[u] + tiles > 0x7FFFFFF0LL) return fail(KT_ERR_SHAPE, "too many elements for one plan");
         prefix[u + 1] = prefix[u] + static_cast<int>(tiles);
     }
-    std::vector<const void *> ptrs(static_cast<size_t>(c->K) * T);
-    for (int k = 0; k < c->K; ++k)
+    std::vector<const void *> ptrs(static_cast<size_t>(n_src) * T);
+    for (int k = 0; k < n_src; ++k)
         for (int u = 0; u < T; ++u)
-            ptrs[static_cast<size_t>(k) * T + u] = grads[static_cast<size_t>(c->order[k]) * T + (T - 1 - u)];
+            ptrs[static_cast<size_t>(k) * T + u] = grads[static_cast<size_t>(source_of(c, k)) * T + (T - 1 - u)];
 
     // ---- upload (one allocation, three 256-byte aligned regions)
     KT_ON_DEVICE(c->device);
@@ -711,7 +798,7 @@ int kt_bucket_pack(kt_ctx *c, const void *const *grads, const int64_t *numel, in
     c->prefix = prefix;
     c->info = info;
     c->planned = true;
-    c->h_ptrs.assign(grads, grads + static_cast<size_t>(c->K) * T);
+    c->h_ptrs.assign(grads, grads + static_cast<size_t>(n_src) * T);
     forget_out_sets(c);
     for (int dir = 0; dir < 2; ++dir) {
         for (auto &s : c->slots[dir]) s.recorded = false;
@@ -776,10 +863,90 @@ int kt_plan_query(const kt_ctx *c, int32_t *n_buckets, int64_t *bucket_start, in
     return KT_OK;
 }
 
+int kt_work_unit(int in_dtype) {
+    if (in_dtype == KT_F32) return TILE_F32;
+    if (in_dtype == KT_BF16) return TILE_BF16;
+    return fail(KT_ERR_INVALID, "unknown dtype %d", in_dtype);
+}
+
+int kt_shard_ranges(const int64_t *numel, int T, int64_t bucket_cap_bytes, int64_t unit, int bucket, int n_members,
+                    int64_t *lo_out, int64_t *n_out) {
+    if (!numel || !lo_out || !n_out) return fail(KT_ERR_INVALID, "NULL argument");
+    if (T < 1) return fail(KT_ERR_INVALID, "T = %d must be >= 1", T);
+    if (bucket_cap_bytes < 4) return fail(KT_ERR_INVALID, "bucket_cap_bytes must be >= 4");
+    if (unit < 1) return fail(KT_ERR_INVALID, "unit must be >= 1");
+    if (n_members < 1 || n_members > KT_MAX_RANKS) return fail(KT_ERR_INVALID, "n_members = %d outside [1, %d]", n_members, KT_MAX_RANKS);
+    for (int t = 0; t < T; ++t)
+        if (numel[t] < 0) return fail(KT_ERR_INVALID, "numel[%d] is negative", t);
+    BucketPlan bp;
+    plan_buckets(numel, T, bucket_cap_bytes, &bp);
+    const int nb = static_cast<int>(bp.start.size());
+    if (bucket < -1 || bucket >= nb) return fail(KT_ERR_SHAPE, "bucket %d out of range [-1, %d)", bucket, nb);
+    // units before every tensor of the range, transport order (u = T - 1 - t)
+    const int u_lo = bucket < 0 ? 0 : bp.u_lo[bucket], u_hi = bucket < 0 ? T : bp.u_hi[bucket];
+    std::vector<int64_t> before(u_hi - u_lo + 1, 0), start(u_hi - u_lo + 1, 0);
+    for (int u = u_lo; u < u_hi; ++u) {
+        const int64_t at = bp.offset[T - 1 - u];
+        const int64_t end = u + 1 < T ? bp.offset[T - 2 - u] : bp.total;
+        start[u - u_lo] = at;
+        before[u - u_lo + 1] = before[u - u_lo] + (end - at + unit - 1) / unit;
+    }
+    const int64_t range_end = u_hi < T ? bp.offset[T - 1 - u_hi] : bp.total;
+    start[u_hi - u_lo] = range_end;
+    const int64_t U = before[u_hi - u_lo];
+    auto element_of = [&](int64_t index) {          // first element of unit `index` of the range
+        const int64_t k = std::upper_bound(before.begin(), before.end(), index) - before.begin() - 1;
+        if (k >= u_hi - u_lo) return range_end;
+        return start[k] + (index - before[k]) * unit;
+    };
+    for (int m = 0; m < n_members; ++m) {
+        int64_t first, past;
+        member_units(U, m, n_members, &first, &past);
+        lo_out[m] = element_of(first);
+        n_out[m] = element_of(past) - lo_out[m];
+    }
+    return KT_OK;
+}
+
+int kt_shard_bind(kt_ctx *c, int rank) {
+    if (int rc = check_ctx(c, false)) return rc;
+    if (rank < 0 || rank >= c->K) return fail(KT_ERR_INVALID, "rank = %d outside [0, %d)", rank, c->K);
+    c->shard_rank = rank;
+    c->shard_g = c->group_of[rank];
+    c->shard_M = 0;
+    for (int r = 0; r < c->K; ++r) {
+        if (c->group_of[r] != c->shard_g) continue;
+        if (r == rank) c->shard_member = c->shard_M;
+        c->shard_M += 1;
+    }
+    refresh_shard(c);
+    c->planned = false;          // the pointer table of an earlier plan had other rows
+    return KT_OK;
+}
+
+int kt_shard_query(const kt_ctx *c, int bucket, int member, int *n_members, int64_t *lo, int64_t *n) {
+    if (int rc = check_ctx(c, true)) return rc;
+    if (!sharded(c)) return fail(KT_ERR_STATE, "kt_shard_bind has not been called on this context");
+    if (bucket < -1 || bucket >= static_cast<int>(c->bucket_start.size()))
+        return fail(KT_ERR_SHAPE, "bucket %d out of range [-1, %d)", bucket, (int)c->bucket_start.size());
+    if (member < -1 || member >= c->shard_M) return fail(KT_ERR_INVALID, "member = %d outside [-1, %d)", member, c->shard_M);
+    int t0, t1;
+    unit_range(c, bucket, member < 0 ? c->shard_member : member, &t0, &t1);
+    if (n_members) *n_members = c->shard_M;
+    if (lo) *lo = unit_start(c, t0);
+    if (n) *n = unit_start(c, t1) - unit_start(c, t0);
+    return KT_OK;
+}
+
 int kt_hier_reduce(kt_ctx *c, int phase, int bucket, float *const *transport, float *combined, void *stream) {
     if (int rc = check_ctx(c, true)) return rc;
     if (phase != KT_INTRA && phase != KT_INTER && phase != KT_BOTH) return fail(KT_ERR_INVALID, "unknown phase %d", phase);
-    if (int rc = check_buffers(c, transport, c->G, "transport")) return rc;
+    if (sharded(c) && phase == KT_INTRA) {       // only the own group's partial is written
+        if (!transport) return fail(KT_ERR_INVALID, "transport is NULL");
+        if (int rc = check_buffers(c, transport + c->shard_g, 1, "transport[own group]")) return rc;
+    } else if (int rc = check_buffers(c, transport, c->G, "transport")) {
+        return rc;
+    }
     if (phase & KT_INTER) {
         if (!combined) return fail(KT_ERR_INVALID, "combined is NULL");
         if (!aligned16(combined)) return fail(KT_ERR_ALIGN, "combined is not 16-byte aligned");
@@ -793,9 +960,9 @@ int kt_hier_reduce(kt_ctx *c, int phase, int bucket, float *const *transport, fl
         K1Params p{};
         p.tp = tp;
         p.ptrs = c->d_ptrs;
-        p.rt = c->rt;
+        p.rt = reduce_table(c);
         for (int g = 0; g < c->G; ++g) p.transport[g] = transport[g];
-        p.wide = all_aligned32(transport, c->G);
+        p.wide = sharded(c) ? all_aligned32(transport + c->shard_g, 1) : all_aligned32(transport, c->G);
         const int rc = c->in_dtype == KT_F32 ? launch_k1<float>(c, p, s) : launch_k1<unsigned short>(c, p, s);
         if (rc) return rc;
     }
@@ -825,8 +992,10 @@ int kt_stage_to_host(kt_ctx *c, int dir, int bucket, float *const *transport, fl
     if (!transport || !host_pinned) return fail(KT_ERR_INVALID, "NULL argument");
     if (bucket < -1 || bucket >= static_cast<int>(c->bucket_start.size()))
         return fail(KT_ERR_SHAPE, "bucket %d out of range", bucket);
+    // bound to one rank: the own group's partial goes down, the other groups' partials come up
+    auto takes_part = [c, dir](int g) { return !sharded(c) || (dir == KT_D2H) == (g == c->shard_g); };
     for (int g = 0; g < c->G; ++g)
-        if (!transport[g] || !host_pinned[g]) return fail(KT_ERR_INVALID, "buffer %d is NULL", g);
+        if (takes_part(g) && (!transport[g] || !host_pinned[g])) return fail(KT_ERR_INVALID, "buffer %d is NULL", g);
     int64_t lo, n;
     bucket_range(c, bucket, &lo, &n);
     KT_ON_DEVICE(c->device);
@@ -844,6 +1013,7 @@ int kt_stage_to_host(kt_ctx *c, int dir, int bucket, float *const *transport, fl
     }
     const size_t es = transport_elem_size(c);
     for (int g = 0; g < c->G && n > 0; ++g) {
+        if (!takes_part(g)) continue;
         char *dev = reinterpret_cast<char *>(transport[g]) + lo * es, *host = reinterpret_cast<char *>(host_pinned[g]) + lo * es;
         if (dir == KT_D2H)
             KT_CUDA(cudaMemcpyAsync(host, dev, n * es, cudaMemcpyDeviceToHost, ss));
@@ -865,6 +1035,9 @@ int kt_relay_through_host(kt_ctx *c, int bucket, float *const *send, float *cons
         return fail(KT_ERR_SHAPE, "bucket %d out of range", bucket);
     if (chunk_bytes < 256) return fail(KT_ERR_INVALID, "chunk_bytes must be >= 256");
     if (d2h_stream == h2d_stream) return fail(KT_ERR_INVALID, "the two copy streams must differ");
+    if (sharded(c))
+        return fail(KT_ERR_STATE, "bound to one rank, the way up reads what other processes copied down: use "
+                                  "kt_stage_to_host per direction with a barrier between them");
     for (int g = 0; g < c->G; ++g)
         if (!send[g] || !host_pinned[g] || !recv[g]) return fail(KT_ERR_INVALID, "buffer %d is NULL", g);
     int64_t lo, n;
@@ -985,6 +1158,9 @@ int kt_unpack_scale(kt_ctx *c, const float *const *src, int from_combined, void 
 
 int kt_sync_direct(kt_ctx *c, void *const *out_grads, int R, int out_dtype, float scale, int bucket, void *stream) {
     if (int rc = check_ctx(c, true)) return rc;
+    if (sharded(c) && c->G > 1)
+        return fail(KT_ERR_STATE, "bound to one rank, the one-pass route needs all ranks in one group (this context "
+                                  "reads its own group's gradients only)");
     if (int rc = check_out_args(c, out_grads, R, out_dtype)) return rc;
     TilePlan tp{};
     if (int rc = make_tile_plan(c, bucket, &tp)) return rc;
@@ -999,7 +1175,7 @@ int kt_sync_direct(kt_ctx *c, void *const *out_grads, int R, int out_dtype, floa
     DirectParams p{};
     p.tp = tp;
     p.ptrs = c->d_ptrs;
-    p.rt = c->rt;
+    p.rt = reduce_table(c);
     p.gt = c->gt;
     p.out_ptrs = static_cast<void *const *>(set->dev);
     p.out_aligned = static_cast<const unsigned char *>(set->dev) + sz_ptrs;
@@ -1011,7 +1187,7 @@ int kt_sync_direct(kt_ctx *c, void *const *out_grads, int R, int out_dtype, floa
     if (c->in_dtype == out_dtype)
         for (int cpy = 0; cpy < R && !inplace; ++cpy)
             for (int t = 0; t < c->T && !inplace; ++t)
-                for (int r = 0; r < c->K && !inplace; ++r)
+                for (int r = 0; r < n_sources(c) && !inplace; ++r)
                     inplace = c->numel[t] > 0 && out_grads[static_cast<size_t>(cpy) * c->T + t] ==
                                                      c->h_ptrs[static_cast<size_t>(r) * c->T + t];
     const bool in32 = c->in_dtype == KT_F32, out32 = out_dtype == KT_F32;
@@ -1037,6 +1213,9 @@ int kt_allreduce(kt_ctx *c, float *const *transport, float *const *host_pinned, 
                  void *d2h_stream, void *h2d_stream) {
     if (int rc = check_ctx(c, true)) return rc;
     if (c->G == 1) return kt_sync_direct(c, out_grads, R, out_dtype, scale, -1, main_stream);
+    if (sharded(c))
+        return fail(KT_ERR_STATE, "bound to one rank, a collective that spans groups needs barriers between "
+                                  "processes: call its parts (kt_hier_reduce, kt_stage_to_host, kt_unpack_scale)");
     if (int rc = check_out_args(c, out_grads, R, out_dtype)) return rc;      // fail before anything is queued
     if (int rc = kt_hier_reduce(c, KT_INTRA, -1, transport, nullptr, main_stream)) return rc;
     if (int rc = kt_relay_through_host(c, -1, transport, host_pinned, recv, chunk_bytes, main_stream, d2h_stream,
@@ -1086,6 +1265,94 @@ int kt_copy_tensors(void *const *dst, const void *const *src, const int64_t *byt
     // which a single copy must not span
     for (int i = 0; i < n; ++i)
         if (bytes[i] > 0) KT_CUDA(cudaMemcpyAsync(dst[i], src[i], static_cast<size_t>(bytes[i]), kind, s));
+    return KT_OK;
+}
+
+// ---- memory shared between the processes of one node
+namespace {
+struct IpcEntry {
+    unsigned char handle[KT_IPC_HANDLE_BYTES];
+    int device;
+    void *base;
+    int refs;
+};
+std::mutex g_ipc_mutex;
+std::vector<IpcEntry> g_ipc_open;      // every handle is opened once per process and device, then counted
+}  // namespace
+
+int kt_ipc_export(const void *dev_ptr, void *handle_out, int64_t *offset_out) {
+    if (!dev_ptr || !handle_out || !offset_out) return fail(KT_ERR_INVALID, "NULL argument");
+    static_assert(sizeof(cudaIpcMemHandle_t) == KT_IPC_HANDLE_BYTES, "handle size");
+    // the handle names the whole allocation; where inside it the pointer lies is asked of the driver
+    typedef int (*range_fn)(unsigned long long *, size_t *, unsigned long long);
+    void *fn = nullptr;
+    cudaDriverEntryPointQueryResult found;
+    KT_CUDA(cudaGetDriverEntryPoint("cuMemGetAddressRange", &fn, cudaEnableDefault, &found));
+    if (!fn || found != cudaDriverEntryPointSuccess) return fail(KT_ERR_CUDA, "the driver does not offer cuMemGetAddressRange");
+    unsigned long long base = 0;
+    size_t size = 0;
+    const int drc = reinterpret_cast<range_fn>(fn)(&base, &size, static_cast<unsigned long long>(reinterpret_cast<uintptr_t>(dev_ptr)));
+    if (drc != 0) return fail(KT_ERR_CUDA, "cuMemGetAddressRange failed with driver status %d (not a device allocation?)", drc);
+    cudaIpcMemHandle_t h;
+    KT_CUDA(cudaIpcGetMemHandle(&h, reinterpret_cast<void *>(static_cast<uintptr_t>(base))));
+    std::memcpy(handle_out, &h, sizeof(h));
+    *offset_out = static_cast<int64_t>(reinterpret_cast<uintptr_t>(dev_ptr) - base);
+    return KT_OK;
+}
+
+int kt_ipc_open(const void *handle, int64_t offset, void **dev_ptr_out) {
+    if (!handle || !dev_ptr_out) return fail(KT_ERR_INVALID, "NULL argument");
+    if (offset < 0) return fail(KT_ERR_INVALID, "offset is negative");
+    int dev = 0;
+    KT_CUDA(cudaGetDevice(&dev));
+    std::lock_guard<std::mutex> lock(g_ipc_mutex);
+    for (IpcEntry &e : g_ipc_open)
+        if (e.device == dev && std::memcmp(e.handle, handle, KT_IPC_HANDLE_BYTES) == 0) {
+            e.refs += 1;
+            *dev_ptr_out = static_cast<char *>(e.base) + offset;
+            return KT_OK;
+        }
+    cudaIpcMemHandle_t h;
+    std::memcpy(&h, handle, sizeof(h));
+    void *base = nullptr;
+    KT_CUDA(cudaIpcOpenMemHandle(&base, h, cudaIpcMemLazyEnablePeerAccess));
+    IpcEntry e;
+    std::memcpy(e.handle, handle, KT_IPC_HANDLE_BYTES);
+    e.device = dev;
+    e.base = base;
+    e.refs = 1;
+    g_ipc_open.push_back(e);
+    *dev_ptr_out = static_cast<char *>(base) + offset;
+    return KT_OK;
+}
+
+int kt_ipc_close(const void *handle) {
+    if (!handle) return fail(KT_ERR_INVALID, "NULL argument");
+    int dev = 0;
+    KT_CUDA(cudaGetDevice(&dev));
+    std::lock_guard<std::mutex> lock(g_ipc_mutex);
+    for (size_t i = 0; i < g_ipc_open.size(); ++i) {
+        IpcEntry &e = g_ipc_open[i];
+        if (e.device != dev || std::memcmp(e.handle, handle, KT_IPC_HANDLE_BYTES) != 0) continue;
+        if (--e.refs == 0) {
+            void *base = e.base;
+            g_ipc_open.erase(g_ipc_open.begin() + static_cast<long>(i));
+            KT_CUDA(cudaIpcCloseMemHandle(base));
+        }
+        return KT_OK;
+    }
+    return fail(KT_ERR_STATE, "this handle is not open on device %d", dev);
+}
+
+int kt_host_register(void *host, int64_t bytes) {
+    if (!host || bytes < 1) return fail(KT_ERR_INVALID, "bad host range");
+    KT_CUDA(cudaHostRegister(host, static_cast<size_t>(bytes), cudaHostRegisterPortable));
+    return KT_OK;
+}
+
+int kt_host_unregister(void *host) {
+    if (!host) return fail(KT_ERR_INVALID, "NULL argument");
+    KT_CUDA(cudaHostUnregister(host));
     return KT_OK;
 }
 
@@ -1313,6 +1580,7 @@ int kt_sampler_indices(const int64_t *list, int64_t dataset_size, const int32_t 
 namespace {
 
 int fill_bcast(const kt_ctx *c, int root, BcastParams *p) {
+    if (sharded(c)) return fail(KT_ERR_STATE, "the broadcast is not available on a context bound to one rank");
     if (root < 0 || root >= c->K) return fail(KT_ERR_INVALID, "root = %d outside [0, %d)", root, c->K);
     p->ptrs = const_cast<void *const *>(reinterpret_cast<const void *const *>(c->d_ptrs));
     p->G = c->G;
@@ -1375,6 +1643,7 @@ int kt_bcast_relay(kt_ctx *c, int root, int bucket, const void *send, void *host
                    int64_t chunk_bytes, void *main_stream, void *d2h_stream, void *h2d_stream) {
     if (int rc = check_ctx(c, true)) return rc;
     if (!send || !host_pinned || !recv) return fail(KT_ERR_INVALID, "NULL argument");
+    if (sharded(c)) return fail(KT_ERR_STATE, "the broadcast is not available on a context bound to one rank");
     if (root < 0 || root >= c->K) return fail(KT_ERR_INVALID, "root = %d outside [0, %d)", root, c->K);
     if (bucket < -1 || bucket >= static_cast<int>(c->bucket_start.size()))
         return fail(KT_ERR_SHAPE, "bucket %d out of range", bucket);

@@ -73,8 +73,9 @@ struct TilePlan {         // which tiles a launch covers and how to decode them
     int tile_lo;          // prefix[u_lo]
     int n_tiles;          // prefix[u_hi] - prefix[u_lo]
     int tile;             // elements per tile the prefix was built for
-    int single;           // the launch covers exactly one tensor: its record travels in `one`
+    int single;           // the launch covers (part of) exactly one tensor: its record travels in `one`
     TInfo one;            // ... and the fused reduce decodes its tiles by arithmetic, without any table
+    int single_skip;      // ... starting this many tiles into the tensor (a device's share may begin mid-tensor)
     const void *tables;   // start of the table allocation (prefix, records, pointers) ...
     int table_bytes;      // ... and how much of it is worth prefetching (0: nothing)
 };
@@ -300,7 +301,7 @@ __device__ __forceinline__ TileRef locate_tile(const TilePlan &tp) {
         TileRef r;
         r.u = tp.u_lo;
         r.ti = tp.one;
-        r.e0 = static_cast<long long>(blockIdx.x) * tp.tile;
+        r.e0 = static_cast<long long>(blockIdx.x + tp.single_skip) * tp.tile;
         return r;
     }
     __shared__ int s_u;

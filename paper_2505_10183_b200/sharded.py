@@ -1,0 +1,168 @@
+"""One rank per device: the multi-process plumbing around the library's sharded calls.
+
+Every rank is a process with a device of its own (paper Section III-A: the devices of a group
+run their collective among themselves; groups exchange through host memory).  This module
+holds no arithmetic.  It moves handles and names between the processes with
+``torch.distributed`` (object collectives and barriers on a host-side process group), maps the
+group mates' gradient and output tensors into this process (``kt_ipc_open``), maps one block of
+host memory that all processes of the node share (POSIX shared memory, page-locked with
+``kt_host_register``), and then issues the library calls of a step in order:
+
+    barrier                         every rank's gradients are complete
+    kt_hier_reduce(KT_INTRA)        my share of each bucket, read from all members of my group
+    kt_stage_to_host(KT_D2H)        my share of my group's partial -> shared host memory
+    wait for my copies, barrier     every share of every group is in host memory
+    kt_stage_to_host(KT_H2D)        my element range of the other groups' partials -> device
+    kt_unpack_scale                 combine, scale, cast; my share written into the output
+                                    tensors of every member of my group
+    wait for my kernels, barrier    every rank holds the whole reduced gradient
+
+With a single group the middle collapses to one kt_sync_direct call.  Ranks wait for one
+another on the host only; no kernel waits for another device.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import mmap
+import os
+import secrets
+from typing import List, Optional, Sequence
+
+import torch
+import torch.distributed as dist
+
+from . import binding as kt
+
+
+class ShardedSync:
+    def __init__(self, rank: int, group_of: Sequence[int], shares: Sequence[int], grads: Sequence[torch.Tensor],
+                 outs: Optional[Sequence[torch.Tensor]] = None, bucket_cap_bytes: int = 25 << 20,
+                 host_group=None, per_bucket: bool = True, wait_ms: int = 60000):
+        """grads: this rank's gradient tensors (device, contiguous, one dtype); outs: where this
+        rank wants the reduced gradients (None: in place, over `grads`); host_group: a
+        torch.distributed group whose collectives run on the host (gloo) and whose ranks are
+        numbered like `group_of`."""
+        self.rank, self.group_of, self.K = rank, list(group_of), len(group_of)
+        self.G = max(group_of) + 1
+        self.g = group_of[rank]
+        self.members = [r for r in range(self.K) if group_of[r] == self.g]
+        self.member = self.members.index(rank)
+        self.host_group = host_group
+        self.wait_ms = wait_ms
+        outs = list(grads) if outs is None else list(outs)
+        self.grads, self.outs = list(grads), outs
+        self.numel = [int(t.numel()) for t in grads]
+        T = len(self.numel)
+        if any(o.numel() != n or not o.is_contiguous() for o, n in zip(outs, self.numel)) or len(outs) != T:
+            raise kt.KtError(kt.KT_ERR_SHAPE, "outs must match grads in count and sizes")
+        self.in_dtype = kt._DTYPES[grads[0].dtype]
+        self.out_dtype = kt._DTYPES[outs[0].dtype]
+
+        # 1. every rank tells every other how its tensors can be reached
+        mine = {"grads": [kt.kt_ipc_export(t.data_ptr()) if t.numel() else (b"", 0) for t in grads],
+                "outs": [kt.kt_ipc_export(t.data_ptr()) if t.numel() else (b"", 0) for t in outs],
+                "numel": self.numel}
+        everyone: List[Optional[dict]] = [None] * self.K
+        dist.all_gather_object(everyone, mine, group=host_group)
+        self._opened: List[bytes] = []
+
+        def address(r: int, kind: str, t: int) -> int:
+            if r == rank:
+                return (grads if kind == "grads" else outs)[t].data_ptr()
+            handle, offset = everyone[r][kind][t]
+            if not handle:
+                return 0
+            self._opened.append(handle)
+            return kt.kt_ipc_open(handle, offset)
+
+        for r in self.members:
+            if everyone[r]["numel"] != self.numel:
+                raise kt.KtError(kt.KT_ERR_SHAPE, "rank %d holds other tensor sizes than rank %d" % (r, rank))
+        grad_ptrs = [address(r, "grads", t) for r in self.members for t in range(T)]
+        out_ptrs = [address(r, "outs", t) for r in self.members for t in range(T)]
+
+        # 2. the context of this rank
+        self.ctx = kt.kt_groups_init(self.group_of, list(shares), self.G)
+        kt.kt_shard_bind(self.ctx, rank, self.group_of)
+        kt.kt_bucket_pack_ptrs(self.ctx, kt.PtrArray.from_addresses(grad_ptrs, keep=self.grads), self.numel,
+                               self.in_dtype, bucket_cap_bytes)
+        self.plan = kt.kt_plan_query(self.ctx)
+        self.buckets = list(range(self.plan.n_buckets)) if per_bucket else [-1]
+        self.out_ptrs = kt.PtrArray.from_addresses(out_ptrs, keep=self.outs)
+        n = self.plan.transport_numel
+        # row g: my share of my group's partial; rows h != g: the other groups' partials over my range
+        self.partials = torch.zeros(self.G, max(n, 1), dtype=torch.float32, device=grads[0].device)
+        self.partial_rows = kt.kt_ptrs(list(self.partials))
+        self.main = torch.cuda.Stream()
+        self.side = torch.cuda.Stream()
+
+        # 3. host memory that all processes share: the G partials, end to end, in a file of the
+        #    node's shared-memory file system that every rank maps and page-locks
+        self.host_rows = None
+        self._map = None
+        if self.G > 1:
+            nbytes = self.G * max(n, 1) * 4
+            name = [None]
+            if rank == 0:
+                name[0] = "/dev/shm/kt_partials_%d_%s" % (os.getpid(), secrets.token_hex(4))
+                fd = os.open(name[0], os.O_CREAT | os.O_EXCL | os.O_RDWR, 0o600)
+                os.ftruncate(fd, nbytes)
+            dist.broadcast_object_list(name, src=0, group=host_group)
+            if rank != 0:
+                fd = os.open(name[0], os.O_RDWR)
+            self._shm_name = name[0]
+            self._map = mmap.mmap(fd, nbytes)
+            os.close(fd)
+            self._view = C.c_char.from_buffer(self._map)
+            self._host_address = C.addressof(self._view)
+            kt.kt_host_register(self._host_address, nbytes)
+            self.host_rows = kt.PtrArray.from_addresses([self._host_address + g * max(n, 1) * 4 for g in range(self.G)],
+                                                        keep=self._map)
+            dist.barrier(group=host_group)
+            if rank == 0:
+                os.unlink(name[0])                    # every rank has it mapped: the name can go
+
+    def my_range(self, bucket: int = -1):
+        return kt.kt_shard_query(self.ctx, bucket)[:2]
+
+    def step(self, scale: float = 1.0) -> None:
+        """One synchronisation.  On return this rank's `outs` hold the reduced gradients and every
+        other rank has finished reading this rank's `grads`."""
+        ctx = self.ctx
+        torch.cuda.synchronize()                      # whatever produced my gradients is done
+        dist.barrier(group=self.host_group)
+        if self.G == 1:
+            for b in self.buckets:
+                kt.kt_sync_direct(ctx, self.out_ptrs, scale=scale, bucket=b, out_dtype=self.out_dtype,
+                                  R=len(self.members), stream=self.main)
+        else:
+            for b in self.buckets:
+                kt.kt_hier_reduce(ctx, kt.KT_INTRA, self.partial_rows, bucket=b, stream=self.main)
+                kt.kt_stage_to_host(ctx, kt.KT_D2H, self.partial_rows, self.host_rows, bucket=b,
+                                    main_stream=self.main, side_stream=self.side)
+            for b in self.buckets:                    # my shares are in host memory ...
+                kt.kt_stage_wait(ctx, kt.KT_D2H, bucket=b, main_stream=self.main, timeout_ms=self.wait_ms)
+            dist.barrier(group=self.host_group)       # ... and so are everybody else's
+            for b in self.buckets:
+                kt.kt_stage_to_host(ctx, kt.KT_H2D, self.partial_rows, self.host_rows, bucket=b,
+                                    main_stream=self.main, side_stream=self.side)
+            for b in self.buckets:
+                kt.kt_stage_wait(ctx, kt.KT_H2D, bucket=b, main_stream=self.main)
+                kt.kt_unpack_scale(ctx, self.partial_rows, self.out_ptrs, scale=scale, bucket=b,
+                                   out_dtype=self.out_dtype, R=len(self.members), stream=self.main)
+        self.main.synchronize()                       # my shares are written everywhere in my group
+        dist.barrier(group=self.host_group)
+
+    def close(self) -> None:
+        torch.cuda.synchronize()
+        dist.barrier(group=self.host_group)           # nobody still reads what is unmapped next
+        kt.kt_destroy(self.ctx)
+        for handle in self._opened:
+            kt.kt_ipc_close(handle)
+        self._opened = []
+        if self._map is not None:
+            kt.kt_host_unregister(self._host_address)
+            self.host_rows = None
+            del self._view
+            self._map.close()
+            self._map = None

@@ -140,3 +140,23 @@ int main(void) {
     subprocess.check_call(["gcc", "-std=c99", "-I", inc, str(src), "-o", str(exe), build.LIB, "-lm", "-ldl", "-lpthread", "-lrt",
                            "-lstdc++", "-Wl,-rpath," + os.path.dirname(build.LIB)])
     assert subprocess.check_output([str(exe)]).decode().strip() == "ok"
+
+
+def test_shard_ranges_match_the_oracle(kt, oracle):
+    """One rank per device: the element ranges the library hands to the members of a group are
+    the oracle's, on random lists, caps, units and member counts; pure host functions."""
+    import random
+    rnd = random.Random(1)
+    sizes = [0, 1, 7, 8, 9, 63, 64, 65, 500, 2047, 2048, 2049, 4096, 5000, 10000, 40000]
+    assert kt.kt_work_unit(kt.KT_F32) == 2048 and kt.kt_work_unit(kt.KT_BF16) == 4096
+    for _ in range(400):
+        numel = [rnd.choice(sizes) for _ in range(rnd.randint(1, 12))]
+        cap, unit, M = rnd.choice([64, 4096, 40000, 1 << 20, 1 << 40]), rnd.choice([2048, 4096, 64]), rnd.randint(1, 9)
+        nb = kt.kt_plan_buckets(numel, cap).n_buckets
+        for b in [-1] + list(range(nb)):
+            assert kt.kt_shard_ranges(numel, cap, unit, b, M) == oracle.shard_ranges(numel, cap, unit, b, M)
+    for bad in (([5], 1 << 20, 0, -1, 2), ([5], 1 << 20, 2048, 1, 2), ([5], 1 << 20, 2048, -1, 0), ([-1], 1 << 20, 2048, -1, 1)):
+        with pytest.raises(kt.KtError):
+            kt.kt_shard_ranges(*bad)
+    with pytest.raises(kt.KtError):
+        kt.kt_work_unit(7)
