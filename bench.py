@@ -695,6 +695,76 @@ def run_e2e(prob, kt, args, barrier) -> dict:
     return {"seconds": a.elapsed_time(b) * 1e-3, "h2d": arm.h2d_bytes, "d2h": arm.d2h_bytes}
 
 
+# ----------------------------------------------------------------------------- one rank per GPU
+def sharded_workload(name: str, world: int):
+    """The named tensor list with one rank per GPU: the first half of the ranks is one vendor
+    group, the second half a slower one (step times 1.0 and 1.6, global batch 256)."""
+    base = W.by_name(name)
+    first = max(1, world // 2)
+    group_of = [0] * first + [1] * (world - first)
+    times = [1.0] * first + [1.6] * (world - first)
+    return W.Workload(base.name + "_sharded", base.config_id, base.shapes, base.dtype, group_of, None,
+                      step_times=times, global_batch=256, bucket_cap_bytes=base.bucket_cap_bytes, staged=world > first)
+
+
+def run_sharded(args) -> dict:
+    """`--sharded`: every GPU is one rank and reduces its share of every bucket from its group
+    mates' gradients (peer-mapped), relays only that share through host memory, and writes its
+    share of the result into every group mate's tensors.  Timed on the device (events on the
+    rank's stream around the K steps, host barriers included), maximum over ranks."""
+    from paper_2505_10183_b200 import binding as kt
+    from paper_2505_10183_b200.sharded import ShardedSync
+    import torch.distributed as dist
+    world, rank, local, started = init_ranks("nccl")
+    torch.cuda.set_device(local)
+    if started is None:
+        dist.init_process_group("gloo", rank=0, world_size=1, init_method="tcp://127.0.0.1:%d" % free_port())
+        host_group = None
+    else:
+        host_group = dist.new_group(backend="gloo")        # barriers and object exchange stay on the host
+    wl = sharded_workload(args.workload, world)
+    shares = kt.kt_schedule(wl.step_times, wl.global_batch)
+    dt = torch.float32 if wl.dtype == "f32" else torch.bfloat16
+    grads = [t.cuda() for t in W.split_tensors(W.rank_gradients(wl, rank, "cuda"), wl.numel)]
+    outs = [torch.zeros(m, dtype=dt, device="cuda") for m in wl.numel]
+    job = ShardedSync(rank, wl.group_of, shares, grads, outs, wl.bucket_cap_bytes, host_group=host_group)
+    M, G, s = len(job.members), wl.G, wl.elem_size
+    mine = sum(kt.kt_shard_query(job.ctx, b)[1] for b in job.buckets)          # transport elements of my shares
+    if G == 1:
+        my_bytes = M * mine * s + M * mine * s
+    else:
+        my_bytes = (M * mine * s + 4 * mine) + (4 * G * mine + M * mine * s)
+    for _ in range(args.warmup):
+        job.step()
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record(job.main)
+    for _ in range(args.steps):
+        job.step()
+    b.record(job.main)
+    torch.cuda.synchronize()
+    t = torch.tensor([a.elapsed_time(b) * 1e-3, 0.0], dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX, group=host_group)
+    total = torch.tensor([float(my_bytes)], dtype=torch.float64)
+    dist.all_reduce(total, op=dist.ReduceOp.SUM, group=host_group)
+    seconds = float(t[0])
+    if not all(bool(torch.isfinite(o).all()) and bool(o.any()) for o in outs if o.numel() > 64):
+        raise RuntimeError("sharded arm: an output tensor was not written")
+    job.close()
+    dist.destroy_process_group()
+    if rank != 0:
+        return None
+    return {"metric": METRIC, "arm": "sharded", "value": round(float(total[0]) * args.steps / seconds / 1e9, 2),
+            "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": round(seconds / args.steps * 1e3, 4), "higher_is_better": True, "scaling": "strong",
+            "vs_baseline": None, "dtype": wl.dtype, "data": "synthetic",
+            "config": {"workload": "%s: %d tensors, %d elements per rank, one rank per GPU, groups %s, shares %s"
+                                   % (wl.name, wl.T, wl.N, wl.group_of, shares),
+                       "bytes_counted": "per GPU: M*n*s read + 4*n written by the fused reduce over its share of n "
+                                        "elements, 4*G*n read + M*n*s written by combine+unpack (M group members); "
+                                        "summed over GPUs",
+                       "host_barriers_per_step": 3, "note": "timing includes the host-side barriers between ranks"}}
+
+
 # ----------------------------------------------------------------------------- the oracle as CPU baseline
 def oracle_inputs(wl):
     host = []
@@ -837,6 +907,8 @@ def main() -> None:
     ap.add_argument("--no-large-bucket", action="store_true")
     ap.add_argument("--cpu-seconds", type=float, default=12.0)
     ap.add_argument("--relay-chunk-mib", type=int, default=4)
+    ap.add_argument("--sharded", action="store_true",
+                    help="one rank per GPU with element-range shares instead of independent replicas")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.sweep:
@@ -850,7 +922,10 @@ def main() -> None:
     if args.impl == "ours" and env_world is None and args.gpus > 1:
         # not started by a launcher: start the N ranks here, one process per GPU
         sys.exit(launch_ranks(args.gpus, os.path.abspath(__file__), sys.argv[1:]).returncode)
-    out = run_reference(args) if args.impl == "reference" else run_ours(args)
+    if args.sharded and args.impl == "ours":
+        out = run_sharded(args)
+    else:
+        out = run_reference(args) if args.impl == "reference" else run_ours(args)
     if out is not None:
         print(json.dumps(out), flush=True)
 
