@@ -459,8 +459,10 @@ __device__ __forceinline__ void k2_tile(const K2Params &p, const TileRef &t) {
     }
 }
 
+// Five resident CTAs per SM (48 registers): measured 1.5-2.5 % faster than the compiler's own
+// choice of 54-64 registers on fp32 outputs, equal on bf16 outputs; six (40 registers) lost.
 template <typename Tout, typename TT, int TILE>
-__global__ void __launch_bounds__(NT) k2_combine_unpack(const __grid_constant__ K2Params p) {
+__global__ void __launch_bounds__(NT, 5) k2_combine_unpack(const __grid_constant__ K2Params p) {
     const TileRef t = locate_tile(p.tp);
     if (p.out_aligned[t.u] && t.e0 + TILE <= t.ti.numel)
         k2_tile<Tout, TT, TILE, false>(p, t);
