@@ -217,17 +217,34 @@ class Problem:
         return sum(a.elapsed_time(b) for a, b in self.k2_events) * 1e-3
 
 
-def host_link_bandwidth(nbytes: int = 256 << 20, reps: int = 10) -> dict:
-    """Pinned cudaMemcpyAsync, best of `reps` (GB/s): each direction alone, and both
-    directions at the same time on two streams (per direction; what a relay whose way down
-    and way up overlap can reach at most)."""
+def host_link_bandwidth(nbytes: int = 256 << 20, reps: int = 10, chunk_bytes: int = 4 << 20) -> dict:
+    """Pinned cudaMemcpyAsync, best of `reps` (GB/s): each direction alone; both directions at
+    the same time on two streams, as one copy each ("both") and cut into independent copies of
+    chunk_bytes ("both_chunked": per direction, what a relay that must work in chunks of that
+    size can reach at most, before the lag of its pipeline)."""
     dev = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
     host = torch.empty(nbytes, dtype=torch.uint8).pin_memory()
     dev2 = torch.empty(nbytes, dtype=torch.uint8, device="cuda")
     host2 = torch.empty(nbytes, dtype=torch.uint8).pin_memory()
-    best = {"d2h": 0.0, "h2d": 0.0, "both": 0.0}
+    best = {"d2h": 0.0, "h2d": 0.0, "both": 0.0, "both_chunked": 0.0}
     s1, s2 = torch.cuda.Stream(), torch.cuda.Stream()
+    cuts = [(lo, min(nbytes, lo + chunk_bytes)) for lo in range(0, nbytes, chunk_bytes)]
     for _ in range(reps):
+        torch.cuda.synchronize()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        s1.wait_event(a)
+        s2.wait_event(a)
+        for lo, hi in cuts:
+            with torch.cuda.stream(s1):
+                host[lo:hi].copy_(dev[lo:hi], non_blocking=True)
+            with torch.cuda.stream(s2):
+                dev2[lo:hi].copy_(host2[lo:hi], non_blocking=True)
+        torch.cuda.current_stream().wait_stream(s1)
+        torch.cuda.current_stream().wait_stream(s2)
+        b.record()
+        b.synchronize()
+        best["both_chunked"] = max(best["both_chunked"], nbytes / (a.elapsed_time(b) * 1e-3) / 1e9)
         for name, (dst, src) in (("d2h", (host, dev)), ("h2d", (dev, host))):
             a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             a.record()
@@ -252,14 +269,29 @@ def host_link_bandwidth(nbytes: int = 256 << 20, reps: int = 10) -> dict:
     return best
 
 
-def time_launches(fn, stream, reps: int) -> float:
-    """Average CUDA-event duration (s) of `reps` launches queued back to back on `stream`,
-    each bracketed by its own pair of events."""
+_FLUSH = {}
+
+
+def l2_flush(stream) -> None:
+    """Writes a buffer twice the size of the 126 MB L2 on `stream`, so that what follows finds
+    none of its data cached."""
+    buf = _FLUSH.get("buf")
+    if buf is None:
+        buf = _FLUSH["buf"] = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    with torch.cuda.stream(stream):
+        buf.fill_(1)
+
+
+def time_launches(fn, stream, reps: int, flush: bool = False) -> float:
+    """Average CUDA-event duration (s) of `reps` launches queued on `stream`, each bracketed by
+    its own pair of events; flush=True clears the L2 before every launch (outside the pair)."""
     pairs = []
     for _ in range(3):
         fn()
     torch.cuda.synchronize()
     for _ in range(reps):
+        if flush:
+            l2_flush(stream)
         a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         a.record(stream)
         fn()
@@ -269,27 +301,63 @@ def time_launches(fn, stream, reps: int) -> float:
     return sum(a.elapsed_time(b) for a, b in pairs) * 1e-3 / reps
 
 
-def large_bucket_roofline(kt, peak: float, K: int = 4, bytes_per_rank: int = 256 << 20) -> dict:
-    """The fused reduce on one flat bucket of 256 MiB per rank (the bucket size the bandwidth
-    target is stated for): algorithmic bytes over the CUDA-event time of a launch."""
-    wl = W.sweep_point(K, bytes_per_rank, "f32")
-    prob = Problem(wl, kt)
+def kernel_rows(kt, prob, peak: float, reps: int = 20, flush: bool = False) -> dict:
+    """K1, K2 and the one-pass kernel on a problem's buffers: algorithmic bytes over the
+    CUDA-event time of a launch."""
+    wl = prob.wl
     by = algorithmic_bytes(wl)
     with torch.cuda.stream(prob.main):
         k1 = time_launches(lambda: kt.kt_hier_reduce(prob.ctx, kt.KT_INTRA, prob.transport, stream=prob.main),
-                           prob.main, 20)
+                           prob.main, reps, flush)
         k2 = time_launches(lambda: kt.kt_unpack_scale(prob.ctx, prob.transport, prob.out_ptrs, out_dtype=prob.out_dtype,
-                                                      R=1, stream=prob.main), prob.main, 20)
-        direct = time_launches(prob.direct, prob.main, 20)
-    kt.kt_destroy(prob.ctx)
+                                                      R=1, stream=prob.main), prob.main, reps, flush)
+        direct = time_launches(prob.direct, prob.main, reps, flush)
     direct_bytes = wl.K * wl.N * wl.elem_size + wl.N * wl.elem_size
 
     def row(nbytes, sec):
         return {"us": round(sec * 1e6, 2), "GBps": round(nbytes / sec / 1e9, 1), "frac": round(nbytes / sec / 1e9 / peak, 4),
-                "frac_of_nominal_8TBs": round(nbytes / sec / 1e9 / NOMINAL_HBM_GBS, 4)}
-    return {"workload": "flat fp32 bucket, %d ranks x %d MiB in 2 groups" % (K, bytes_per_rank >> 20),
-            "k1_intra_reduce": row(by["k1"], k1), "k2_combine_unpack": row(by["k2"], k2),
+                "frac_of_nominal_8TBs": round(nbytes / sec / 1e9 / NOMINAL_HBM_GBS, 4), "bytes_per_launch": int(nbytes)}
+    return {"k1_intra_reduce": row(by["k1"], k1), "k2_combine_unpack": row(by["k2"], k2),
             "k_direct_sync": row(direct_bytes, direct)}
+
+
+def large_bucket_roofline(kt, peak: float, K: int = 4, bytes_per_rank: int = 256 << 20, dtype: str = "f32") -> dict:
+    """The kernels on one flat bucket per rank of the size the bandwidth target is stated for
+    (64 MiB and up): algorithmic bytes over the CUDA-event time of a launch.  The buffers
+    exceed the L2 several times over."""
+    wl = W.sweep_point(K, bytes_per_rank, dtype)
+    prob = Problem(wl, kt)
+    out = {"workload": "flat %s bucket, %d ranks x %d MiB in 2 groups" % ("fp32" if dtype == "f32" else "bf16", K,
+                                                                          bytes_per_rank >> 20)}
+    out.update(kernel_rows(kt, prob, peak))
+    kt.kt_destroy(prob.ctx)
+    del prob
+    torch.cuda.empty_cache()
+    return out
+
+
+LARGE_BUCKETS = [(8, 64 << 20, "f32"), (16, 64 << 20, "f32"), (8, 256 << 20, "f32"), (16, 256 << 20, "f32"),
+                 (8, 64 << 20, "bf16"), (16, 64 << 20, "bf16"), (8, 256 << 20, "bf16"), (16, 256 << 20, "bf16")]
+
+
+def named_config_rows(kt, peak: float) -> dict:
+    """The kernels on the other named configurations (the step itself runs on ResNet-18):
+    ResNet-50 with bf16 gradients and 8 ranks, MobileNetV2's ragged list with 8 ranks in three
+    groups.  The L2 is flushed before every timed launch."""
+    out = {"l2": "flushed before every timed launch (a 256 MiB buffer is written outside the event pair)"}
+    for name in ("resnet50", "mobilenet_v2"):
+        wl = W.by_name(name)
+        prob = Problem(wl, kt)
+        rows = kernel_rows(kt, prob, peak, flush=True)
+        rows["workload"] = "%s: %d tensors, %d elements per rank, %s, K=%d ranks in %d groups, shares %s" % (
+            wl.name, wl.T, wl.N, wl.dtype, wl.K, wl.G, prob.shares)
+        rows["k1_intra_reduce"]["traffic"] = TRAFFIC_K1.get(name)
+        rows["default_route_without_staging"] = "k_direct_sync (one pass)"
+        out[name] = rows
+        kt.kt_destroy(prob.ctx)
+        del prob
+        torch.cuda.empty_cache()
+    return out
 
 
 def broadcast_phases(kt, wl, peak: float, chunk_bytes: int) -> dict:
@@ -479,7 +547,7 @@ def run_ours(args) -> dict:
     wl = W.by_name(args.workload)
     prob = Problem(wl, kt, chunk_bytes=args_chunk(args))
     nbytes = algorithmic_bytes(wl)
-    link = host_link_bandwidth() if wl.staged else None
+    link = host_link_bandwidth(chunk_bytes=args_chunk(args)) if wl.staged else None
 
     def barrier():
         torch.cuda.synchronize()
@@ -560,7 +628,7 @@ def run_ours(args) -> dict:
                      "peak": peak, "unit": "GB/s", "frac": round(achieved / peak, 4),
                      "peak_kind": peak_kind, "frac_of_nominal_8TBs": round(achieved / NOMINAL_HBM_GBS, 4),
                      "bytes_per_launch": int(k1_launch_bytes), "us_per_launch": round(k1_launch_s * 1e6, 2),
-                     "traffic": TRAFFIC_K1.get(wl.name)},
+                     "traffic": TRAFFIC_K1.get(wl.name), "traffic_source": TRAFFIC_SOURCE},
         "e2e": {"value": round(job_throughput(nbytes["step"], args.steps, world, e2e["seconds"]), 2), "unit": UNIT,
                 "h2d_bytes_per_step": e2e["h2d"], "d2h_bytes_per_step": e2e["d2h"],
                 "ms_per_step": round(e2e["seconds"] / args.steps * 1e3, 4),
@@ -574,10 +642,17 @@ def run_ours(args) -> dict:
         result["host_link"] = {"d2h_GBps": round(link["d2h"], 1), "h2d_GBps": round(link["h2d"], 1),
                                "both_ways_at_once_GBps_each": round(link["both"], 1),
                                "relay_frac_of_both_ways": round(nbytes["stage_each_way"] / relay_s / 1e9 / link["both"], 3),
-                               "how": "pinned copy of 256 MiB, best of 10; both ways = one copy down and one "
-                                      "up on two streams at the same time"}
+                               "both_ways_in_relay_chunks_GBps_each": round(link["both_chunked"], 1),
+                               "relay_frac_of_both_ways_in_relay_chunks": round(
+                                   nbytes["stage_each_way"] / relay_s / 1e9 / link["both_chunked"], 3),
+                               "how": "pinned copies of 256 MiB, best of 10; both ways = one copy down and one up on "
+                                      "two streams at the same time; in relay chunks = the same bytes as independent "
+                                      "copies of the relay's chunk size (a relay must work in chunks: the way up of a "
+                                      "chunk starts when its way down is done)"}
     if rank == 0 and world == 1 and not args.no_large_bucket:
         result["roofline_large_bucket"] = large_bucket_roofline(kt, peak)
+        result["roofline_large_bucket"]["more"] = [large_bucket_roofline(kt, peak, K, nb, dt) for K, nb, dt in LARGE_BUCKETS]
+        result["configs"] = named_config_rows(kt, peak)
         result["broadcast"] = broadcast_phases(kt, wl, peak, args_chunk(args))
         result["bf16_transport"] = narrow_transport_step(kt, wl, args_chunk(args), min(args.steps, 20))
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
@@ -589,10 +664,11 @@ def run_ours(args) -> dict:
     return result if rank == 0 else None
 
 
-# ncu dram__bytes_read.sum + dram__bytes_write.sum per launch of the dominant kernel, captured
-# for the kernel as it stands (profiles/k1_k2_resnet18.md); a workload without a capture
-# reports null.
-TRAFFIC_K1 = {"resnet18": 216686336}
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the fused reduce on each named
+# workload, from ncu captures of the kernel as committed (not measured in this run: a run under
+# a profiler reports no times).  A workload without a capture reports null.
+TRAFFIC_K1 = {}
+TRAFFIC_SOURCE = None
 
 
 def args_chunk(args) -> int:

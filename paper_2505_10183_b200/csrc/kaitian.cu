@@ -335,9 +335,6 @@ int make_tile_plan(const kt_ctx *c, int bucket, TilePlan *tp) {
         tp->one = c->info[tp->u_lo];
         tp->single_skip = t0 - c->prefix[tp->u_lo];
     }
-    tp->tables = c->d_tables;
-    tp->table_bytes = static_cast<int>(c->d_tables_bytes < static_cast<size_t>(NT) * 128 ? c->d_tables_bytes
-                                                                                          : static_cast<size_t>(NT) * 128);
     return KT_OK;
 }
 
@@ -1829,8 +1826,6 @@ extern "C" int kt_sync_flat_static(const int32_t *group_of, const int32_t *share
     tp.tile = tile;
     tp.single = 1;
     tp.one = tab.info;
-    tp.tables = scratch;
-    tp.table_bytes = static_cast<int>(sizeof(StaticTables));
     float *partials = reinterpret_cast<float *>(scratch + STATIC_TABLE_BYTES);
     p1.tp = tp;
     p1.ptrs = reinterpret_cast<const void *const *>(scratch + offsetof(StaticTables, in_ptrs));

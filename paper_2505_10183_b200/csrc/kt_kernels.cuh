@@ -33,9 +33,6 @@ namespace {
 #ifndef KT_KB_DIRECT_BF16
 #define KT_KB_DIRECT_BF16 2      /* the same for the direct path on bf16 gradients (keeps it at 4 CTAs per SM) */
 #endif
-#ifndef KT_WARM_CTAS
-#define KT_WARM_CTAS 1184        /* about two waves: CTAs that prefetch the tables into L2 */
-#endif
 constexpr int NT = KT_NT;        // threads per CTA
 // transport elements per work unit (one CTA each): chosen by the gradient dtype so that every
 // thread has KT_ITERS 16-byte loads per rank in flight
@@ -76,8 +73,6 @@ struct TilePlan {         // which tiles a launch covers and how to decode them
     int single;           // the launch covers (part of) exactly one tensor: its record travels in `one`
     TInfo one;            // ... and the fused reduce decodes its tiles by arithmetic, without any table
     int single_skip;      // ... starting this many tiles into the tensor (a device's share may begin mid-tensor)
-    const void *tables;   // start of the table allocation (prefix, records, pointers) ...
-    int table_bytes;      // ... and how much of it is worth prefetching (0: nothing)
 };
 
 struct K1Params {
@@ -289,9 +284,9 @@ struct TileRef {
 // Tile -> tensor: the u with prefix[u] <= tile < prefix[u + 1] (prefix is non-decreasing, so
 // empty tensors never match).  One memory round trip: thread i tests tensor u_lo + i (in
 // strides of the CTA when there are more tensors than threads), the one that matches
-// publishes it through shared memory.  The first CTAs of a launch also pull the small tables
-// into L2 up front, so that the dependent look-ups that follow (record, pointers) do not
-// each wait for DRAM while the machine is still empty.  SINGLE_SHORTCUT: a launch that covers
+// publishes it through shared memory.  (Prefetching the tables into L2 by the first CTAs of a
+// launch was measured and taken out: it cost 1-4 % on the named workloads and 14 % on the
+// combine of the ragged MobileNetV2 list.)  SINGLE_SHORTCUT: a launch that covers
 // exactly one tensor (flat buffers, one-tensor buckets) carries that tensor's record in its
 // parameters and decodes tiles by arithmetic, with no table access at all (used by the fused
 // reduce, where it measured 1-8 % faster on flat buffers; the other kernels did not gain).
@@ -306,10 +301,6 @@ __device__ __forceinline__ TileRef locate_tile(const TilePlan &tp) {
     }
     __shared__ int s_u;
     const int tile = blockIdx.x + tp.tile_lo;
-    if (blockIdx.x < KT_WARM_CTAS) {
-        const char *line = static_cast<const char *>(tp.tables) + 128 * threadIdx.x;
-        if (128 * threadIdx.x < tp.table_bytes) asm volatile("prefetch.global.L2 [%0];" ::"l"(line));
-    }
     for (int u = tp.u_lo + threadIdx.x; u < tp.u_hi; u += NT) {
         const int a = __ldg(tp.prefix + u), b = __ldg(tp.prefix + u + 1);
         if (a <= tile && tile < b) s_u = u;
