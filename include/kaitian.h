@@ -269,6 +269,19 @@ int kt_ipc_close(const void *handle);
 int kt_host_register(void *host, int64_t bytes);
 int kt_host_unregister(void *host);
 
+/* A barrier between the processes of one node (the ranks of Section III-A's one-server
+ * deployment meet between the copy down and the copy up of the relay, and before and after a
+ * collective).  `shared` (host): KT_HOST_BARRIER_BYTES bytes, 64-byte aligned, in memory that
+ * every participating process maps, zeroed once before the first use.  Every one of the n_ranks
+ * processes calls kt_host_barrier; the call returns KT_OK once all have arrived.  Reusable at
+ * once.  The wait is on the host and bounded: with timeout_ms >= 0 a process that has waited that
+ * long returns KT_ERR_TIMEOUT (a rank died, hung or never joined), the device is not involved
+ * and stays usable; after a timeout the block is in an undefined state and must be zeroed
+ * again, by agreement of the survivors, before it is reused.  timeout_ms < 0 waits without
+ * limit.  Pure host function.  Errors: KT_ERR_INVALID, KT_ERR_ALIGN, KT_ERR_TIMEOUT. */
+#define KT_HOST_BARRIER_BYTES 128
+int kt_host_barrier(void *shared, int n_ranks, int timeout_ms);
+
 /* The two reductions of Section III-A.
  * transport: host array of G device pointers, fp32, transport_numel elements each,
  *        16-byte aligned.

@@ -30,7 +30,7 @@ EXPORTS = ["kt_schedule", "kt_scores", "kt_adapt_create", "kt_adapt_observe", "k
            "kt_get_coefficients", "kt_set_transport_dtype", "kt_route", "kt_bucket_pack", "kt_plan_buckets", "kt_plan_query", "kt_hier_reduce",
            "kt_stage_to_host", "kt_relay_through_host", "kt_stage_wait", "kt_unpack_scale", "kt_sync_direct", "kt_allreduce", "kt_bcast_send", "kt_bcast_relay", "kt_bcast_recv", "kt_cast", "kt_copy_tensors", "kt_sync_flat_static", "kt_launch_count",
            "kt_last_error", "kt_destroy", "kt_work_unit", "kt_shard_ranges", "kt_shard_bind", "kt_shard_query",
-           "kt_ipc_export", "kt_ipc_open", "kt_ipc_close", "kt_host_register", "kt_host_unregister"]
+           "kt_ipc_export", "kt_ipc_open", "kt_ipc_close", "kt_host_register", "kt_host_unregister", "kt_host_barrier"]
 
 _DTYPES = {torch.float32: KT_F32, torch.bfloat16: KT_BF16}
 
@@ -96,6 +96,7 @@ def _load() -> C.CDLL:
         "kt_ipc_close": ([vp], C.c_int),
         "kt_host_register": ([vp, C.c_int64], C.c_int),
         "kt_host_unregister": ([vp], C.c_int),
+        "kt_host_barrier": ([vp, C.c_int, C.c_int], C.c_int),
         "kt_launch_count": ([vp], C.c_int64),
         "kt_last_error": ([vp], C.c_char_p),
         "kt_destroy": ([vp], None),
@@ -419,6 +420,15 @@ def kt_host_register(address: int, nbytes: int) -> None:
 
 def kt_host_unregister(address: int) -> None:
     _check(_lib.kt_host_unregister(C.c_void_p(int(address))))
+
+
+KT_HOST_BARRIER_BYTES = 128
+
+
+def kt_host_barrier(address: int, n_ranks: int, timeout_ms: int = -1) -> None:
+    """Barrier between the processes of a node on a zeroed, 64-byte aligned block of shared host
+    memory; raises KtError(KT_ERR_TIMEOUT) when the others do not arrive in time."""
+    _check(_lib.kt_host_barrier(C.c_void_p(int(address)), int(n_ranks), int(timeout_ms)))
 
 
 def kt_plan_buckets(numel: Sequence[int], bucket_cap_bytes: int) -> Plan:

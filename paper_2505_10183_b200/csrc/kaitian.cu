@@ -19,6 +19,7 @@
 #include "kt_kernels.cuh"
 
 #include <algorithm>
+#include <atomic>
 #include <chrono>
 #include <cmath>
 #include <cstdarg>
@@ -1351,6 +1352,41 @@ int kt_host_unregister(void *host) {
     if (!host) return fail(KT_ERR_INVALID, "NULL argument");
     KT_CUDA(cudaHostUnregister(host));
     return KT_OK;
+}
+
+// ---- a barrier for the processes of one node, in host memory they all map
+namespace {
+struct HostBarrier {                       // KT_HOST_BARRIER_BYTES of shared memory, zero before first use
+    std::atomic<uint32_t> arrived;
+    char pad_[60];
+    std::atomic<uint32_t> generation;
+    char pad2_[60];
+};
+static_assert(sizeof(HostBarrier) == KT_HOST_BARRIER_BYTES, "barrier layout");
+static_assert(std::atomic<uint32_t>::is_always_lock_free, "the barrier needs lock-free 32-bit atomics");
+}  // namespace
+
+int kt_host_barrier(void *shared, int n_ranks, int timeout_ms) {
+    if (!shared) return fail(KT_ERR_INVALID, "shared is NULL");
+    if (reinterpret_cast<uintptr_t>(shared) % 64) return fail(KT_ERR_ALIGN, "the barrier block must be 64-byte aligned");
+    if (n_ranks < 1) return fail(KT_ERR_INVALID, "n_ranks = %d must be >= 1", n_ranks);
+    HostBarrier *b = static_cast<HostBarrier *>(shared);
+    const uint32_t gen = b->generation.load(std::memory_order_acquire);
+    if (b->arrived.fetch_add(1, std::memory_order_acq_rel) + 1 == static_cast<uint32_t>(n_ranks)) {
+        b->arrived.store(0, std::memory_order_relaxed);          // before the release below: the next round starts clean
+        b->generation.store(gen + 1, std::memory_order_release);
+        return KT_OK;
+    }
+    const auto deadline = std::chrono::steady_clock::now() + std::chrono::milliseconds(timeout_ms < 0 ? 0 : timeout_ms);
+    for (unsigned spins = 0;; ++spins) {
+        if (b->generation.load(std::memory_order_acquire) != gen) return KT_OK;
+        if (spins < 4096) continue;                              // a few microseconds of plain polling first
+        if (timeout_ms >= 0 && std::chrono::steady_clock::now() >= deadline)
+            return fail(KT_ERR_TIMEOUT, "host barrier: %u of %d ranks had arrived after %d ms",
+                        b->arrived.load(std::memory_order_relaxed), n_ranks, timeout_ms);
+        if (spins & 1) std::this_thread::yield();
+        else std::this_thread::sleep_for(std::chrono::microseconds(20));
+    }
 }
 
 int64_t kt_launch_count(const kt_ctx *c) { return c ? c->launches : 0; }

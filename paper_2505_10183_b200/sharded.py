@@ -3,10 +3,11 @@
 Every rank is a process with a device of its own (paper Section III-A: the devices of a group
 run their collective among themselves; groups exchange through host memory).  This module
 holds no arithmetic.  It moves handles and names between the processes with
-``torch.distributed`` (object collectives and barriers on a host-side process group), maps the
+``torch.distributed`` (object collectives on a host-side process group, at set-up only), maps the
 group mates' gradient and output tensors into this process (``kt_ipc_open``), maps one block of
 host memory that all processes of the node share (POSIX shared memory, page-locked with
-``kt_host_register``), and then issues the library calls of a step in order:
+``kt_host_register``; it also holds the block of ``kt_host_barrier``, where the ranks meet
+during a step), and then issues the library calls of a step in order:
 
     barrier                         every rank's gradients are complete
     kt_hier_reduce(KT_INTRA)        my share of each bucket, read from all members of my group
@@ -96,31 +97,37 @@ class ShardedSync:
         self.main = torch.cuda.Stream()
         self.side = torch.cuda.Stream()
 
-        # 3. host memory that all processes share: the G partials, end to end, in a file of the
-        #    node's shared-memory file system that every rank maps and page-locks
+        # 3. host memory that all processes share: a barrier block, then the G partials end to
+        #    end, in a file of the node's shared-memory file system that every rank maps and
+        #    page-locks
+        self._header = 4096
+        nbytes = self._header + (self.G * max(n, 1) * 4 if self.G > 1 else 0)
+        name = [None]
+        if rank == 0:
+            name[0] = "/dev/shm/kt_partials_%d_%s" % (os.getpid(), secrets.token_hex(4))
+            fd = os.open(name[0], os.O_CREAT | os.O_EXCL | os.O_RDWR, 0o600)
+            os.ftruncate(fd, nbytes)                      # new pages read as zero: the barrier starts clean
+        dist.broadcast_object_list(name, src=0, group=host_group)
+        if rank != 0:
+            fd = os.open(name[0], os.O_RDWR)
+        self._map = mmap.mmap(fd, nbytes)
+        os.close(fd)
+        self._view = C.c_char.from_buffer(self._map)
+        self._host_address = C.addressof(self._view)
+        kt.kt_host_register(self._host_address, nbytes)
         self.host_rows = None
-        self._map = None
         if self.G > 1:
-            nbytes = self.G * max(n, 1) * 4
-            name = [None]
-            if rank == 0:
-                name[0] = "/dev/shm/kt_partials_%d_%s" % (os.getpid(), secrets.token_hex(4))
-                fd = os.open(name[0], os.O_CREAT | os.O_EXCL | os.O_RDWR, 0o600)
-                os.ftruncate(fd, nbytes)
-            dist.broadcast_object_list(name, src=0, group=host_group)
-            if rank != 0:
-                fd = os.open(name[0], os.O_RDWR)
-            self._shm_name = name[0]
-            self._map = mmap.mmap(fd, nbytes)
-            os.close(fd)
-            self._view = C.c_char.from_buffer(self._map)
-            self._host_address = C.addressof(self._view)
-            kt.kt_host_register(self._host_address, nbytes)
-            self.host_rows = kt.PtrArray.from_addresses([self._host_address + g * max(n, 1) * 4 for g in range(self.G)],
+            first = self._host_address + self._header
+            self.host_rows = kt.PtrArray.from_addresses([first + g * max(n, 1) * 4 for g in range(self.G)],
                                                         keep=self._map)
-            dist.barrier(group=host_group)
-            if rank == 0:
-                os.unlink(name[0])                    # every rank has it mapped: the name can go
+        dist.barrier(group=host_group)
+        if rank == 0:
+            os.unlink(name[0])                            # every rank has it mapped: the name can go
+
+    def barrier(self) -> None:
+        """All ranks of the job meet here, on the host, in the shared block; a rank that does not
+        come within `wait_ms` ends the wait of the others with KT_ERR_TIMEOUT."""
+        kt.kt_host_barrier(self._host_address, self.K, self.wait_ms)
 
     def my_range(self, bucket: int = -1):
         return kt.kt_shard_query(self.ctx, bucket)[:2]
@@ -130,7 +137,7 @@ class ShardedSync:
         other rank has finished reading this rank's `grads`."""
         ctx = self.ctx
         torch.cuda.synchronize()                      # whatever produced my gradients is done
-        dist.barrier(group=self.host_group)
+        self.barrier()
         if self.G == 1:
             for b in self.buckets:
                 kt.kt_sync_direct(ctx, self.out_ptrs, scale=scale, bucket=b, out_dtype=self.out_dtype,
@@ -142,7 +149,7 @@ class ShardedSync:
                                     main_stream=self.main, side_stream=self.side)
             for b in self.buckets:                    # my shares are in host memory ...
                 kt.kt_stage_wait(ctx, kt.KT_D2H, bucket=b, main_stream=self.main, timeout_ms=self.wait_ms)
-            dist.barrier(group=self.host_group)       # ... and so are everybody else's
+            self.barrier()                            # ... and so are everybody else's
             for b in self.buckets:
                 kt.kt_stage_to_host(ctx, kt.KT_H2D, self.partial_rows, self.host_rows, bucket=b,
                                     main_stream=self.main, side_stream=self.side)
@@ -151,18 +158,17 @@ class ShardedSync:
                 kt.kt_unpack_scale(ctx, self.partial_rows, self.out_ptrs, scale=scale, bucket=b,
                                    out_dtype=self.out_dtype, R=len(self.members), stream=self.main)
         self.main.synchronize()                       # my shares are written everywhere in my group
-        dist.barrier(group=self.host_group)
+        self.barrier()
 
     def close(self) -> None:
         torch.cuda.synchronize()
-        dist.barrier(group=self.host_group)           # nobody still reads what is unmapped next
+        self.barrier()                                # nobody still reads what is unmapped next
         kt.kt_destroy(self.ctx)
         for handle in self._opened:
             kt.kt_ipc_close(handle)
         self._opened = []
-        if self._map is not None:
-            kt.kt_host_unregister(self._host_address)
-            self.host_rows = None
-            del self._view
-            self._map.close()
-            self._map = None
+        kt.kt_host_unregister(self._host_address)
+        self.host_rows = None
+        del self._view
+        self._map.close()
+        self._map = None
