@@ -15,6 +15,8 @@
  *   kt_unpack_scale  per-parameter gradients = cast(scale * S)
  * or, when no host relay is needed (Section III-B, homogeneous dispatch),
  *   kt_sync_direct   all of the above arithmetic in one pass, no transport
+ * With every rank a process on a device of its own, the same calls work on one member's share
+ * of each bucket after kt_shard_bind (group mates' tensors through peer-mapped addresses).
  *
  * Conventions
  *  - Every pointer argument says "host" or "device".  "host array of device pointers"
@@ -488,7 +490,8 @@ int kt_sync_flat_static(const int32_t *group_of, const int32_t *shares, int K, i
  * destination table returns KT_ERR_STATE and kt_graph_end then drops the recording with
  * KT_ERR_STATE); every copy stream must be waited
  * for with kt_stage_wait(..., timeout_ms < 0) before kt_graph_end; pointers, sizes, shares
- * and scale are frozen into the recording (record again after kt_set_shares).
+ * and scale are frozen into the recording (record again after kt_set_shares; a recording is
+ * void once kt_bucket_pack has re-planned the context and must not be launched again).
  * kt_graph_nodes: number of recorded operations.  The graph owns no buffers.
  * Errors: KT_ERR_STATE, KT_ERR_INVALID, KT_ERR_NOMEM, KT_ERR_CUDA. */
 int kt_graph_begin(kt_ctx *ctx, void *stream);

@@ -91,7 +91,8 @@ struct OutSet {
     size_t cap = 0;                  // bytes of both
     std::vector<void *> ptrs;        // what was uploaded (caller's order)
     int R = 0, dtype = -1;
-    cudaEvent_t uploaded = nullptr;  // the upload has read the staging image
+    cudaEvent_t uploaded = nullptr;  // the upload has read the staging image and written the table
+    cudaStream_t upload_stream = nullptr;   // where that copy was queued
     cudaEvent_t used = nullptr;      // the last kernel that reads the device table
     uint64_t stamp = 0;              // last use, for replacement
     bool in_recording = false;       // a recorded step reads this table whenever it is replayed: never replaced
@@ -437,6 +438,9 @@ int upload_out_table(kt_ctx *c, void *const *out_grads, int R, int out_dtype, cu
             std::memcmp(o.ptrs.data(), out_grads, np * sizeof(void *)) == 0) {
             o.stamp = ++c->out_clock;
             o.in_recording = o.in_recording || capturing;
+            // the table was uploaded on another stream: this one must not run ahead of that copy
+            // (while recording nothing is pending: kt_graph_begin has waited for every upload)
+            if (!capturing && s != o.upload_stream) KT_CUDA(cudaStreamWaitEvent(s, o.uploaded, 0));
             *set_out = &o;
             return KT_OK;
         }
@@ -501,6 +505,7 @@ int upload_out_table(kt_ctx *c, void *const *out_grads, int R, int out_dtype, cu
     KT_CUDA(cudaMemcpyAsync(o.dev, o.staging, need, cudaMemcpyHostToDevice, s));
     KT_CUDA(cudaEventRecord(o.uploaded, s));
     KT_CUDA(cudaEventRecord(o.used, s));
+    o.upload_stream = s;
     o.ptrs.assign(out_grads, out_grads + np);
     o.R = R;
     o.dtype = out_dtype;
@@ -1429,6 +1434,10 @@ extern "C" {
 int kt_graph_begin(kt_ctx *c, void *stream) {
     if (int rc = check_ctx(c, true)) return rc;
     KT_ON_DEVICE(c->device);
+    // destination tables uploaded by earlier calls must be complete before a recording relies on
+    // them: a recorded launch cannot wait for an event from outside the recording
+    for (OutSet &o : c->out_sets)
+        if (o.uploaded) KT_CUDA(cudaEventSynchronize(o.uploaded));
     // thread-local mode: other threads of the process may keep allocating while this one records
     KT_CUDA(cudaStreamBeginCapture(static_cast<cudaStream_t>(stream), cudaStreamCaptureModeThreadLocal));
     c->recording_broken = false;

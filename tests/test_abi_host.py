@@ -160,3 +160,14 @@ def test_shard_ranges_match_the_oracle(kt, oracle):
             kt.kt_shard_ranges(*bad)
     with pytest.raises(kt.KtError):
         kt.kt_work_unit(7)
+
+
+def test_shared_memory_calls_validate_arguments(kt):
+    """kt_ipc_* and kt_host_register refuse null addresses, negative offsets and empty ranges on
+    the host, before any CUDA call (so this runs without a device)."""
+    for call in (lambda: kt.kt_ipc_export(0), lambda: kt.kt_ipc_open(b"\0" * kt.KT_IPC_HANDLE_BYTES, -1),
+                 lambda: kt.kt_host_register(0, 4096), lambda: kt.kt_host_register(4096, 0),
+                 lambda: kt.kt_host_unregister(0)):
+        with pytest.raises(kt.KtError) as e:
+            call()
+        assert e.value.status == kt.KT_ERR_INVALID

@@ -159,3 +159,34 @@ def test_alternating_output_sets_eager_and_recorded(kt, oracle, name):
     for g in graphs:
         kt.kt_graph_destroy(g)
     kt.kt_destroy(ctx)
+
+
+def test_destination_table_uploaded_on_one_stream_is_safe_to_use_on_another(kt, oracle):
+    """A set of output tensors is first seen by a call on stream A, whose queue is long (the
+    upload of its destination table sits behind a large fill); a call on stream B uses the same
+    set right away.  B's kernel must wait for that upload, not for the rest of A."""
+    wl = W.mobilenet_v2()
+    shares = H.shares_of(wl, kt)
+    host, dev = H.device_gradients(wl)
+    ctx = kt.kt_groups_init(wl.group_of, shares, wl.G)
+    kt.kt_bucket_pack(ctx, dev, wl.bucket_cap_bytes)
+    n = kt.kt_plan_query(ctx).transport_numel
+    transport = [torch.full((n,), float("nan"), device="cuda") for _ in range(wl.G)]
+    out = [[torch.full((m,), float("nan"), device="cuda") for m in wl.numel]]
+    want, _, _, _ = H.run_oracle_path(oracle, wl, host, shares)
+    A, B = torch.cuda.Stream(), torch.cuda.Stream()
+    ballast = torch.empty(2 << 30, dtype=torch.uint8, device="cuda")
+    kt.kt_hier_reduce(ctx, kt.KT_INTRA, transport, stream=A)
+    reduced = torch.cuda.Event()
+    reduced.record(A)
+    with torch.cuda.stream(A):
+        for _ in range(4):
+            ballast.fill_(1)                                    # A is busy for a while
+    kt.kt_unpack_scale(ctx, transport, out, stream=A)           # first use of the set: upload queued on A
+    B.wait_event(reduced)
+    kt.kt_unpack_scale(ctx, transport, out, scale=1.0, stream=B)   # same set, other stream
+    B.synchronize()
+    for t in range(wl.T):
+        H.assert_bit_equal(out[0][t], want[t], "out[%d] written from stream B" % t)
+    torch.cuda.synchronize()
+    kt.kt_destroy(ctx)
