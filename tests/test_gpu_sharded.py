@@ -36,7 +36,7 @@ def kt():
     return binding
 
 
-def run_emulated(kt, oracle, wl, host, dev, out_dtype, scale, per_bucket, relay, in_place=False):
+def run_emulated(kt, oracle, wl, host, dev, out_dtype, scale, per_bucket, relay, in_place=False, narrow=False):
     """All ranks of the job as contexts of one process.  Every rank reduces its share of every
     range; the shares of a group land in one buffer per group, which stands for the host
     memory all ranks can reach (with relay=True they really cross pinned host memory)."""
@@ -51,13 +51,17 @@ def run_emulated(kt, oracle, wl, host, dev, out_dtype, scale, per_bucket, relay,
     for r in range(K):
         ctx = kt.kt_groups_init(wl.group_of, wl.shares, G)
         kt.kt_shard_bind(ctx, r, wl.group_of)
+        if narrow:                                       # the library's bf16 transport (an extension)
+            kt.kt_set_transport_dtype(ctx, kt.KT_BF16)
         kt.kt_bucket_pack(ctx, [dev[q] for q in members[wl.group_of[r]]], wl.bucket_cap_bytes)
         ctxs.append(ctx)
     plan = kt.kt_plan_query(ctxs[0])
     n = plan.transport_numel
     poison = float(np.float32(-7.25e33))
-    own = [torch.full((G, n), poison, device="cuda") for _ in range(K)]         # every rank's device rows
-    shared = list(torch.full((G, n), poison).pin_memory()) if relay else None     # the host block all ranks reach
+    tdt = torch.bfloat16 if narrow else torch.float32
+    own = [torch.full((G, n), poison, dtype=tdt, device="cuda") for _ in range(K)]   # every rank's device rows
+    poison = float(own[0][0, 0]) if n else poison                                 # the value as the buffer holds it
+    shared = list(torch.full((G, n), poison, dtype=tdt).pin_memory()) if relay else None   # the host block all ranks reach
     buckets = list(range(plan.n_buckets)) if per_bucket else [-1]
     side = torch.cuda.Stream()
     # the ranges the library hands out are the oracle's
@@ -69,7 +73,8 @@ def run_emulated(kt, oracle, wl, host, dev, out_dtype, scale, per_bucket, relay,
                 assert (lo, cnt) == want[m] and M == len(members[g])
                 assert kt.kt_shard_query(ctxs[members[g][0]], b, member=m)[:2] == want[m]
     want_out, want_parts, _, _ = oracle.sync_step(host, wl.numel, dt, wl.group_of, wl.shares, G,
-                                                  wl.bucket_cap_bytes, scale, odt)
+                                                  wl.bucket_cap_bytes, scale, odt, 1 if narrow else 0)
+    bits = torch.int16 if narrow else torch.int32
     if G == 1:
         for b in buckets:
             for r in range(K):
@@ -88,8 +93,8 @@ def run_emulated(kt, oracle, wl, host, dev, out_dtype, scale, per_bucket, relay,
             for b in buckets:
                 lo, cnt, _ = kt.kt_shard_query(ctxs[r], b)
                 mask[lo:lo + cnt] = True
-            part = torch.from_numpy(want_parts[g]).cuda()
-            assert torch.equal(own[r][g][mask].view(torch.int32), part[mask].view(torch.int32))
+            part = torch.from_numpy(want_parts[g].view(np.int16) if narrow else want_parts[g]).cuda()
+            assert torch.equal(own[r][g][mask].view(bits), part[mask].view(bits))
             assert bool((own[r][g][~mask] == poison).all())
             for h in range(G):
                 if h != g:
@@ -144,6 +149,17 @@ def test_emulated_ranks_random_problems(kt, oracle, seed):
         in_place = out_dtype == H.TORCH_DT[wl.dtype] and rnd.random() < 0.4
         run_emulated(kt, oracle, wl, host, dev, out_dtype, rnd.choice([1.0, 1.0 / 3.0]), rnd.random() < 0.5,
                      rnd.random() < 0.5, in_place)
+
+
+@pytest.mark.parametrize("name", ["tiny", "mobilenet_v2", "resnet50"])
+def test_emulated_ranks_with_the_bf16_transport(kt, oracle, name):
+    """The narrow transport (an extension of this library) on shares: the partial a member stores
+    is rounded once, where the oracle rounds it."""
+    wl = W.by_name(name)
+    wl.shares = H.shares_of(wl, kt)
+    host, dev = H.device_gradients(wl)
+    run_emulated(kt, oracle, wl, host, dev, H.TORCH_DT[wl.dtype], 0.5, True, True, False, narrow=True)
+    run_emulated(kt, oracle, wl, host, dev, torch.float32, 1.0, False, False, False, narrow=True)
 
 
 def test_calls_that_need_all_ranks_are_refused_on_a_bound_context(kt):
