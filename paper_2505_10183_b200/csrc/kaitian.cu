@@ -1382,15 +1382,27 @@ int kt_host_barrier(void *shared, int n_ranks, int timeout_ms) {
         b->generation.store(gen + 1, std::memory_order_release);
         return KT_OK;
     }
-    const auto deadline = std::chrono::steady_clock::now() + std::chrono::milliseconds(timeout_ms < 0 ? 0 : timeout_ms);
+    // Poll without giving up the core for the first 200 us (ranks of one step arrive within
+    // microseconds of each other), then yield between polls, and after 5 ms sleep between them.
+    const auto begin = std::chrono::steady_clock::now();
+    const auto deadline = begin + std::chrono::milliseconds(timeout_ms < 0 ? 0 : timeout_ms);
     for (unsigned spins = 0;; ++spins) {
         if (b->generation.load(std::memory_order_acquire) != gen) return KT_OK;
-        if (spins < 4096) continue;                              // a few microseconds of plain polling first
-        if (timeout_ms >= 0 && std::chrono::steady_clock::now() >= deadline)
+        if ((spins & 63u) != 63u) {
+#if defined(__x86_64__) || defined(__i386__)
+            __builtin_ia32_pause();
+#elif defined(__aarch64__)
+            asm volatile("yield");
+#endif
+            continue;
+        }
+        const auto now = std::chrono::steady_clock::now();
+        if (timeout_ms >= 0 && now >= deadline)
             return fail(KT_ERR_TIMEOUT, "host barrier: %u of %d ranks had arrived after %d ms",
                         b->arrived.load(std::memory_order_relaxed), n_ranks, timeout_ms);
-        if (spins & 1) std::this_thread::yield();
-        else std::this_thread::sleep_for(std::chrono::microseconds(20));
+        if (now - begin < std::chrono::microseconds(200)) continue;
+        if (now - begin < std::chrono::milliseconds(5)) std::this_thread::yield();
+        else std::this_thread::sleep_for(std::chrono::microseconds(50));
     }
 }
 
