@@ -5,7 +5,7 @@
 // Work decomposition.  The fp32 transport is cut into tiles of TILE elements that never
 // cross a tensor boundary; one CTA handles one tile (the grid is the tile count, so the
 // hardware scheduler balances ragged tensor lists and partial waves by itself).  A CTA
-// finds its tensor by binary search in the per-tensor tile prefix, then streams the K rank
+// finds its tensor in the per-tensor tile prefix (one thread per tensor), then streams the K rank
 // buffers of that tile with 128-bit loads, all loads of a batch of ranks issued before the
 // first multiply.  Interior tiles of 16-byte aligned tensors run without predicates; tiles
 // that hold a tensor's tail, zero padding, or a misaligned tensor use the same code with
@@ -67,8 +67,8 @@ struct TilePlan {         // which tiles a launch covers and how to decode them
     const TInfo *info;    // [T]
     int T;
     int u_lo, u_hi;       // tensors [u_lo, u_hi) take part
-    int tile_lo;          // prefix[u_lo]
-    int n_tiles;          // prefix[u_hi] - prefix[u_lo]
+    int tile_lo;          // first tile of the launch: prefix[u_lo], or later when a device's share starts mid-tensor
+    int n_tiles;          // tiles of the launch (it may end before prefix[u_hi] for the same reason)
     int tile;             // elements per tile the prefix was built for
     int single;           // the launch covers (part of) exactly one tensor: its record travels in `one`
     TInfo one;            // ... and the fused reduce decodes its tiles by arithmetic, without any table
