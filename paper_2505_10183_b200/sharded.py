@@ -38,11 +38,12 @@ from . import binding as kt
 class ShardedSync:
     def __init__(self, rank: int, group_of: Sequence[int], shares: Sequence[int], grads: Sequence[torch.Tensor],
                  outs: Optional[Sequence[torch.Tensor]] = None, bucket_cap_bytes: int = 25 << 20,
-                 host_group=None, per_bucket: bool = True, wait_ms: int = 60000):
+                 host_group=None, per_bucket: bool = True, wait_ms: int = 60000, narrow_transport: bool = False):
         """grads: this rank's gradient tensors (device, contiguous, one dtype); outs: where this
         rank wants the reduced gradients (None: in place, over `grads`); host_group: a
         torch.distributed group whose collectives run on the host (gloo) and whose ranks are
-        numbered like `group_of`."""
+        numbered like `group_of`; narrow_transport: the library's bf16 transport (an extension:
+        half the bytes through host memory, one extra rounding of every group partial)."""
         self.rank, self.group_of, self.K = rank, list(group_of), len(group_of)
         self.G = max(group_of) + 1
         self.g = group_of[rank]
@@ -85,6 +86,9 @@ class ShardedSync:
         # 2. the context of this rank
         self.ctx = kt.kt_groups_init(self.group_of, list(shares), self.G)
         kt.kt_shard_bind(self.ctx, rank, self.group_of)
+        if narrow_transport:
+            kt.kt_set_transport_dtype(self.ctx, kt.KT_BF16)
+        tdt, tsize = (torch.bfloat16, 2) if narrow_transport else (torch.float32, 4)
         kt.kt_bucket_pack_ptrs(self.ctx, kt.PtrArray.from_addresses(grad_ptrs, keep=self.grads), self.numel,
                                self.in_dtype, bucket_cap_bytes)
         self.plan = kt.kt_plan_query(self.ctx)
@@ -92,7 +96,7 @@ class ShardedSync:
         self.out_ptrs = kt.PtrArray.from_addresses(out_ptrs, keep=self.outs)
         n = self.plan.transport_numel
         # row g: my share of my group's partial; rows h != g: the other groups' partials over my range
-        self.partials = torch.zeros(self.G, max(n, 1), dtype=torch.float32, device=grads[0].device)
+        self.partials = torch.zeros(self.G, max(n, 1), dtype=tdt, device=grads[0].device)
         self.partial_rows = kt.kt_ptrs(list(self.partials))
         self.main = torch.cuda.Stream()
         self.side = torch.cuda.Stream()
@@ -101,7 +105,7 @@ class ShardedSync:
         #    end, in a file of the node's shared-memory file system that every rank maps and
         #    page-locks
         self._header = 4096
-        nbytes = self._header + (self.G * max(n, 1) * 4 if self.G > 1 else 0)
+        nbytes = self._header + (self.G * max(n, 1) * tsize if self.G > 1 else 0)
         name = [None]
         if rank == 0:
             name[0] = "/dev/shm/kt_partials_%d_%s" % (os.getpid(), secrets.token_hex(4))
@@ -118,7 +122,7 @@ class ShardedSync:
         self.host_rows = None
         if self.G > 1:
             first = self._host_address + self._header
-            self.host_rows = kt.PtrArray.from_addresses([first + g * max(n, 1) * 4 for g in range(self.G)],
+            self.host_rows = kt.PtrArray.from_addresses([first + g * max(n, 1) * tsize for g in range(self.G)],
                                                         keep=self._map)
         dist.barrier(group=host_group)
         if rank == 0:

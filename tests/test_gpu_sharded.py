@@ -202,6 +202,8 @@ CASES = [
          in_place=True),
     dict(name="bf16_to_f32", wl="tiny", dtype="bf16", out_dtype="f32", group_of=[0, 1, 1, 1], shares=[64, 64, 32, 32],
          per_bucket=True, in_place=False),
+    dict(name="narrow_transport", wl="mobilenet_v2", group_of=[0, 1, 0, 1], shares=[79, 49, 79, 49], per_bucket=True,
+         in_place=False, narrow=True),
 ]
 
 
@@ -238,8 +240,9 @@ def rank_main(rank, world, port, cases):
         mine = [t.cuda() for t in W.split_tensors(W.rank_gradients(wl, rank, "cpu"), wl.numel)]
         outs = None if case["in_place"] else [torch.full((m,), float("nan"), dtype=H.TORCH_DT[odt_name], device="cuda")
                                               for m in wl.numel]
+        narrow = case.get("narrow", False)
         job = ShardedSync(rank, wl.group_of, wl.shares, mine, outs, wl.bucket_cap_bytes, host_group=None,
-                          per_bucket=case["per_bucket"])
+                          per_bucket=case["per_bucket"], narrow_transport=narrow)
         assert job.my_range(-1 if not case["per_bucket"] else 0) == oracle.shard_ranges(
             wl.numel, wl.bucket_cap_bytes, kt.kt_work_unit(dt), -1 if not case["per_bucket"] else 0,
             len(job.members))[job.member]
@@ -247,7 +250,7 @@ def rank_main(rank, world, port, cases):
         for scale in scales:
             job.step(scale=scale)
             want, _, _, _ = oracle.sync_step(host, wl.numel, dt, wl.group_of, wl.shares, wl.G, wl.bucket_cap_bytes,
-                                             scale, H.ORACLE_DT[odt_name])
+                                             scale, H.ORACLE_DT[odt_name], 1 if narrow else 0)
             result = mine if case["in_place"] else outs
             for t in range(wl.T):
                 H.assert_bit_equal(result[t], want[t], "%s rank %d out[%d] scale %g" % (case["name"], rank, t, scale))
