@@ -164,9 +164,13 @@ class ShardedSync:
         self.main.synchronize()                       # my shares are written everywhere in my group
         self.barrier()
 
-    def close(self) -> None:
+    def close(self, meet: bool = True) -> None:
+        """Unmaps everything.  meet=False skips the barrier in the shared block: for ranks that
+        have seen a barrier time out (the block is then in an undefined state) and have made sure
+        by other means that no rank still uses this one's memory."""
         torch.cuda.synchronize()
-        self.barrier()                                # nobody still reads what is unmapped next
+        if meet:
+            self.barrier()                            # nobody still reads what is unmapped next
         kt.kt_destroy(self.ctx)
         for handle in self._opened:
             kt.kt_ipc_close(handle)

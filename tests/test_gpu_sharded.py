@@ -270,3 +270,52 @@ def test_ranks_as_processes_over_mapped_memory(world):
     assert cases
     port = 29600 + (os.getpid() * 7 + world) % 2000
     mp.spawn(rank_main, args=(world, port, cases), nprocs=world, join=True)
+
+
+def leaving_rank_main(rank, world, port):
+    """Ranks 0..2 keep stepping; rank 3 stops after the first step, between steps, with none of
+    its kernels or copies in flight, and simply stays away from the next one."""
+    sys.path.insert(0, ROOT)
+    sys.path.insert(0, os.path.join(ROOT, "tests"))
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    import time
+    import torch.distributed as dist
+    from oracle import kt_oracle as oracle
+    from paper_2505_10183_b200 import binding as kt
+    from paper_2505_10183_b200.sharded import ShardedSync
+    torch.cuda.set_device(0)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    wl = W.tiny()
+    host = [[W.as_numpy(t) for t in W.split_tensors(W.rank_gradients(wl, r, "cpu"), wl.numel)] for r in range(wl.K)]
+    mine = [t.cuda() for t in W.split_tensors(W.rank_gradients(wl, rank, "cpu"), wl.numel)]
+    outs = [torch.full((m,), float("nan"), device="cuda") for m in wl.numel]
+    job = ShardedSync(rank, wl.group_of, wl.shares, mine, outs, wl.bucket_cap_bytes, wait_ms=400)
+    job.step()                                              # everybody takes part in the first step
+    want, _, _, _ = oracle.sync_step(host, wl.numel, 0, wl.group_of, wl.shares, wl.G, wl.bucket_cap_bytes)
+    for t in range(wl.T):
+        H.assert_bit_equal(outs[t], want[t], "rank %d out[%d]" % (rank, t))
+    if rank != world - 1:
+        t0 = time.time()
+        try:
+            job.step()
+            raise AssertionError("rank %d: the step went through without rank %d" % (rank, world - 1))
+        except kt.KtError as e:                             # the wait ended on the host, with a status
+            assert e.status == kt.KT_ERR_TIMEOUT and time.time() - t0 < 10.0
+        # the device is untouched by the failed step and still works
+        probe = torch.empty(wl.numel[0], device="cuda")
+        kt.kt_cast(mine[0].to(torch.bfloat16), probe)
+        torch.cuda.synchronize()
+        assert bool(torch.isfinite(probe).all())
+    dist.barrier()                                          # the survivors and the leaver agree to stop
+    job.close(meet=False)
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+def test_a_rank_that_stays_away_between_steps_is_noticed_on_the_host():
+    """Failure handling of the one-rank-per-device path: nothing on any GPU waits for the missing
+    rank, so the others get KT_ERR_TIMEOUT from the host barrier and keep a usable device."""
+    import torch.multiprocessing as mp
+    if not torch.cuda.is_available():
+        pytest.fail("this test needs a CUDA device")
+    mp.spawn(leaving_rank_main, args=(4, 29600 + (os.getpid() * 11) % 2000), nprocs=4, join=True)
