@@ -828,13 +828,13 @@ def run_sharded(args) -> dict:
     from paper_2505_10183_b200 import binding as kt
     from paper_2505_10183_b200.sharded import ShardedSync
     import torch.distributed as dist
-    world, rank, local, started = init_ranks("nccl")
+    # the ranks talk to each other on the host only (handles and names at set-up, then the
+    # shared-memory barrier): a gloo group is all this arm needs
+    world, rank, local, started = init_ranks("gloo")
     torch.cuda.set_device(local)
     if started is None:
         dist.init_process_group("gloo", rank=0, world_size=1, init_method="tcp://127.0.0.1:%d" % free_port())
-        host_group = None
-    else:
-        host_group = dist.new_group(backend="gloo")        # barriers and object exchange stay on the host
+    host_group = None
     wl = sharded_workload(args.workload, world)
     shares = kt.kt_schedule(wl.step_times, wl.global_batch)
     dt = torch.float32 if wl.dtype == "f32" else torch.bfloat16
