@@ -343,6 +343,8 @@ int kt_stage_wait(kt_ctx *ctx, int dir, int bucket, void *main_stream, int timeo
  *        R = 1, or up to K to hand every rank its own copy; element type out_dtype;
  *        numel as registered.  16-byte aligned tensors take the vectorised path.
  * out[t][j] = cast(scale * S[tensor_offset[t] + j]); one rounded multiply; padding ignored.
+ * In place: the outputs may be the registered gradient tensors themselves (the reduce that
+ *        read them is an earlier launch on the stream); they must not overlap `src`.
  * Destination tables: the R*T output pointers live in a small device table.  A context keeps
  *        up to 8 such tables, one per set of output tensors it has seen (least recently used
  *        replaced), so a caller that alternates between sets -- double-buffered gradients --

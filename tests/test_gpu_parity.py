@@ -271,6 +271,27 @@ def test_identical_ranks_and_equal_shares(kt, oracle):
     assert np.max(np.abs(got - stack.mean(0)) / np.abs(stack).mean(0)) < 1e-6
 
 
+@pytest.mark.parametrize("name", ["tiny", "mobilenet_v2"])
+def test_two_kernel_route_in_place(kt, oracle, name):
+    """The reduced gradients overwrite the registered gradient tensors of every rank (the usual
+    in-place all-reduce): the fused reduce has read everything before the combine writes."""
+    wl = W.by_name(name)
+    shares = H.shares_of(wl, kt)
+    host, dev = H.device_gradients(wl, misalign=1)
+    ctx = kt.kt_groups_init(wl.group_of, shares, wl.G)
+    kt.kt_bucket_pack(ctx, dev, wl.bucket_cap_bytes)
+    n = kt.kt_plan_query(ctx).transport_numel
+    transport = [torch.full((n,), float("nan"), device="cuda") for _ in range(wl.G)]
+    kt.kt_hier_reduce(ctx, kt.KT_INTRA, transport)
+    kt.kt_unpack_scale(ctx, transport, dev, scale=0.25)          # R = K copies: every rank's own tensors
+    torch.cuda.synchronize()
+    want, _, _, _ = H.run_oracle_path(oracle, wl, host, shares, scale=0.25)
+    for r in range(wl.K):
+        for t in range(wl.T):
+            H.assert_bit_equal(dev[r][t], want[t], "rank %d tensor %d" % (r, t))
+    kt.kt_destroy(ctx)
+
+
 def test_sum_then_divide_coefficients(kt, oracle):
     """Plain sums across the hierarchy with one final division (weights a_r = b_r, W_g = 1,
     scale 1/B) through kt_set_coefficients; oracle fed the same coefficients."""
