@@ -397,6 +397,22 @@ def broadcast_phases(kt, wl, peak: float, chunk_bytes: int) -> dict:
             "ms_whole": round(t_all * 1e3, 4), "relay_bytes_down": N * es, "relay_bytes_up": N * es * (wl.G - 1)}
 
 
+def sampler_phase(kt, shares, peak: float, dataset_size: int = 1281167) -> dict:
+    """The load-adaptive sampler's index kernel on an ImageNet-sized epoch (1 281 167 indices)
+    with the step's shares: every index read once from the epoch's permutation and written once
+    into its rank's list."""
+    perm = torch.randperm(dataset_size, device="cuda")
+    steps = kt.kt_sampler_steps(dataset_size, sum(shares), False)
+    out = [torch.empty(steps * b, dtype=torch.int64, device="cuda") for b in shares]
+    main = torch.cuda.Stream()
+    with torch.cuda.stream(main):
+        sec = time_launches(lambda: kt.kt_sampler_indices(perm, dataset_size, shares, out, stream=main), main, 20)
+    nbytes = 16 * steps * sum(shares)
+    return {"what": "index lists of one epoch of %d samples for shares %s" % (dataset_size, list(shares)),
+            "k_sampler": {"us": round(sec * 1e6, 2), "GBps": round(nbytes / sec / 1e9, 1), "frac": round(nbytes / sec / 1e9 / peak, 4),
+                          "bytes": nbytes, "note": "20 MB once per epoch: two to three times the fixed cost of a launch; not on the per-step path"}}
+
+
 def narrow_transport_step(kt, wl, chunk_bytes: int, steps: int) -> dict:
     """The same step with the library's bf16 transport (an extension: partials rounded once
     to bf16, half the bytes on the host link).  Reported beside the headline, never as it."""
@@ -690,6 +706,7 @@ def run_ours(args) -> dict:
         result["configs"] = named_config_rows(kt, peak)
         result["broadcast"] = broadcast_phases(kt, wl, peak, args_chunk(args))
         result["bf16_transport"] = narrow_transport_step(kt, wl, args_chunk(args), min(args.steps, 20))
+        result["sampler"] = sampler_phase(kt, prob.shares, peak)
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         result["cpu_baseline"] = cpu_baseline(wl, prob.shares, budget_s=args.cpu_seconds)
     if dist is not None:
