@@ -30,7 +30,7 @@ EXPORTS = ["kt_schedule", "kt_scores", "kt_adapt_create", "kt_adapt_observe", "k
            "kt_get_coefficients", "kt_set_transport_dtype", "kt_route", "kt_bucket_pack", "kt_plan_buckets", "kt_plan_query", "kt_hier_reduce",
            "kt_stage_to_host", "kt_relay_through_host", "kt_stage_wait", "kt_unpack_scale", "kt_sync_direct", "kt_allreduce", "kt_bcast_send", "kt_bcast_relay", "kt_bcast_recv", "kt_cast", "kt_copy_tensors", "kt_sync_flat_static", "kt_launch_count",
            "kt_last_error", "kt_destroy", "kt_work_unit", "kt_shard_ranges", "kt_shard_bind", "kt_shard_query",
-           "kt_ipc_export", "kt_ipc_open", "kt_ipc_close", "kt_host_register", "kt_host_unregister", "kt_host_barrier"]
+           "kt_ipc_export", "kt_ipc_open", "kt_ipc_close", "kt_host_register", "kt_host_unregister", "kt_host_barrier", "kt_shard_step"]
 
 _DTYPES = {torch.float32: KT_F32, torch.bfloat16: KT_BF16}
 
@@ -97,6 +97,7 @@ def _load() -> C.CDLL:
         "kt_host_register": ([vp, C.c_int64], C.c_int),
         "kt_host_unregister": ([vp], C.c_int),
         "kt_host_barrier": ([vp, C.c_int, C.c_int], C.c_int),
+        "kt_shard_step": ([vp, vp, vpp, vpp, vpp, C.c_int, C.c_int, C.c_float, C.c_int, vp, vp, C.c_int], C.c_int),
         "kt_launch_count": ([vp], C.c_int64),
         "kt_last_error": ([vp], C.c_char_p),
         "kt_destroy": ([vp], None),
@@ -429,6 +430,21 @@ def kt_host_barrier(address: int, n_ranks: int, timeout_ms: int = -1) -> None:
     """Barrier between the processes of a node on a zeroed, 64-byte aligned block of shared host
     memory; raises KtError(KT_ERR_TIMEOUT) when the others do not arrive in time."""
     _check(_lib.kt_host_barrier(C.c_void_p(int(address)), int(n_ranks), int(timeout_ms)))
+
+
+def kt_shard_step(ctx: Ctx, barrier_address: int, partials: Optional[Ptrs], host_shared: Optional[Ptrs],
+                  out_grads: PtrArray, R: int, out_dtype: int, scale: float = 1.0, per_bucket: bool = True,
+                  main_stream=None, side_stream=None, timeout_ms: int = -1) -> None:
+    """One whole step of a rank-bound context; blocks until every rank has finished it."""
+    pa = kt_ptrs(partials) if partials is not None else None
+    hs = kt_ptrs(host_shared) if host_shared is not None else None
+    if out_grads.n != R * ctx.T:
+        raise KtError(KT_ERR_SHAPE, "expected %d output pointers" % (R * ctx.T))
+    _check(_lib.kt_shard_step(ctx.handle, C.c_void_p(int(barrier_address)), pa.array if pa is not None else None,
+                              hs.array if hs is not None else None, out_grads.array, int(R), int(out_dtype),
+                              C.c_float(scale), int(bool(per_bucket)), _stream(main_stream), _stream(side_stream),
+                              int(timeout_ms)))
+    ctx._keep["out"] = out_grads
 
 
 def kt_plan_buckets(numel: Sequence[int], bucket_cap_bytes: int) -> Plan:

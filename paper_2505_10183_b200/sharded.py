@@ -7,7 +7,7 @@ holds no arithmetic.  It moves handles and names between the processes with
 group mates' gradient and output tensors into this process (``kt_ipc_open``), maps one block of
 host memory that all processes of the node share (POSIX shared memory, page-locked with
 ``kt_host_register``; it also holds the block of ``kt_host_barrier``, where the ranks meet
-during a step), and then issues the library calls of a step in order:
+during a step), and then runs steps, each one library call (``kt_shard_step``) that does, in order:
 
     barrier                         every rank's gradients are complete
     kt_hier_reduce(KT_INTRA)        my share of each bucket, read from all members of my group
@@ -137,32 +137,13 @@ class ShardedSync:
         return kt.kt_shard_query(self.ctx, bucket)[:2]
 
     def step(self, scale: float = 1.0) -> None:
-        """One synchronisation.  On return this rank's `outs` hold the reduced gradients and every
-        other rank has finished reading this rank's `grads`."""
-        ctx = self.ctx
-        torch.cuda.synchronize()                      # whatever produced my gradients is done
-        self.barrier()
-        if self.G == 1:
-            for b in self.buckets:
-                kt.kt_sync_direct(ctx, self.out_ptrs, scale=scale, bucket=b, out_dtype=self.out_dtype,
-                                  R=len(self.members), stream=self.main)
-        else:
-            for b in self.buckets:
-                kt.kt_hier_reduce(ctx, kt.KT_INTRA, self.partial_rows, bucket=b, stream=self.main)
-                kt.kt_stage_to_host(ctx, kt.KT_D2H, self.partial_rows, self.host_rows, bucket=b,
-                                    main_stream=self.main, side_stream=self.side)
-            for b in self.buckets:                    # my shares are in host memory ...
-                kt.kt_stage_wait(ctx, kt.KT_D2H, bucket=b, main_stream=self.main, timeout_ms=self.wait_ms)
-            self.barrier()                            # ... and so are everybody else's
-            for b in self.buckets:
-                kt.kt_stage_to_host(ctx, kt.KT_H2D, self.partial_rows, self.host_rows, bucket=b,
-                                    main_stream=self.main, side_stream=self.side)
-            for b in self.buckets:
-                kt.kt_stage_wait(ctx, kt.KT_H2D, bucket=b, main_stream=self.main)
-                kt.kt_unpack_scale(ctx, self.partial_rows, self.out_ptrs, scale=scale, bucket=b,
-                                   out_dtype=self.out_dtype, R=len(self.members), stream=self.main)
-        self.main.synchronize()                       # my shares are written everywhere in my group
-        self.barrier()
+        """One synchronisation (kt_shard_step: the whole sequence of the module's header in one
+        library call).  On return this rank's `outs` hold the reduced gradients and every other
+        rank has finished reading this rank's `grads`."""
+        kt.kt_shard_step(self.ctx, self._host_address, self.partial_rows if self.G > 1 else None, self.host_rows,
+                         self.out_ptrs, len(self.members), self.out_dtype, scale=scale,
+                         per_bucket=self.buckets != [-1], main_stream=self.main, side_stream=self.side,
+                         timeout_ms=self.wait_ms)
 
     def close(self, meet: bool = True) -> None:
         """Unmaps everything.  meet=False skips the barrier in the shared block: for ranks that
