@@ -289,8 +289,9 @@ def leaving_rank_main(rank, world, port):
     host = [[W.as_numpy(t) for t in W.split_tensors(W.rank_gradients(wl, r, "cpu"), wl.numel)] for r in range(wl.K)]
     mine = [t.cuda() for t in W.split_tensors(W.rank_gradients(wl, rank, "cpu"), wl.numel)]
     outs = [torch.full((m,), float("nan"), device="cuda") for m in wl.numel]
-    job = ShardedSync(rank, wl.group_of, wl.shares, mine, outs, wl.bucket_cap_bytes, wait_ms=400)
+    job = ShardedSync(rank, wl.group_of, wl.shares, mine, outs, wl.bucket_cap_bytes)
     job.step()                                              # everybody takes part in the first step
+    job.wait_ms = 400                                       # from now on a rank is missed after 0.4 s
     want, _, _, _ = oracle.sync_step(host, wl.numel, 0, wl.group_of, wl.shares, wl.G, wl.bucket_cap_bytes)
     for t in range(wl.T):
         H.assert_bit_equal(outs[t], want[t], "rank %d out[%d]" % (rank, t))
