@@ -89,3 +89,19 @@ def test_asking_for_more_gpus_than_there_are_fails_loudly():
                           stdout=subprocess.PIPE, stderr=subprocess.PIPE, text=True,
                           env=dict(os.environ, WORLD_SIZE="2", RANK="0", LOCAL_RANK="0"))
     assert proc.returncode != 0 and "disagrees with WORLD_SIZE=2" in proc.stderr
+
+
+def test_nccl_start_up_log_is_summarised(tmp_path, monkeypatch):
+    """What the benchmark reports about the communicator comes from NCCL's own start-up log."""
+    sys.path.insert(0, ROOT)
+    import bench
+    log = tmp_path / ("nccl_host_%d.log" % os.getpid())
+    log.write_text("host:1:1 [0] NCCL INFO NCCL version 2.28.9+cuda12.9\n"
+                   "host:1:2 [0] NCCL INFO comm 0x55 rank 0 nranks 4 cudaDev 0 nvmlDev 0 busId 1000 commId 0x1 - Init START\n"
+                   "host:1:2 [0] NCCL INFO NVLS multicast support is available on dev 0\n"
+                   "host:1:2 [0] NCCL INFO comm 0x55 rank 0 nranks 4 cudaDev 0 - Init COMPLETE\n")
+    monkeypatch.setenv("NCCL_DEBUG_FILE", str(tmp_path / "nccl_%h_%p.log"))
+    got = bench.nccl_log_summary()
+    assert got["nranks"] == 4 and got["version"].startswith("2.28.9") and got["nvls"] is True
+    monkeypatch.setenv("NCCL_DEBUG_FILE", str(tmp_path / "absent_%h_%p.log"))
+    assert bench.nccl_log_summary() == {}
