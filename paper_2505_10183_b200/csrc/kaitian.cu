@@ -1106,14 +1106,19 @@ int kt_stage_wait(kt_ctx *c, int dir, int bucket, void *main_stream, int timeout
     if (!slot.recorded) return fail(KT_ERR_STATE, "no staging copy queued for direction %d, bucket %d", dir, bucket);
     KT_CUDA(cudaStreamWaitEvent(static_cast<cudaStream_t>(main_stream), slot.done, 0));
     if (timeout_ms < 0) return KT_OK;
-    const auto deadline = std::chrono::steady_clock::now() + std::chrono::milliseconds(timeout_ms);
+    // poll back to back for the first 300 us (a bucket's share crosses the link in about that
+    // time), then with short sleeps, then with longer ones
+    const auto begin = std::chrono::steady_clock::now();
+    const auto deadline = begin + std::chrono::milliseconds(timeout_ms);
     for (;;) {
         const cudaError_t e = cudaEventQuery(slot.done);
         if (e == cudaSuccess) return KT_OK;
         if (e != cudaErrorNotReady) return fail(KT_ERR_CUDA, "cudaEventQuery: %s", cudaGetErrorString(e));
-        if (std::chrono::steady_clock::now() >= deadline)
+        const auto now = std::chrono::steady_clock::now();
+        if (now >= deadline)
             return fail(KT_ERR_TIMEOUT, "staging copy (direction %d, bucket %d) not finished after %d ms", dir, bucket, timeout_ms);
-        std::this_thread::sleep_for(std::chrono::microseconds(50));
+        if (now - begin < std::chrono::microseconds(300)) continue;
+        std::this_thread::sleep_for(std::chrono::microseconds(now - begin < std::chrono::milliseconds(5) ? 20 : 200));
     }
 }
 
