@@ -236,8 +236,9 @@ int kt_plan_query(const kt_ctx *ctx, int32_t *n_buckets, int64_t *bucket_start,
  *            (peer-mapped again) every member receives this member's share of the result,
  *            so that after all members have run, and a barrier, every rank holds the whole
  *            reduced gradient.  kt_sync_direct needs G == 1 (it reads all ranks).
- *          - kt_relay_through_host, kt_allreduce across groups, the broadcast calls and the
- *            standalone pack return KT_ERR_STATE.
+ *          - the broadcast calls take this rank's part in a broadcast (see kt_shard_bcast);
+ *          - kt_relay_through_host, kt_allreduce across groups and the standalone pack return
+ *            KT_ERR_STATE.
  *        Per element the arithmetic and its order are unchanged: results are bit-identical to
  *        the unsharded calls.  Ranks synchronise on the host (barriers); no kernel waits for
  *        another device.  Errors: KT_ERR_INVALID.
@@ -307,6 +308,29 @@ int kt_host_barrier(void *shared, int n_ranks, int timeout_ms);
 int kt_shard_step(kt_ctx *ctx, void *barrier_block, float *const *partials, float *const *host_shared,
                   void *const *out_grads, int R, int out_dtype, float scale, int per_bucket,
                   void *main_stream, void *side_stream, int timeout_ms);
+
+/* Model synchronisation with one rank per device (the Broadcast of Section III routed through
+ * the hierarchy of Section III-A): rank `root`'s registered tensors reach the registered tensors
+ * of every other rank, bit for bit.  On a rank-bound context the three broadcast calls take the
+ * part that this rank has in it and are no-ops otherwise:
+ *   kt_bcast_send   the root alone: one pass over its tensors (the whole range, not a share)
+ *                   into its flat send buffer and, by peer stores, into its group mates' tensors;
+ *   kt_bcast_relay  the root: copies the range of `send` into `host_pinned` (memory all ranks
+ *                   map); a rank of another group: copies ITS SHARE of `host_pinned` into
+ *                   recv[own group]; between the two the caller needs a barrier across ranks;
+ *                   completion is what kt_stage_wait(KT_D2H / KT_H2D, bucket) waits for;
+ *   kt_bcast_recv   a rank of another group: unpacks its share of recv[own group] into the
+ *                   tensors of every member of its group (peer stores), so that after all
+ *                   members have run every tensor is complete.
+ * kt_shard_bcast is the whole sequence in one blocking call, like kt_shard_step: barrier ->
+ * root sends and copies down, waits -> barrier -> the other groups' ranks copy their shares up
+ * and unpack -> wait for the own stream, barrier.
+ *   send (device, root only), recv (device, ranks outside the root's group): flat buffers of
+ *        transport_numel elements of the registered dtype, 16-byte aligned;
+ *   host_shared (host): the same size, page-locked, mapped by all ranks (NULL with one group).
+ * Errors: those of the parts. */
+int kt_shard_bcast(kt_ctx *ctx, int root, void *barrier_block, void *send, void *host_shared, void *recv,
+                   int per_bucket, void *main_stream, void *d2h_stream, void *h2d_stream, int timeout_ms);
 
 /* The two reductions of Section III-A.
  * transport: host array of G device pointers, fp32, transport_numel elements each,

@@ -30,7 +30,7 @@ EXPORTS = ["kt_schedule", "kt_scores", "kt_adapt_create", "kt_adapt_observe", "k
            "kt_get_coefficients", "kt_set_transport_dtype", "kt_route", "kt_bucket_pack", "kt_plan_buckets", "kt_plan_query", "kt_hier_reduce",
            "kt_stage_to_host", "kt_relay_through_host", "kt_stage_wait", "kt_unpack_scale", "kt_sync_direct", "kt_allreduce", "kt_bcast_send", "kt_bcast_relay", "kt_bcast_recv", "kt_cast", "kt_copy_tensors", "kt_sync_flat_static", "kt_launch_count",
            "kt_last_error", "kt_destroy", "kt_work_unit", "kt_shard_ranges", "kt_shard_bind", "kt_shard_query",
-           "kt_ipc_export", "kt_ipc_open", "kt_ipc_close", "kt_host_register", "kt_host_unregister", "kt_host_barrier", "kt_shard_step"]
+           "kt_ipc_export", "kt_ipc_open", "kt_ipc_close", "kt_host_register", "kt_host_unregister", "kt_host_barrier", "kt_shard_step", "kt_shard_bcast"]
 
 _DTYPES = {torch.float32: KT_F32, torch.bfloat16: KT_BF16}
 
@@ -98,6 +98,7 @@ def _load() -> C.CDLL:
         "kt_host_unregister": ([vp], C.c_int),
         "kt_host_barrier": ([vp, C.c_int, C.c_int], C.c_int),
         "kt_shard_step": ([vp, vp, vpp, vpp, vpp, C.c_int, C.c_int, C.c_float, C.c_int, vp, vp, C.c_int], C.c_int),
+        "kt_shard_bcast": ([vp, C.c_int, vp, vp, vp, vp, C.c_int, vp, vp, vp, C.c_int], C.c_int),
         "kt_launch_count": ([vp], C.c_int64),
         "kt_last_error": ([vp], C.c_char_p),
         "kt_destroy": ([vp], None),
@@ -447,6 +448,17 @@ def kt_shard_step(ctx: Ctx, barrier_address: int, partials: Optional[Ptrs], host
     ctx._keep["out"] = out_grads
 
 
+def kt_shard_bcast(ctx: Ctx, root: int, barrier_address: int, send_address: int, host_address: int,
+                   recv_address: int, per_bucket: bool, main_stream, d2h_stream, h2d_stream,
+                   timeout_ms: int = -1) -> None:
+    """Broadcast of rank `root`'s registered tensors to every rank (rank-bound contexts); blocks
+    until every rank has finished.  Addresses may be 0 where the header allows NULL."""
+    _check(_lib.kt_shard_bcast(ctx.handle, int(root), C.c_void_p(int(barrier_address)),
+                               C.c_void_p(int(send_address) or None), C.c_void_p(int(host_address) or None),
+                               C.c_void_p(int(recv_address) or None), int(bool(per_bucket)), _stream(main_stream),
+                               _stream(d2h_stream), _stream(h2d_stream), int(timeout_ms)))
+
+
 def kt_plan_buckets(numel: Sequence[int], bucket_cap_bytes: int) -> Plan:
     T = len(numel)
     n = (C.c_int64 * max(T, 1))(*[int(v) for v in numel])
@@ -583,10 +595,12 @@ def kt_bcast_send(ctx: Ctx, root: int, send: torch.Tensor, bucket: int = -1, str
     _check(_lib.kt_bcast_send(ctx.handle, int(root), int(bucket), C.c_void_p(send.data_ptr()), _stream(stream)))
 
 
-def kt_bcast_relay(ctx: Ctx, root: int, send: torch.Tensor, host_pinned: torch.Tensor,
+def kt_bcast_relay(ctx: Ctx, root: int, send: Optional[torch.Tensor], host_pinned: torch.Tensor,
                    recv: Sequence[Optional[torch.Tensor]], d2h_stream, h2d_stream, bucket: int = -1,
                    chunk_bytes: int = 4 << 20, main_stream=None) -> None:
-    _check(_lib.kt_bcast_relay(ctx.handle, int(root), int(bucket), C.c_void_p(send.data_ptr()),
+    """send may be None on a rank-bound context that is not the root's."""
+    _check(_lib.kt_bcast_relay(ctx.handle, int(root), int(bucket),
+                               C.c_void_p(send.data_ptr()) if send is not None else None,
                                C.c_void_p(host_pinned.data_ptr()), _recv_array(ctx, recv), int(chunk_bytes),
                                _stream(main_stream), _stream(d2h_stream), _stream(h2d_stream)))
 

@@ -313,15 +313,18 @@ int64_t unit_start(const kt_ctx *c, int tile) {
 }
 
 // tile range of a bucket (or of everything for bucket == -1)
-int make_tile_plan(const kt_ctx *c, int bucket, TilePlan *tp) {
+// whole: the full range even on a context bound to one rank (the root of a broadcast sends
+// everything, not a share)
+int make_tile_plan(const kt_ctx *c, int bucket, TilePlan *tp, bool whole = false) {
     if (bucket < -1 || bucket >= static_cast<int>(c->bucket_start.size()))
         return fail(KT_ERR_SHAPE, "bucket %d out of range [-1, %d)", bucket, (int)c->bucket_start.size());
+    const bool share = sharded(c) && !whole;
     int t0, t1;
-    unit_range(c, bucket, sharded(c) ? c->shard_member : -1, &t0, &t1);
+    unit_range(c, bucket, share ? c->shard_member : -1, &t0, &t1);
     tp->prefix = c->d_prefix;
     tp->info = c->d_info;
     tp->T = c->T;
-    if (sharded(c)) {            // the tensors that hold the share's first and last unit
+    if (share) {                 // the tensors that hold the share's first and last unit
         tp->u_lo = t1 > t0 ? tensor_of_unit(c, t0) : 0;
         tp->u_hi = t1 > t0 ? tensor_of_unit(c, t1 - 1) + 1 : 0;
     } else {
@@ -340,8 +343,8 @@ int make_tile_plan(const kt_ctx *c, int bucket, TilePlan *tp) {
     return KT_OK;
 }
 
-void bucket_range(const kt_ctx *c, int bucket, int64_t *lo, int64_t *n) {
-    if (sharded(c)) {
+void bucket_range(const kt_ctx *c, int bucket, int64_t *lo, int64_t *n, bool whole = false) {
+    if (sharded(c) && !whole) {
         int t0, t1;
         unit_range(c, bucket, c->shard_member, &t0, &t1);
         *lo = unit_start(c, t0);
@@ -1453,6 +1456,54 @@ int kt_shard_step(kt_ctx *c, void *barrier_block, float *const *partials, float 
     return kt_host_barrier(barrier_block, c->K, timeout_ms);
 }
 
+int kt_shard_bcast(kt_ctx *c, int root, void *barrier_block, void *send, void *host_shared, void *recv,
+                   int per_bucket, void *main_stream, void *d2h_stream, void *h2d_stream, int timeout_ms) {
+    if (int rc = check_ctx(c, true)) return rc;
+    if (!sharded(c)) return fail(KT_ERR_STATE, "kt_shard_bind has not been called on this context");
+    if (root < 0 || root >= c->K) return fail(KT_ERR_INVALID, "root = %d outside [0, %d)", root, c->K);
+    if (!barrier_block) return fail(KT_ERR_INVALID, "barrier_block is NULL");
+    const bool is_root = c->shard_rank == root, roots_group = c->group_of[root] == c->shard_g;
+    if (is_root && !send) return fail(KT_ERR_INVALID, "send is NULL");
+    if (c->G > 1 && !host_shared) return fail(KT_ERR_INVALID, "host_shared is NULL");
+    if (!roots_group && !recv) return fail(KT_ERR_INVALID, "recv is NULL");
+    const int nb = static_cast<int>(c->bucket_start.size());
+    const int first = per_bucket ? 0 : -1, past = per_bucket ? nb : 0;
+    const int64_t chunk = int64_t(1) << 40;                  // each half is one copy per range
+    void *recv_rows[KT_MAX_GROUPS] = {};
+    recv_rows[c->shard_g] = recv;
+    {
+        KT_ON_DEVICE(c->device);
+        KT_CUDA(cudaDeviceSynchronize());                     // nothing on this device still touches the tensors
+    }
+    if (int rc = kt_host_barrier(barrier_block, c->K, timeout_ms)) return rc;
+    if (is_root) {
+        for (int b = first; b < past; ++b) {
+            if (int rc = kt_bcast_send(c, root, b, send, main_stream)) return rc;
+            if (c->G > 1)
+                if (int rc = kt_bcast_relay(c, root, b, send, host_shared, recv_rows, chunk, main_stream, d2h_stream, h2d_stream))
+                    return rc;
+        }
+        if (c->G > 1)
+            for (int b = first; b < past; ++b)
+                if (int rc = kt_stage_wait(c, KT_D2H, b, main_stream, timeout_ms < 0 ? 3600 * 1000 : timeout_ms)) return rc;
+    }
+    if (int rc = kt_host_barrier(barrier_block, c->K, timeout_ms)) return rc;   // the root's tensors are in host memory
+    if (!roots_group) {
+        for (int b = first; b < past; ++b)
+            if (int rc = kt_bcast_relay(c, root, b, nullptr, host_shared, recv_rows, chunk, main_stream, d2h_stream, h2d_stream))
+                return rc;
+        for (int b = first; b < past; ++b) {
+            if (int rc = kt_stage_wait(c, KT_H2D, b, main_stream, -1)) return rc;
+            if (int rc = kt_bcast_recv(c, root, b, recv_rows, main_stream)) return rc;
+        }
+    }
+    {
+        KT_ON_DEVICE(c->device);
+        KT_CUDA(cudaStreamSynchronize(static_cast<cudaStream_t>(main_stream)));
+    }
+    return kt_host_barrier(barrier_block, c->K, timeout_ms);
+}
+
 int64_t kt_launch_count(const kt_ctx *c) { return c ? c->launches : 0; }
 
 const char *kt_last_error(const kt_ctx *) { return g_err; }
@@ -1681,9 +1732,28 @@ int kt_sampler_indices(const int64_t *list, int64_t dataset_size, const int32_t 
 namespace {
 
 int fill_bcast(const kt_ctx *c, int root, BcastParams *p) {
-    if (sharded(c)) return fail(KT_ERR_STATE, "the broadcast is not available on a context bound to one rank");
     if (root < 0 || root >= c->K) return fail(KT_ERR_INVALID, "root = %d outside [0, %d)", root, c->K);
     p->ptrs = const_cast<void *const *>(reinterpret_cast<const void *const *>(c->d_ptrs));
+    if (sharded(c)) {
+        // The pointer table holds the M members of this rank's group only.  The kernels see two
+        // "groups": 0 is the root's side (the members, when this rank's group is the root's; empty
+        // otherwise), 1 the receiving side (the members, when it is not).
+        p->G = 2;
+        p->g_root = 0;
+        p->k_root = 0;
+        const bool roots_group = c->group_of[root] == c->shard_g;
+        p->k_lo[0] = 0;
+        p->k_hi[0] = static_cast<unsigned char>(roots_group ? c->shard_M : 0);
+        p->k_lo[1] = 0;
+        p->k_hi[1] = static_cast<unsigned char>(roots_group ? 0 : c->shard_M);
+        if (roots_group)
+            for (int r = 0, m = 0; r < c->K; ++r) {
+                if (c->group_of[r] != c->shard_g) continue;
+                if (r == root) p->k_root = m;
+                ++m;
+            }
+        return KT_OK;
+    }
     p->G = c->G;
     p->g_root = c->group_of[root];
     for (int g = 0; g < c->G; ++g) p->k_lo[g] = p->k_hi[g] = 0;
@@ -1706,7 +1776,8 @@ int kt_bcast_send(kt_ctx *c, int root, int bucket, void *send, void *stream) {
     if (!aligned16(send)) return fail(KT_ERR_ALIGN, "send is not 16-byte aligned");
     BcastParams p{};
     if (int rc = fill_bcast(c, root, &p)) return rc;
-    if (int rc = make_tile_plan(c, bucket, &p.tp)) return rc;
+    if (sharded(c) && c->shard_rank != root) return KT_OK;      // only the root's own device sends
+    if (int rc = make_tile_plan(c, bucket, &p.tp, true)) return rc;
     if (p.tp.n_tiles == 0) return KT_OK;
     p.flat[p.g_root] = send;
     KT_ON_DEVICE(c->device);
@@ -1723,11 +1794,21 @@ int kt_bcast_recv(kt_ctx *c, int root, int bucket, void *const *recv, void *stre
     if (!recv) return fail(KT_ERR_INVALID, "recv is NULL");
     BcastParams p{};
     if (int rc = fill_bcast(c, root, &p)) return rc;
-    for (int g = 0; g < c->G; ++g) {
-        if (g == p.g_root) continue;
-        if (!recv[g]) return fail(KT_ERR_INVALID, "recv[%d] is NULL", g);
-        if (!aligned16(recv[g])) return fail(KT_ERR_ALIGN, "recv[%d] is not 16-byte aligned", g);
-        p.flat[g] = recv[g];
+    if (sharded(c)) {
+        // a rank of another group unpacks its share of its group's receive buffer into the tensors
+        // of every member; the ranks of the root's group were written by the root itself
+        if (c->group_of[root] == c->shard_g) return KT_OK;
+        void *mine = recv[c->shard_g];
+        if (!mine) return fail(KT_ERR_INVALID, "recv[%d] is NULL", c->shard_g);
+        if (!aligned16(mine)) return fail(KT_ERR_ALIGN, "recv[%d] is not 16-byte aligned", c->shard_g);
+        p.flat[1] = mine;
+    } else {
+        for (int g = 0; g < c->G; ++g) {
+            if (g == p.g_root) continue;
+            if (!recv[g]) return fail(KT_ERR_INVALID, "recv[%d] is NULL", g);
+            if (!aligned16(recv[g])) return fail(KT_ERR_ALIGN, "recv[%d] is not 16-byte aligned", g);
+            p.flat[g] = recv[g];
+        }
     }
     if (int rc = make_tile_plan(c, bucket, &p.tp)) return rc;
     if (p.tp.n_tiles == 0 || c->G == 1) return KT_OK;
@@ -1743,13 +1824,42 @@ int kt_bcast_recv(kt_ctx *c, int root, int bucket, void *const *recv, void *stre
 int kt_bcast_relay(kt_ctx *c, int root, int bucket, const void *send, void *host_pinned, void *const *recv,
                    int64_t chunk_bytes, void *main_stream, void *d2h_stream, void *h2d_stream) {
     if (int rc = check_ctx(c, true)) return rc;
-    if (!send || !host_pinned || !recv) return fail(KT_ERR_INVALID, "NULL argument");
-    if (sharded(c)) return fail(KT_ERR_STATE, "the broadcast is not available on a context bound to one rank");
+    if (!host_pinned) return fail(KT_ERR_INVALID, "host_pinned is NULL");
     if (root < 0 || root >= c->K) return fail(KT_ERR_INVALID, "root = %d outside [0, %d)", root, c->K);
     if (bucket < -1 || bucket >= static_cast<int>(c->bucket_start.size()))
         return fail(KT_ERR_SHAPE, "bucket %d out of range", bucket);
     if (chunk_bytes < 256) return fail(KT_ERR_INVALID, "chunk_bytes must be >= 256");
     if (d2h_stream == h2d_stream) return fail(KT_ERR_INVALID, "the two copy streams must differ");
+    if (sharded(c)) {
+        // One half per role, the caller's barrier between them: the root copies the whole range
+        // down; a rank of another group copies its share up; the root's group mates do nothing.
+        const bool is_root = c->shard_rank == root, roots_group = c->group_of[root] == c->shard_g;
+        if (!is_root && roots_group) return KT_OK;
+        if (is_root && !send) return fail(KT_ERR_INVALID, "send is NULL");
+        if (!is_root && (!recv || !recv[c->shard_g])) return fail(KT_ERR_INVALID, "recv[%d] is NULL", c->shard_g);
+        int64_t lo, n;
+        bucket_range(c, bucket, &lo, &n, is_root);
+        const size_t es = c->in_dtype == KT_F32 ? 4 : 2;
+        KT_ON_DEVICE(c->device);
+        cudaStream_t ms = static_cast<cudaStream_t>(main_stream);
+        cudaStream_t cs = static_cast<cudaStream_t>(is_root ? d2h_stream : h2d_stream);
+        KT_CUDA(cudaEventRecord(c->ev_main, ms));
+        KT_CUDA(cudaStreamWaitEvent(cs, c->ev_main, 0));
+        char *host = static_cast<char *>(host_pinned) + static_cast<size_t>(lo) * es;
+        if (n > 0) {
+            if (is_root)
+                KT_CUDA(cudaMemcpyAsync(host, static_cast<const char *>(send) + static_cast<size_t>(lo) * es,
+                                        static_cast<size_t>(n) * es, cudaMemcpyDeviceToHost, cs));
+            else
+                KT_CUDA(cudaMemcpyAsync(static_cast<char *>(recv[c->shard_g]) + static_cast<size_t>(lo) * es, host,
+                                        static_cast<size_t>(n) * es, cudaMemcpyHostToDevice, cs));
+        }
+        StageSlot &slot = c->slots[is_root ? KT_D2H : KT_H2D][bucket + 1];
+        KT_CUDA(cudaEventRecord(slot.done, cs));
+        slot.recorded = true;
+        return KT_OK;
+    }
+    if (!send || !recv) return fail(KT_ERR_INVALID, "NULL argument");
     const int g_root = c->group_of[root];
     for (int g = 0; g < c->G; ++g)
         if (g != g_root && !recv[g]) return fail(KT_ERR_INVALID, "recv[%d] is NULL", g);

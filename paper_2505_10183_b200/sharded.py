@@ -145,6 +145,18 @@ class ShardedSync:
                          per_bucket=self.buckets != [-1], main_stream=self.main, side_stream=self.side,
                          timeout_ms=self.wait_ms)
 
+    def broadcast(self, root: int) -> None:
+        """Model synchronisation: rank `root`'s `grads` tensors (here: parameters) reach the same
+        tensors of every other rank, bit for bit (kt_shard_bcast; blocks until all ranks are done)."""
+        if getattr(self, "_bcast_flat", None) is None:
+            n = max(self.plan.transport_numel, 1)
+            self._bcast_flat = torch.empty(n, dtype=self.grads[0].dtype, device=self.grads[0].device)
+            self._bcast_stream = torch.cuda.Stream()
+        flat = self._bcast_flat.data_ptr()
+        host = self._host_address + self._header if self.G > 1 else 0
+        kt.kt_shard_bcast(self.ctx, root, self._host_address, flat, host, flat, self.buckets != [-1], self.main,
+                          self.side, self._bcast_stream, timeout_ms=self.wait_ms)
+
     def close(self, meet: bool = True) -> None:
         """Unmaps everything.  meet=False skips the barrier in the shared block: for ranks that
         have seen a barrier time out (the block is then in an undefined state) and have made sure

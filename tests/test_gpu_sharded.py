@@ -162,6 +162,85 @@ def test_emulated_ranks_with_the_bf16_transport(kt, oracle, name):
     run_emulated(kt, oracle, wl, host, dev, torch.float32, 1.0, False, False, False, narrow=True)
 
 
+def run_emulated_broadcast(kt, oracle, wl, root, per_bucket, misalign=0):
+    """Model synchronisation with every rank a context of its own: the root sends (whole range)
+    and copies down; every rank of another group copies ITS SHARE up into a receive buffer of
+    its own and unpacks it into all members of its group; nobody else does anything."""
+    K, G = wl.K, wl.G
+    dt = H.ORACLE_DT[wl.dtype]
+    tdt = H.TORCH_DT[wl.dtype]
+    host, dev = H.device_gradients(wl, misalign=misalign)
+    members = [[r for r in range(K) if wl.group_of[r] == g] for g in range(G)]
+    ctxs = []
+    for r in range(K):
+        ctx = kt.kt_groups_init(wl.group_of, [1] * K, G)
+        kt.kt_shard_bind(ctx, r, wl.group_of)
+        kt.kt_bucket_pack(ctx, [dev[q] for q in members[wl.group_of[r]]], wl.bucket_cap_bytes)
+        ctxs.append(ctx)
+    plan = kt.kt_plan_query(ctxs[0])
+    n = plan.transport_numel
+    buckets = list(range(plan.n_buckets)) if per_bucket else [-1]
+    want, flat, _ = oracle.broadcast(host, root, wl.numel, dt, wl.bucket_cap_bytes)
+    send = torch.full((n,), 7.0, dtype=tdt, device="cuda")
+    shared = torch.full((n,), 7.0, dtype=tdt).pin_memory()
+    recvs = {r: torch.full((n,), 7.0, dtype=tdt, device="cuda") for r in range(K)}
+    s1, s2 = torch.cuda.Stream(), torch.cuda.Stream()
+    g_root = wl.group_of[root]
+    for b in buckets:                                   # the root's half
+        for r in range(K):                              # everybody may call; only the root acts
+            kt.kt_bcast_send(ctxs[r], root, send, bucket=b)
+        kt.kt_bcast_relay(ctxs[root], root, send, shared, [None] * G, s1, s2, bucket=b)
+        kt.kt_stage_wait(ctxs[root], kt.KT_D2H, bucket=b, timeout_ms=20000)
+    torch.cuda.synchronize()                            # stands for the barrier
+    H.assert_bit_equal(shared, flat, "what crossed the host")
+    for b in buckets:                                   # the other groups' half
+        for r in range(K):
+            if r == root:
+                continue
+            rows = [recvs[r] if g == wl.group_of[r] else None for g in range(G)]
+            kt.kt_bcast_relay(ctxs[r], root, None, shared, rows, s1, s2, bucket=b)
+            if wl.group_of[r] != g_root:
+                kt.kt_stage_wait(ctxs[r], kt.KT_H2D, bucket=b)
+            kt.kt_bcast_recv(ctxs[r], root, rows, bucket=b)
+    torch.cuda.synchronize()
+    for r in range(K):
+        for t in range(wl.T):
+            H.assert_bit_equal(dev[r][t], want[r][t], "rank %d tensor %d" % (r, t))
+    # a rank outside the root's group copied up its own share and nothing else
+    for r in range(K):
+        if wl.group_of[r] == g_root:
+            assert bool((recvs[r] == 7.0).all())
+            continue
+        mask = torch.zeros(n, dtype=torch.bool, device="cuda")
+        for b in buckets:
+            lo, cnt, _ = kt.kt_shard_query(ctxs[r], b)
+            mask[lo:lo + cnt] = True
+        assert bool((recvs[r][~mask] == 7.0).all())
+        m = mask.cpu().numpy()
+        assert np.array_equal(H.bits(W.as_numpy(recvs[r]))[m], H.bits(flat)[m])
+    for ctx in ctxs:
+        kt.kt_destroy(ctx)
+
+
+@pytest.mark.parametrize("name", ["tiny", "mobilenet_v2", "resnet18"])
+def test_emulated_ranks_broadcast_named_configurations(kt, oracle, name):
+    for dtype, root, per_bucket in (("f32", 0, False), ("bf16", None, True)):
+        wl = W.by_name(name)
+        wl.dtype = dtype
+        run_emulated_broadcast(kt, oracle, wl, wl.K - 1 if root is None else root, per_bucket)
+
+
+@pytest.mark.parametrize("seed", range(3))
+def test_emulated_ranks_broadcast_random_problems(kt, oracle, seed):
+    rnd = random.Random(9900 + seed)
+    for _ in range(12):
+        wl = TR.random_problem(rnd)
+        if rnd.random() < 0.4:
+            wl = W.Workload("random_long", wl.config_id, [(rnd.choice([5000, 20000, 70001]),) for _ in range(rnd.randint(1, 3))],
+                            wl.dtype, wl.group_of, wl.shares, bucket_cap_bytes=rnd.choice([40000, 1 << 20, 1 << 40]))
+        run_emulated_broadcast(kt, oracle, wl, rnd.randrange(wl.K), rnd.random() < 0.5, misalign=rnd.choice([0, 0, 1, 3]))
+
+
 def test_calls_that_need_all_ranks_are_refused_on_a_bound_context(kt):
     wl = W.tiny()
     _, dev = H.device_gradients(wl)
@@ -181,8 +260,7 @@ def test_calls_that_need_all_ranks_are_refused_on_a_bound_context(kt):
     s1, s2 = torch.cuda.Stream(), torch.cuda.Stream()
     for call in (lambda: kt.kt_relay_through_host(ctx, rows, pinned, rows, s1, s2),
                  lambda: kt.kt_sync_direct(ctx, out),
-                 lambda: kt.kt_allreduce(ctx, out, rows, pinned, rows, s1, s2),
-                 lambda: kt.kt_bcast_send(ctx, 0, rows[0])):
+                 lambda: kt.kt_allreduce(ctx, out, rows, pinned, rows, s1, s2)):
         with pytest.raises(kt.KtError) as e:
             call()
         assert e.value.status == kt.KT_ERR_STATE
@@ -320,3 +398,56 @@ def test_a_rank_that_stays_away_between_steps_is_noticed_on_the_host():
     if not torch.cuda.is_available():
         pytest.fail("this test needs a CUDA device")
     mp.spawn(leaving_rank_main, args=(4, 29600 + (os.getpid() * 11) % 2000), nprocs=4, join=True)
+
+
+BCAST_CASES = [
+    dict(wl="tiny", root=0, per_bucket=False),
+    dict(wl="tiny", root=3, per_bucket=True, dtype="bf16"),
+    dict(wl="mobilenet_v2", root=2, group_of=[0, 0, 1, 0, 1], per_bucket=True),
+    dict(wl="resnet18", root=1, per_bucket=True),
+    dict(wl="tiny", root=2, group_of=[0, 0, 0, 0], per_bucket=False),          # one group: no host relay at all
+]
+
+
+def bcast_rank_main(rank, world, port, cases):
+    sys.path.insert(0, ROOT)
+    sys.path.insert(0, os.path.join(ROOT, "tests"))
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    import torch.distributed as dist
+    from oracle import kt_oracle as oracle
+    from paper_2505_10183_b200.sharded import ShardedSync
+    torch.cuda.set_device(0)
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    for case in cases:
+        wl = W.by_name(case["wl"])
+        wl.dtype = case.get("dtype", wl.dtype)
+        if "group_of" in case:
+            wl.group_of = list(case["group_of"])
+        if wl.K != world:
+            continue
+        dt = H.ORACLE_DT[wl.dtype]
+        host = [[W.as_numpy(t) for t in W.split_tensors(W.rank_gradients(wl, r, "cpu"), wl.numel)] for r in range(wl.K)]
+        params = [t.cuda() for t in W.split_tensors(W.rank_gradients(wl, rank, "cpu"), wl.numel)]     # every rank starts with its own values
+        job = ShardedSync(rank, wl.group_of, [1] * wl.K, params, None, wl.bucket_cap_bytes, per_bucket=case["per_bucket"])
+        job.broadcast(case["root"])
+        want, _, _ = oracle.broadcast(host, case["root"], wl.numel, dt, wl.bucket_cap_bytes)
+        for t in range(wl.T):
+            H.assert_bit_equal(params[t], want[rank][t], "%s root %d: rank %d tensor %d" % (case["wl"], case["root"], rank, t))
+        job.broadcast(case["root"])                              # again: nothing may change
+        for t in range(wl.T):
+            H.assert_bit_equal(params[t], want[rank][t], "second broadcast: rank %d tensor %d" % (rank, t))
+        job.close()
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+@pytest.mark.parametrize("world", [4, 5])
+def test_broadcast_with_ranks_as_processes(world):
+    """Model synchronisation over IPC-mapped tensors and the shared host block: every rank starts
+    with its own values and must end with the root's, bit for bit."""
+    import torch.multiprocessing as mp
+    if not torch.cuda.is_available():
+        pytest.fail("this test needs a CUDA device")
+    cases = [c for c in BCAST_CASES if len(c.get("group_of", W.by_name(c["wl"]).group_of)) == world]
+    assert cases
+    mp.spawn(bcast_rank_main, args=(world, 29600 + (os.getpid() * 13 + world) % 2000, cases), nprocs=world, join=True)
