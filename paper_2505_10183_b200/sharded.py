@@ -145,6 +145,11 @@ class ShardedSync:
                          per_bucket=self.buckets != [-1], main_stream=self.main, side_stream=self.side,
                          timeout_ms=self.wait_ms)
 
+    def set_shares(self, shares: Sequence[int]) -> None:
+        """New batch shares (every rank calls this with the same list, between steps): the weights
+        of all later steps follow them (kt_set_shares)."""
+        kt.kt_set_shares(self.ctx, list(shares))
+
     def broadcast(self, root: int) -> None:
         """Model synchronisation: rank `root`'s `grads` tensors (here: parameters) reach the same
         tensors of every other rank, bit for bit (kt_shard_bcast; blocks until all ranks are done)."""
