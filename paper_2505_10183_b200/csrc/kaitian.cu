@@ -11,6 +11,11 @@
 //               multiples of 64, zero padding in the gaps
 //   tensor table  one 32-byte record per tensor (transport offset, numel, numel + padding,
 //               flags) and a prefix sum of TILE-sized work units per tensor
+//
+// One rank per device (kt_shard_bind): the same tables, but the pointer table holds the M
+// members of the rank's group only (its own tensors and its mates' peer-mapped ones), and every
+// launch and copy covers the member's share of the range: a contiguous run of work units
+// (unit_range), which is one contiguous element range of the transport (unit_start).
 
 #include "../../include/kaitian.h"
 
@@ -525,6 +530,23 @@ void forget_out_sets(kt_ctx *c) {
         o.dtype = -1;
         o.in_recording = false;
     }
+}
+
+// A range of n elements cut into chunks of `chunk` elements (the last one shorter).
+std::vector<int64_t> cut_chunks(int64_t n, int64_t chunk) {
+    std::vector<int64_t> sizes;
+    for (int64_t left = n; left > 0; left -= sizes.back()) sizes.push_back(left < chunk ? left : chunk);
+    return sizes;
+}
+
+// One event per chunk of a relay ("chunk k went down: its way up may start"), created on demand.
+int ensure_chunk_events(kt_ctx *c, size_t n_chunks) {
+    while (c->chunk_events.size() < n_chunks) {
+        cudaEvent_t e;
+        KT_CUDA(cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
+        c->chunk_events.push_back(e);
+    }
+    return KT_OK;
 }
 
 bool is_capturing(cudaStream_t s) {
@@ -1067,16 +1089,10 @@ int kt_relay_through_host(kt_ctx *c, int bucket, float *const *send, float *cons
     }
     // Uniform chunks (elements, a multiple of 64).  Shorter chunks at the two ends of the
     // pipeline were tried and measured slower: small copies use the host link badly.
-    const int64_t chunk = chunk_bytes / 256 * 256 / static_cast<int64_t>(es);
-    std::vector<int64_t> sizes;
-    for (int64_t left = n; left > 0; left -= sizes.back()) sizes.push_back(left < chunk ? left : chunk);
+    const std::vector<int64_t> sizes = cut_chunks(n, chunk_bytes / 256 * 256 / static_cast<int64_t>(es));
     const int64_t n_chunks = static_cast<int64_t>(sizes.size());
     KT_ON_DEVICE(c->device);
-    while (static_cast<int64_t>(c->chunk_events.size()) < n_chunks) {
-        cudaEvent_t e;
-        KT_CUDA(cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
-        c->chunk_events.push_back(e);
-    }
+    if (int rc = ensure_chunk_events(c, sizes.size())) return rc;
     cudaStream_t ms = static_cast<cudaStream_t>(main_stream);
     cudaStream_t ds = static_cast<cudaStream_t>(d2h_stream), hs = static_cast<cudaStream_t>(h2d_stream);
     KT_CUDA(cudaEventRecord(c->ev_main, ms));
@@ -1866,16 +1882,10 @@ int kt_bcast_relay(kt_ctx *c, int root, int bucket, const void *send, void *host
     int64_t lo, n;
     bucket_range(c, bucket, &lo, &n);
     const size_t es = c->in_dtype == KT_F32 ? 4 : 2;
-    const int64_t chunk = chunk_bytes / 256 * 256 / static_cast<int64_t>(es);   // elements per chunk
-    std::vector<int64_t> sizes;
-    for (int64_t left = n; left > 0; left -= sizes.back()) sizes.push_back(left < chunk ? left : chunk);
+    const std::vector<int64_t> sizes = cut_chunks(n, chunk_bytes / 256 * 256 / static_cast<int64_t>(es));
     const int64_t n_chunks = static_cast<int64_t>(sizes.size());
     KT_ON_DEVICE(c->device);
-    while (static_cast<int64_t>(c->chunk_events.size()) < n_chunks) {
-        cudaEvent_t e;
-        KT_CUDA(cudaEventCreateWithFlags(&e, cudaEventDisableTiming));
-        c->chunk_events.push_back(e);
-    }
+    if (int rc = ensure_chunk_events(c, sizes.size())) return rc;
     cudaStream_t ms = static_cast<cudaStream_t>(main_stream);
     cudaStream_t ds = static_cast<cudaStream_t>(d2h_stream), hs = static_cast<cudaStream_t>(h2d_stream);
     KT_CUDA(cudaEventRecord(c->ev_main, ms));
