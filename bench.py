@@ -879,6 +879,7 @@ def run_sharded(args) -> dict:
     seconds = float(t[0])
     if not all(bool(torch.isfinite(o).all()) and bool(o.any()) for o in outs if o.numel() > 64):
         raise RuntimeError("sharded arm: an output tensor was not written")
+    job_buckets = list(job.buckets)
     job.close()
     dist.destroy_process_group()
     if rank != 0:
@@ -892,7 +893,8 @@ def run_sharded(args) -> dict:
                        "bytes_counted": "per GPU: M*n*s read + 4*n written by the fused reduce over its share of n "
                                         "elements, 4*G*n read + M*n*s written by combine+unpack (M group members); "
                                         "summed over GPUs",
-                       "host_barriers_per_step": 3, "note": "timing includes the host-side barriers between ranks"}}
+                       "host_barriers_per_step": 2 + (len(job_buckets) if G > 1 else 0),
+                       "note": "timing includes the host-side barriers between ranks"}}
 
 
 # ----------------------------------------------------------------------------- the oracle as CPU baseline

@@ -287,19 +287,22 @@ int kt_host_barrier(void *shared, int n_ranks, int timeout_ms);
 
 /* One synchronisation step of a rank-bound context (kt_shard_bind), start to finish, in the
  * order of Section III-A / III-B step 3: barrier (all ranks' gradients are complete; this rank's
- * device is synchronised first) -> fused reduce over this member's share of every range ->
- * copy of the share into host memory all ranks map -> wait for the own copies, barrier -> copy
- * of the same element range of the other groups' partials up -> combine + scale + cast + unpack
- * of the share into the R = M output sets (this rank's and, peer-mapped, its group mates') ->
- * wait for the own stream, barrier.  With one group the middle is kt_sync_direct.
+ * device is synchronised first) -> fused reduce over this member's share of every range and,
+ * behind each, the copy of the share into host memory all ranks map (down_stream) -> then range
+ * by range: wait for the own copy, barrier (every rank's share of the range is down), copy of
+ * the same element range of the other groups' partials up (up_stream, while later ranges are
+ * still going down), combine + scale + cast + unpack of the share into the R = M output sets
+ * (this rank's and, peer-mapped, its group mates') -> wait for the own stream, barrier.  With
+ * one group the middle is kt_sync_direct.
  *   barrier_block (host): the kt_host_barrier block shared by all K ranks of kt_groups_init.
  *   partials: host array of G device pointers, this rank's rows of transport_numel elements
  *        (row of its own group: the share it reduces; other rows: what it receives).
  *   host_shared: host array of G pointers into page-locked host memory that all ranks map,
  *        the same layout in every process.  Both may be NULL with one group.
  *   out_grads, R, out_dtype, scale: as in kt_unpack_scale, R = number of group members.
- *   per_bucket != 0: one launch and one copy per bucket (copies of a bucket overlap the reduce
- *        of the next); 0: one range, the whole transport.
+ *   per_bucket != 0: the ranges are the buckets (2 + number of buckets barriers per step; both
+ *        directions of the host link work at the same time); 0: one range, the whole transport.
+ *   down_stream, up_stream: two different copy streams (ignored with one group).
  *   timeout_ms: limit of every barrier and of the wait for the own copies (< 0: none).
  * The call blocks the calling thread until the step is complete on every rank (it returns
  * after the last barrier).  On return the outputs of this rank hold the reduced gradients and no
@@ -307,7 +310,7 @@ int kt_host_barrier(void *shared, int n_ranks, int timeout_ms);
  * rank did not arrive (nothing is left running on this rank's device that waits for it). */
 int kt_shard_step(kt_ctx *ctx, void *barrier_block, float *const *partials, float *const *host_shared,
                   void *const *out_grads, int R, int out_dtype, float scale, int per_bucket,
-                  void *main_stream, void *side_stream, int timeout_ms);
+                  void *main_stream, void *down_stream, void *up_stream, int timeout_ms);
 
 /* Model synchronisation with one rank per device (the Broadcast of Section III routed through
  * the hierarchy of Section III-A): rank `root`'s registered tensors reach the registered tensors

@@ -97,7 +97,7 @@ def _load() -> C.CDLL:
         "kt_host_register": ([vp, C.c_int64], C.c_int),
         "kt_host_unregister": ([vp], C.c_int),
         "kt_host_barrier": ([vp, C.c_int, C.c_int], C.c_int),
-        "kt_shard_step": ([vp, vp, vpp, vpp, vpp, C.c_int, C.c_int, C.c_float, C.c_int, vp, vp, C.c_int], C.c_int),
+        "kt_shard_step": ([vp, vp, vpp, vpp, vpp, C.c_int, C.c_int, C.c_float, C.c_int, vp, vp, vp, C.c_int], C.c_int),
         "kt_shard_bcast": ([vp, C.c_int, vp, vp, vp, vp, C.c_int, vp, vp, vp, C.c_int], C.c_int),
         "kt_launch_count": ([vp], C.c_int64),
         "kt_last_error": ([vp], C.c_char_p),
@@ -435,7 +435,7 @@ def kt_host_barrier(address: int, n_ranks: int, timeout_ms: int = -1) -> None:
 
 def kt_shard_step(ctx: Ctx, barrier_address: int, partials: Optional[Ptrs], host_shared: Optional[Ptrs],
                   out_grads: PtrArray, R: int, out_dtype: int, scale: float = 1.0, per_bucket: bool = True,
-                  main_stream=None, side_stream=None, timeout_ms: int = -1) -> None:
+                  main_stream=None, down_stream=None, up_stream=None, timeout_ms: int = -1) -> None:
     """One whole step of a rank-bound context; blocks until every rank has finished it."""
     pa = kt_ptrs(partials) if partials is not None else None
     hs = kt_ptrs(host_shared) if host_shared is not None else None
@@ -443,8 +443,8 @@ def kt_shard_step(ctx: Ctx, barrier_address: int, partials: Optional[Ptrs], host
         raise KtError(KT_ERR_SHAPE, "expected %d output pointers" % (R * ctx.T))
     _check(_lib.kt_shard_step(ctx.handle, C.c_void_p(int(barrier_address)), pa.array if pa is not None else None,
                               hs.array if hs is not None else None, out_grads.array, int(R), int(out_dtype),
-                              C.c_float(scale), int(bool(per_bucket)), _stream(main_stream), _stream(side_stream),
-                              int(timeout_ms)))
+                              C.c_float(scale), int(bool(per_bucket)), _stream(main_stream), _stream(down_stream),
+                              _stream(up_stream), int(timeout_ms)))
     ctx._keep["out"] = out_grads
 
 

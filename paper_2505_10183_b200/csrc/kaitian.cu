@@ -1432,11 +1432,12 @@ int kt_host_barrier(void *shared, int n_ranks, int timeout_ms) {
 
 int kt_shard_step(kt_ctx *c, void *barrier_block, float *const *partials, float *const *host_shared,
                   void *const *out_grads, int R, int out_dtype, float scale, int per_bucket, void *main_stream,
-                  void *side_stream, int timeout_ms) {
+                  void *down_stream, void *up_stream, int timeout_ms) {
     if (int rc = check_ctx(c, true)) return rc;
     if (!sharded(c)) return fail(KT_ERR_STATE, "kt_shard_bind has not been called on this context");
     if (!barrier_block) return fail(KT_ERR_INVALID, "barrier_block is NULL");
     if (c->G > 1 && (!partials || !host_shared)) return fail(KT_ERR_INVALID, "partials and host_shared are needed with several groups");
+    if (c->G > 1 && down_stream == up_stream) return fail(KT_ERR_INVALID, "the two copy streams must differ");
     if (int rc = check_out_args(c, out_grads, R, out_dtype)) return rc;          // fail before the first barrier
     const int nb = static_cast<int>(c->bucket_start.size());
     const int first = per_bucket ? 0 : -1, past = per_bucket ? nb : 0;
@@ -1450,17 +1451,18 @@ int kt_shard_step(kt_ctx *c, void *barrier_block, float *const *partials, float 
         for (int b = first; b < past; ++b)
             if (int rc = kt_sync_direct(c, out_grads, R, out_dtype, scale, b, main_stream)) return rc;
     } else {
+        // all reduces are queued at once; the shares go down range by range behind them
         for (int b = first; b < past; ++b) {
             if (int rc = kt_hier_reduce(c, KT_INTRA, b, partials, nullptr, main_stream)) return rc;
-            if (int rc = kt_stage_to_host(c, KT_D2H, b, partials, host_shared, main_stream, side_stream)) return rc;
+            if (int rc = kt_stage_to_host(c, KT_D2H, b, partials, host_shared, main_stream, down_stream)) return rc;
         }
-        // a wait without limit would hide a dead device behind a dead rank: the copies get the same limit
-        for (int b = first; b < past; ++b)
-            if (int rc = kt_stage_wait(c, KT_D2H, b, main_stream, timeout_ms < 0 ? 3600 * 1000 : timeout_ms)) return rc;
-        if (int rc = kt_host_barrier(barrier_block, c->K, timeout_ms)) return rc; // every share of every group is down
-        for (int b = first; b < past; ++b)
-            if (int rc = kt_stage_to_host(c, KT_H2D, b, partials, host_shared, main_stream, side_stream)) return rc;
+        // range by range: once every rank's share of a range is in host memory its way up starts,
+        // on the other copy stream, while the later ranges are still on their way down
         for (int b = first; b < past; ++b) {
+            // a wait without limit would hide a dead device behind a dead rank: the copy gets the same limit
+            if (int rc = kt_stage_wait(c, KT_D2H, b, main_stream, timeout_ms < 0 ? 3600 * 1000 : timeout_ms)) return rc;
+            if (int rc = kt_host_barrier(barrier_block, c->K, timeout_ms)) return rc;
+            if (int rc = kt_stage_to_host(c, KT_H2D, b, partials, host_shared, main_stream, up_stream)) return rc;
             if (int rc = kt_stage_wait(c, KT_H2D, b, main_stream, -1)) return rc;
             if (int rc = kt_unpack_scale(c, partials, 0, out_grads, R, out_dtype, scale, b, main_stream)) return rc;
         }

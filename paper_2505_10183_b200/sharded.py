@@ -12,9 +12,10 @@ during a step), and then runs steps, each one library call (``kt_shard_step``) t
     barrier                         every rank's gradients are complete
     kt_hier_reduce(KT_INTRA)        my share of each bucket, read from all members of my group
     kt_stage_to_host(KT_D2H)        my share of my group's partial -> shared host memory
-    wait for my copies, barrier     every share of every group is in host memory
-    kt_stage_to_host(KT_H2D)        my element range of the other groups' partials -> device
-    kt_unpack_scale                 combine, scale, cast; my share written into the output
+    then bucket by bucket:
+      wait for my copy, barrier     every rank's share of the bucket is in host memory
+      kt_stage_to_host(KT_H2D)      my element range of the other groups' partials -> device
+      kt_unpack_scale               combine, scale, cast; my share written into the output
                                     tensors of every member of my group
     wait for my kernels, barrier    every rank holds the whole reduced gradient
 
@@ -99,7 +100,8 @@ class ShardedSync:
         self.partials = torch.zeros(self.G, max(n, 1), dtype=tdt, device=grads[0].device)
         self.partial_rows = kt.kt_ptrs(list(self.partials))
         self.main = torch.cuda.Stream()
-        self.side = torch.cuda.Stream()
+        self.side = torch.cuda.Stream()                   # copies down
+        self.up = torch.cuda.Stream()                     # copies up
 
         # 3. host memory that all processes share: a barrier block, then the G partials end to
         #    end, in a file of the node's shared-memory file system that every rank maps and
@@ -142,8 +144,8 @@ class ShardedSync:
         rank has finished reading this rank's `grads`."""
         kt.kt_shard_step(self.ctx, self._host_address, self.partial_rows if self.G > 1 else None, self.host_rows,
                          self.out_ptrs, len(self.members), self.out_dtype, scale=scale,
-                         per_bucket=self.buckets != [-1], main_stream=self.main, side_stream=self.side,
-                         timeout_ms=self.wait_ms)
+                         per_bucket=self.buckets != [-1], main_stream=self.main, down_stream=self.side,
+                         up_stream=self.up, timeout_ms=self.wait_ms)
 
     def set_shares(self, shares: Sequence[int]) -> None:
         """New batch shares (every rank calls this with the same list, between steps): the weights
@@ -156,11 +158,10 @@ class ShardedSync:
         if getattr(self, "_bcast_flat", None) is None:
             n = max(self.plan.transport_numel, 1)
             self._bcast_flat = torch.empty(n, dtype=self.grads[0].dtype, device=self.grads[0].device)
-            self._bcast_stream = torch.cuda.Stream()
         flat = self._bcast_flat.data_ptr()
         host = self._host_address + self._header if self.G > 1 else 0
         kt.kt_shard_bcast(self.ctx, root, self._host_address, flat, host, flat, self.buckets != [-1], self.main,
-                          self.side, self._bcast_stream, timeout_ms=self.wait_ms)
+                          self.side, self.up, timeout_ms=self.wait_ms)
 
     def close(self, meet: bool = True) -> None:
         """Unmaps everything.  meet=False skips the barrier in the shared block: for ranks that
