@@ -75,3 +75,24 @@ def test_three_thousand_small_tensors(kt, oracle):
     all_routes(kt, oracle, wl)
     plan = kt.kt_plan_buckets(wl.numel, wl.bucket_cap_bytes)
     assert plan.n_buckets > 10
+
+
+def test_maximum_ranks_and_groups_with_one_context_per_rank(kt, oracle):
+    """The same limits with every rank a context of its own (one rank per device, emulated in
+    one process): 64 ranks in 16 groups of uneven sizes, shares that leave members of the big
+    groups with an empty range on the short tensors; then one group of 64 (the one-pass route
+    split 64 ways)."""
+    import test_gpu_sharded as TS
+    rnd = random.Random(640)
+    group_of = [min(15, r // 3) for r in range(64)]            # 15 groups of 3 and one of 19
+    shares = [rnd.randint(1, 300) for _ in range(64)]
+    shapes = [(5,), (40000,), (1,), (2049,), (300000,), (17,)]
+    for dtype, relay in (("f32", True), ("bf16", False)):
+        wl = W.Workload("max_sharded", 72, shapes, dtype, group_of, shares, bucket_cap_bytes=1 << 20)
+        host, dev = H.device_gradients(wl)
+        TS.run_emulated(kt, oracle, wl, host, dev, H.TORCH_DT[dtype], 1.0 / 3.0, True, relay)
+    wl = W.Workload("one_group_of_64", 73, shapes, "f32", [0] * 64, shares)
+    host, dev = H.device_gradients(wl)
+    TS.run_emulated(kt, oracle, wl, host, dev, torch.float32, 1.0, False, False, True)
+    wl = W.Workload("max_sharded_bcast", 74, shapes, "bf16", group_of, shares, bucket_cap_bytes=1 << 20)
+    TS.run_emulated_broadcast(kt, oracle, wl, 63, True)
