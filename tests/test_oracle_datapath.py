@@ -281,6 +281,34 @@ def test_hierarchical_equals_flat_within_tolerance(oracle, dtype):
         assert np.max(np.abs(got_b - F) / np.maximum(np.abs(F), absF * 0.5)) < 1e-2
 
 
+def test_unpack_scale_is_slicing_one_multiply_and_the_library_cast(oracle):
+    """kto_unpack_scale pinned exactly, both output types: out[t][j] must be the fp32 product
+    S[off_t + j] * scale (numpy's float32 multiply, one rounding) and, for bf16 outputs, torch's
+    round-to-nearest-even cast of that product, bit for bit; padding never reaches an output."""
+    rng = np.random.default_rng(12)
+    numel = [1, 7, 4096, 513, 0, 10]
+    plan = oracle.bucket_plan(numel, 3000 * 4)
+    assert plan.n_buckets > 1
+    S = (rng.standard_normal(plan.transport_numel) * 1e-3).astype(np.float32)
+    S[::97] *= np.float32(1e30)                              # large magnitudes: rounding carries into the exponent
+    S[5::101] = np.float32(3e-41)                            # subnormals
+    covered = np.zeros(plan.transport_numel, bool)
+    for t, n in enumerate(numel):
+        covered[plan.tensor_offset[t]:plan.tensor_offset[t] + n] = True
+    S_poisoned = S.copy()
+    S_poisoned[~covered] = np.float32(np.nan)                # whatever sits in the padding
+    for scale in (1.0, 0.5, 1.0 / 3.0, 1.0 / 256.0):
+        for S_in in (S, S_poisoned):
+            out32 = oracle.unpack_scale(S_in, plan, scale, F32)
+            out16 = oracle.unpack_scale(S_in, plan, scale, BF16)
+            for t, n in enumerate(numel):
+                off = int(plan.tensor_offset[t])
+                want32 = S[off:off + n] * np.float32(scale)
+                assert out32[t].tobytes() == want32.tobytes()
+                want16 = torch.from_numpy(want32.copy()).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
+                assert out16[t].tobytes() == want16.tobytes()
+
+
 def test_sum_then_divide_reading_agrees(oracle):
     """Weights a_r = b_r, W_g = 1 and a final scale 1/B (plain sums across the
     hierarchy, one division at the end) give the same mean within tolerance."""
