@@ -281,6 +281,72 @@ def test_hierarchical_equals_flat_within_tolerance(oracle, dtype):
         assert np.max(np.abs(got_b - F) / np.maximum(np.abs(F), absF * 0.5)) < 1e-2
 
 
+def _round_to_f32(x: Fraction) -> np.float32:
+    """Correctly rounded (nearest, ties to even) binary32 value of an exact rational."""
+    if x == 0:
+        return np.float32(0.0)
+    sign, mag = (-1 if x < 0 else 1), abs(x)
+    e = mag.numerator.bit_length() - mag.denominator.bit_length()
+    if Fraction(2) ** e > mag:
+        e -= 1                                               # now 2^e <= mag < 2^(e+1)
+    q = max(e, -126) - 23                                    # weight of the last kept bit (subnormals: fixed)
+    scaled = mag / Fraction(2) ** q
+    n = scaled.numerator // scaled.denominator
+    rest = scaled - n
+    if rest > Fraction(1, 2) or (rest == Fraction(1, 2) and n % 2 == 1):
+        n += 1
+    return np.float32(sign * float(Fraction(n) * Fraction(2) ** q))   # n * 2^q has at most 24 bits: exact in double
+
+
+def test_reduction_chains_are_one_product_then_fused_multiply_adds_exactly(oracle):
+    """The order and the roundings the oracle states -- first term one rounded product, every
+    later term ONE rounding of a*x + acc -- checked element by element against exact rational
+    arithmetic with a correctly rounded conversion written here.  A chain that rounded the
+    product and the sum separately, started from zero, or took the ranks in another order
+    fails this on inputs like these."""
+    rng = np.random.default_rng(23)
+    for d in np.concatenate([rng.standard_normal(500) * 1e-3, rng.standard_normal(200) * 1e-42, [0.0, 1.0, -2.5e38]]):
+        assert _round_to_f32(Fraction(float(d))).tobytes() == np.float32(d).tobytes()      # the helper rounds as numpy does
+    numel = [37, 8]
+    group_of, shares, G = [0, 1, 0, 1, 0], [40, 29, 40, 19, 7], 2
+    K = len(group_of)
+    grads = [[(rng.standard_normal(n) * 1e-3).astype(np.float32) for n in numel] for _ in range(K)]
+    a, Wg, w = oracle.coefficients(group_of, shares, G)
+    plan = oracle.bucket_plan(numel, 25 * MIB)
+    parts = oracle.intra_reduce(grads, plan, F32, group_of, a, G)
+    S = oracle.combine(parts, Wg)
+    flat = oracle.flat_reduce_f32([np.concatenate(g) for g in grads], F32, w)
+    fr = lambda v: Fraction(float(v))
+
+    def chain(weights, values):
+        acc = _round_to_f32(fr(weights[0]) * fr(values[0]))
+        for wt, v in zip(weights[1:], values[1:]):
+            acc = _round_to_f32(fr(wt) * fr(v) + fr(acc))
+        return acc
+
+    separate_roundings_differ = 0
+    for t, n in enumerate(numel):
+        off = int(plan.tensor_offset[t])
+        for j in range(n):
+            want_parts = []
+            for g in range(G):
+                members = [r for r in range(K) if group_of[r] == g]
+                want = chain([a[r] for r in members], [grads[r][t][j] for r in members])
+                assert parts[g][off + j].tobytes() == want.tobytes()
+                want_parts.append(want)
+                two = np.float32(a[members[0]]) * grads[members[0]][t][j]
+                for r in members[1:]:
+                    two = np.float32(np.float32(a[r]) * grads[r][t][j]) + two
+                separate_roundings_differ += two.tobytes() != want.tobytes()
+            assert S[off + j].tobytes() == chain(list(Wg), want_parts).tobytes()
+    pos = 0
+    for t, n in enumerate(numel):
+        for j in range(n):
+            assert flat[pos].tobytes() == chain(list(w), [grads[r][t][j] for r in range(K)]).tobytes()
+            pos += 1
+    assert separate_roundings_differ > 0          # the inputs do tell the two kinds of chain apart
+
+
 def test_unpack_scale_is_slicing_one_multiply_and_the_library_cast(oracle):
     """kto_unpack_scale pinned exactly, both output types: out[t][j] must be the fp32 product
     S[off_t + j] * scale (numpy's float32 multiply, one rounding) and, for bf16 outputs, torch's
