@@ -292,6 +292,53 @@ def test_two_kernel_route_in_place(kt, oracle, name):
     kt.kt_destroy(ctx)
 
 
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_special_values_pass_through_like_in_the_oracle(kt, oracle, dtype):
+    """Infinities, NaNs, subnormals, signed zeros and the largest finite values among the
+    gradients (an overflowed mixed-precision step looks like this): wherever the oracle's result
+    is a NaN the kernels' is one too; everything else -- infinities, subnormal results (nothing
+    is flushed to zero), the sign of a zero -- is bit-equal, on both routes."""
+    wl = W.Workload("special", 11, [(4099,), (64,), (9,)], dtype, [0, 0, 1, 1, 1], [3, 5, 7, 2, 1])
+    rng = np.random.default_rng(41)
+    specials32 = np.array([np.inf, -np.inf, np.nan, 0.0, -0.0, 1e-45, -3e-41, 1.1754942e-38, 3.4028235e38, -3.4028235e38,
+                           1e-30, 65504.0], np.float32)
+    host, dev = [], []
+    for r in range(wl.K):
+        ts = []
+        for t_i, n in enumerate(wl.numel):
+            x = (rng.standard_normal(n) * 1e-3).astype(np.float32)
+            where = rng.random(n) < 0.2
+            x[where] = rng.choice(specials32, size=int(where.sum()))
+            t = torch.from_numpy(x)
+            ts.append(t.to(torch.bfloat16) if dtype == "bf16" else t)
+        host.append([W.as_numpy(t) for t in ts])
+        dev.append([t.cuda() for t in ts])
+    for odt in (torch.float32, torch.bfloat16):
+        out, transport, plan, ctx = H.run_gpu_path(kt, wl, dev, wl.shares, out_dtype=odt, scale=0.5)
+        direct = [[torch.full_like(o, 1.0) for o in out[0]]]
+        kt.kt_sync_direct(ctx, direct, scale=0.5)
+        torch.cuda.synchronize()
+        want, parts, _, _ = H.run_oracle_path(oracle, wl, host, wl.shares, out_dtype=0 if odt == torch.float32 else 1, scale=0.5)
+
+        def same(got, exp, what):
+            g = W.as_numpy(got)
+            gf = g if g.dtype == np.float32 else oracle.bf16_to_f32(g)
+            ef = exp if exp.dtype == np.float32 else oracle.bf16_to_f32(exp)
+            nan = np.isnan(ef)
+            assert np.array_equal(np.isnan(gf), nan), what
+            assert np.array_equal(H.bits(g)[~nan], H.bits(exp)[~nan]), what
+            return int(nan.sum()), int(np.isinf(ef).sum()), int(((ef != 0) & (np.abs(ef) < 1.1754942e-38)).sum())
+
+        seen = np.zeros(3, int)
+        for g in range(wl.G):
+            seen += same(transport[g], parts[g], "partial %d" % g)
+        for t in range(wl.T):
+            same(out[0][t], want[t], "out[%d]" % t)
+            same(direct[0][t], want[t], "one-pass out[%d]" % t)
+        assert seen[0] > 0 and seen[1] > 0 and (seen[2] > 0 or dtype == "bf16")      # the cases did occur
+        kt.kt_destroy(ctx)
+
+
 def test_sum_then_divide_coefficients(kt, oracle):
     """Plain sums across the hierarchy with one final division (weights a_r = b_r, W_g = 1,
     scale 1/B) through kt_set_coefficients; oracle fed the same coefficients."""
