@@ -215,6 +215,47 @@ def test_sweep_large_points_sampled_windows(kt, oracle, K, dtype, nbytes):
     check_sampled_windows(kt, oracle, K, nbytes, dtype)
 
 
+def test_a_tensor_of_more_than_two_to_the_31_elements(kt, oracle):
+    """One tensor per rank with 2^31 + 2^20 + 40 elements (8.6 GB of fp32 per rank, two ranks, two
+    groups): element offsets no longer fit 32 bits; the windows checked include the last 2^20
+    elements and one that straddles element 2^31."""
+    n = (1 << 31) + (1 << 20) + 40
+    wl = W.sweep_point(2, n * 4, "f32")
+    assert wl.N == n
+    dev = [[W.rank_gradients(wl, r, "cuda")] for r in range(wl.K)]
+    ctx = kt.kt_groups_init(wl.group_of, wl.shares, wl.G)
+    kt.kt_bucket_pack(ctx, dev, wl.bucket_cap_bytes)
+    plan = kt.kt_plan_query(ctx)
+    tn = plan.transport_numel
+    assert tn == -(-n // 64) * 64
+    transport = [torch.full((tn,), float("nan"), device="cuda") for _ in range(wl.G)]
+    out = [[torch.full((n,), float("nan"), device="cuda")]]
+    kt.kt_hier_reduce(ctx, kt.KT_INTRA, transport)
+    kt.kt_unpack_scale(ctx, transport, out)
+    torch.cuda.synchronize()
+    win = 1 << 20
+    for s in (0, (1 << 31) - win // 2, n - win, (1 << 30) + 12344):
+        hx = [[W.as_numpy(dev[r][0][s:s + win])] for r in range(wl.K)]
+        o_out, o_parts, _, _ = oracle.sync_step(hx, [win], F32, wl.group_of, wl.shares, wl.G, 1 << 62)
+        for g in range(wl.G):
+            H.assert_bit_equal(transport[g][s:s + win], o_parts[g], "window %d transport[%d]" % (s, g))
+        H.assert_bit_equal(out[0][0][s:s + win], o_out[0], "window %d out" % s)
+    assert not bool(torch.isnan(out[0][0]).any())
+    assert bool((transport[0][n:] == 0).all()) and bool((transport[1][n:] == 0).all())      # the padding behind the tail
+    # the one-pass route into the same output
+    out[0][0].fill_(float("nan"))
+    kt.kt_sync_direct(ctx, out)
+    torch.cuda.synchronize()
+    s = n - win
+    hx = [[W.as_numpy(dev[r][0][s:s + win])] for r in range(wl.K)]
+    o_out, _, _, _ = oracle.sync_step(hx, [win], F32, wl.group_of, wl.shares, wl.G, 1 << 62)
+    H.assert_bit_equal(out[0][0][s:s + win], o_out[0], "one-pass, last window")
+    assert not bool(torch.isnan(out[0][0]).any())
+    kt.kt_destroy(ctx)
+    del dev, transport, out
+    torch.cuda.empty_cache()
+
+
 # ------------------------------------------------------------------ variants and edge cases
 def test_misaligned_sources_take_the_element_path(kt, oracle):
     for wl in (W.tiny(), W.sweep_point(4, 1 << 20, "bf16"), W.sweep_point(2, 1 << 20, "f32")):
