@@ -10,8 +10,8 @@ import sys
 
 _PKG = os.path.dirname(os.path.abspath(__file__))
 _ROOT = os.path.dirname(_PKG)
-SOURCES = [os.path.join(_PKG, "csrc", "kaitian.cu")]
-DEPENDS = [os.path.join(_PKG, "csrc", "kt_kernels.cuh")]
+SOURCES = [os.path.join(_PKG, "csrc", "kaitian.cu"), os.path.join(_PKG, "csrc", "kt_host.cu")]
+DEPENDS = [os.path.join(_PKG, "csrc", "kt_kernels.cuh"), os.path.join(_PKG, "csrc", "kt_internal.h")]
 HEADERS = [os.path.join(_ROOT, "include", "kaitian.h")]
 LIB = os.path.join(_PKG, "libkaitian_b200.so")
 
