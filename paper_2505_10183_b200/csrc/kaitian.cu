@@ -1,7 +1,9 @@
-// kaitian.cu -- host side of the C ABI for KAITIAN's hierarchical, load-weighted gradient
-// synchronisation (paper Sections III-A and III-C): scheduler, weights, bucket plan, device
-// tables, launches, pinned-host staging.  The kernels are in kt_kernels.cuh; the contract of
-// every entry point is in include/kaitian.h.
+// kaitian.cu -- the device side of the C ABI for KAITIAN's hierarchical, load-weighted gradient
+// synchronisation (paper Sections III-A and III-C): contexts and weights, device tables,
+// launches, pinned-host staging, the broadcast, recorded steps, memory shared between processes,
+// the entry point that allocates nothing.  The kernels are in kt_kernels.cuh, the entry points
+// that are pure host arithmetic (scheduler, plan, share ranges, host barrier ...) in kt_host.cu;
+// the contract of every entry point is in include/kaitian.h.
 //
 // Data layout in device memory
 //   gradients   K*T caller-owned tensors (fp32 or bf16), read in place through a pointer
