@@ -32,8 +32,10 @@
  *    call made by the calling thread.
  *  - Kernel launches and copies are asynchronous with respect to the given stream.
  *    kt_scores, kt_schedule, kt_route, kt_adapt_*, kt_sampler_steps, kt_plan_buckets,
- *    kt_set_shares, kt_set_coefficients and kt_plan_query are pure host functions; the first
- *    six need no CUDA device at all.
+ *    kt_shard_ranges, kt_work_unit, kt_host_barrier, kt_set_shares, kt_set_coefficients,
+ *    kt_plan_query and kt_shard_query are pure host functions; those before kt_set_shares
+ *    need no CUDA device at all.  kt_shard_step and kt_shard_bcast block the calling thread
+ *    until every rank has finished.
  *  - A context is bound to the CUDA device that was current in kt_groups_init.  Calls on it
  *    make that device current for their own duration and leave the calling thread's current
  *    device as they found it.
