@@ -725,7 +725,7 @@ def run_ours(args) -> dict:
 # dram__bytes_read.sum + dram__bytes_write.sum per launch of the fused reduce on each named
 # workload, from ncu captures of the kernel as committed (not measured in this run: a run under
 # a profiler reports no times).  A workload without a capture reports null.
-TRAFFIC_K1 = {"resnet18": 217007104, "mobilenet_v2": 120187136, "resnet50": 559726592}
+TRAFFIC_K1 = {"resnet18": 216022272, "mobilenet_v2": 120217856, "resnet50": 560153856}
 TRAFFIC_SOURCE = ("ncu --set full captures of the fused reduce as committed, first launch: profiles/k1_k2_resnet18.md, "
                   "profiles/k1_k2_mobilenet_v2_resnet50.md (read + write bytes; below the algorithmic bytes because part "
                   "of the output is still dirty in the 126 MB L2 when a 27-92 us kernel ends)")
