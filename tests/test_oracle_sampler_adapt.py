@@ -147,6 +147,27 @@ def test_adapt_hysteresis_keeps_shares_under_noise_and_follows_a_real_slowdown(o
     assert ad.shares[0] < 79 / 1.5
 
 
+def test_adapt_hysteresis_threshold_worked_by_hand(oracle):
+    """Two ranks at 50 / 50 of 100 samples, every observation adopted into the average at once
+    (alpha = 1, period = 1).  Per-sample times 1 and 1.5 (in 1/64 s): the step now takes
+    max(50, 75) = 75; the schedule of those times is 60 / 40 and predicts max(60, 60) = 60, that is
+    0.8 of 75.  New shares are taken only if they predict less than (1 - hysteresis) of the
+    present step: at 0.25 they are not, at 0.15 they are.  With times 1 and 3 the candidate 75 / 25
+    predicts 75 of 150, exactly one half: a hysteresis of one half keeps the old shares (the
+    comparison is strict), a quarter lets them go."""
+    def after_one(x, h):
+        ad = oracle.Adapter([50, 50], 100, 1.0, 1, h)
+        changed = ad.observe([50 * 1.0 / 64.0, 50 * x / 64.0])
+        return bool(changed), ad.shares.tolist()
+    assert after_one(1.5, 0.25) == (False, [50, 50])
+    assert after_one(1.5, 0.15) == (True, [60, 40])
+    assert after_one(1.5, 0.0) == (True, [60, 40])
+    assert after_one(3.0, 0.5) == (False, [50, 50])
+    assert after_one(3.0, 0.25) == (True, [75, 25])
+    # equal speeds: the candidate is the present split, nothing to adopt whatever the threshold
+    assert after_one(1.0, 0.0) == (False, [50, 50])
+
+
 def test_adapt_rejects_bad_input(oracle):
     for alpha, period, h in ((0.0, 1, 0.0), (1.5, 1, 0.0), (0.5, 0, 0.0), (0.5, 1, 1.0), (0.5, 1, -0.1)):
         with pytest.raises(oracle.OracleError):
