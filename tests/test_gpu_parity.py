@@ -159,6 +159,19 @@ def test_mobilenet_v2_ragged(kt, oracle):
     check_tolerance(oracle, wl, host, out, shares)
 
 
+@pytest.mark.parametrize("name", ["tiny", "resnet18", "mobilenet_v2", "resnet50"])
+def test_named_workloads_with_unequal_shares_inside_groups(kt, oracle, name):
+    """The named configurations put equally fast devices in a group: in-group weights of 1/2
+    and 1/4, with which every product of the reduce is exact and a fused multiply-add cannot
+    differ from a multiply and an add.  The same tensor lists with shares that differ inside
+    every group make each term of each chain round."""
+    wl = W.by_name(name)
+    wl.shares = {4: [83, 75, 45, 53], 8: [37, 41, 43, 47, 23, 31, 17, 17]}[wl.K]
+    host, out, shares = compare_all(kt, oracle, wl)
+    assert shares == wl.shares
+    check_tolerance(oracle, wl, host, out, shares)
+
+
 @pytest.mark.parametrize("K", [2, 4, 8, 16])
 @pytest.mark.parametrize("dtype", ["f32", "bf16"])
 @pytest.mark.parametrize("nbytes", [4 << 10, 64 << 10, 1 << 20, 16 << 20])

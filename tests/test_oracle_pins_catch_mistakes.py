@@ -18,6 +18,8 @@ from concurrent.futures import ThreadPoolExecutor
 
 import pytest
 
+from _planted import write_oracle_copy
+
 ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 PIN_FILES = ["test_oracle_schedule.py", "test_oracle_sampler_adapt.py", "test_oracle_sharding.py",
              "test_oracle_datapath.py"]
@@ -171,29 +173,12 @@ def make_tree(tmp, name, old, new, occurrence):
     """A miniature of the repository in `tmp`: the pin tests and their fixtures, the package (by
     link: the pin tests take the workloads' shapes from it), and the oracle with one mistake."""
     os.makedirs(os.path.join(tmp, "tests"))
-    os.makedirs(os.path.join(tmp, "oracle"))
     for f in PIN_FILES + ["conftest.py"]:
         shutil.copy(os.path.join(ROOT, "tests", f), os.path.join(tmp, "tests", f))
     shutil.copytree(os.path.join(ROOT, "tests", "golden"), os.path.join(tmp, "tests", "golden"))
     os.symlink(os.path.join(ROOT, "paper_2505_10183_b200"), os.path.join(tmp, "paper_2505_10183_b200"))
     os.symlink(os.path.join(ROOT, "include"), os.path.join(tmp, "include"))
-    for f in ("__init__.py", "kt_oracle.py"):
-        shutil.copy(os.path.join(ROOT, "oracle", f), os.path.join(tmp, "oracle", f))
-    # the text is looked for in the C source first, then in the Python side (the whole-path drivers)
-    for target in ("kt_oracle.c", "kt_oracle.py"):
-        src = open(os.path.join(ROOT, "oracle", target)).read()
-        if old in src:
-            break
-    at = -1
-    for _ in range((occurrence or 0) + 1):
-        at = src.find(old, at + 1)
-        assert at >= 0, "mistake %r: the text to change is not in the oracle's source (any more)" % name
-    if occurrence is None:
-        assert src.find(old, at + 1) < 0, "mistake %r: the text to change is not unique" % name
-    if target != "kt_oracle.c":
-        shutil.copy(os.path.join(ROOT, "oracle", "kt_oracle.c"), os.path.join(tmp, "oracle", "kt_oracle.c"))
-    with open(os.path.join(tmp, "oracle", target), "w") as f:
-        f.write(src[:at] + new + src[at + len(old):])
+    write_oracle_copy(os.path.join(tmp, "oracle"), name, old, new, occurrence)
 
 
 def run_pins(tmp, pin_file):
