@@ -375,8 +375,10 @@ int kt_stage_to_host(kt_ctx *ctx, int dir, int bucket, float *const *transport,
  * down / up is what kt_stage_wait(KT_D2H / KT_H2D, bucket) waits for.
  * send, host_pinned, recv: host arrays of G pointers (device fp32, pinned host, device fp32),
  * same element offsets in all three.  chunk_bytes >= 256; the two copy streams must differ.
- * With bucket == -1, if the G buffers of each list lie back to back in memory (rows of one
- * allocation of G * transport_numel elements), a chunk of all groups moves in one copy.
+ * With bucket == -1, if the G buffers of each list are rows of one allocation of
+ * G * transport_numel elements (back to back in memory, and the driver confirms that each
+ * list's range is a single allocation: buffers that merely happen to be neighbours do not
+ * count), a chunk of all groups moves in one copy.
  * Errors: KT_ERR_STATE, KT_ERR_SHAPE, KT_ERR_INVALID, KT_ERR_CUDA. */
 int kt_relay_through_host(kt_ctx *ctx, int bucket, float *const *send, float *const *host_pinned,
                           float *const *recv, int64_t chunk_bytes, void *main_stream,

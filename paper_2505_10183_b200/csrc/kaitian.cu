@@ -21,6 +21,7 @@
 
 #include "../../include/kaitian.h"
 
+#include <cuda.h>            // types and enumerators only: driver entry points are asked of the runtime
 #include <cuda_runtime.h>
 
 #include "kt_kernels.cuh"
@@ -473,6 +474,31 @@ std::vector<int64_t> cut_chunks(int64_t n, int64_t chunk) {
     return sizes;
 }
 
+// Whether [p, p + bytes) lies inside ONE allocation (device memory, or host memory page-locked by
+// one call).  Two allocations can be neighbours in the address space, yet a single copy must
+// not run across the seam: the runtime rejects it.  Asked of the driver (start and size of the
+// allocation that holds p); "no" whenever the driver cannot say.
+bool one_allocation(const void *p, size_t bytes) {
+    typedef CUresult (*attr_fn)(void *, CUpointer_attribute, CUdeviceptr);
+    static const attr_fn query = [] {
+        void *fn = nullptr;
+        cudaDriverEntryPointQueryResult found;
+        if (cudaGetDriverEntryPoint("cuPointerGetAttribute", &fn, cudaEnableDefault, &found) != cudaSuccess ||
+            found != cudaDriverEntryPointSuccess) {
+            cudaGetLastError();
+            fn = nullptr;
+        }
+        return reinterpret_cast<attr_fn>(fn);
+    }();
+    if (!query) return false;
+    const CUdeviceptr at = static_cast<CUdeviceptr>(reinterpret_cast<uintptr_t>(p));
+    CUdeviceptr start = 0;
+    size_t size = 0;
+    if (query(&start, CU_POINTER_ATTRIBUTE_RANGE_START_ADDR, at) != CUDA_SUCCESS) return false;
+    if (query(&size, CU_POINTER_ATTRIBUTE_RANGE_SIZE, at) != CUDA_SUCCESS) return false;
+    return at >= start && bytes <= size && at - start <= size - bytes;
+}
+
 // One event per chunk of a relay ("chunk k went down: its way up may start"), created on demand.
 int ensure_chunk_events(kt_ctx *c, size_t n_chunks) {
     while (c->chunk_events.size() < n_chunks) {
@@ -856,6 +882,11 @@ int kt_relay_through_host(kt_ctx *c, int bucket, float *const *send, float *cons
             rows = rows && at_elem(send[g], n) == at_elem(send[g + 1], 0) &&
                    at_elem(host_pinned[g], n) == at_elem(host_pinned[g + 1], 0) &&
                    at_elem(recv[g], n) == at_elem(recv[g + 1], 0);
+        // neighbours by address are not enough: each set must be one allocation, or a copy that
+        // runs across the seam between two of them is refused
+        const size_t all = static_cast<size_t>(n) * es * c->G;
+        rows = rows && c->G > 1 && one_allocation(send[0], all) && one_allocation(host_pinned[0], all) &&
+               one_allocation(recv[0], all);
         if (rows) {
             n *= c->G;
             groups = 1;

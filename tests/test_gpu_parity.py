@@ -498,6 +498,51 @@ def test_staging_bytes_and_ordering(kt, oracle):
     kt.kt_destroy(ctx)
 
 
+def test_relay_of_host_buffers_that_are_neighbours_but_separate_allocations(kt, oracle):
+    """The relay moves a chunk of all groups in one copy when the G buffers of each set are rows
+    of one allocation.  Lying back to back is not enough for that: here the device buffers are
+    rows of one allocation, but the host buffers are two halves of one mapping that were
+    page-locked by two separate calls -- neighbours in the address space, two allocations to the
+    driver, which refuses a copy that runs across the seam.  The relay has to notice and copy
+    group by group."""
+    import ctypes
+    import mmap
+    wl = W.sweep_point(4, 4096 * 4, "f32")
+    host, dev = H.device_gradients(wl)
+    ctx = kt.kt_groups_init(wl.group_of, wl.shares, wl.G)
+    kt.kt_bucket_pack(ctx, dev, wl.bucket_cap_bytes)
+    n = kt.kt_plan_query(ctx).transport_numel
+    nbytes = n * 4
+    assert nbytes % mmap.PAGESIZE == 0
+    block = mmap.mmap(-1, wl.G * nbytes)
+    view = (ctypes.c_char * (wl.G * nbytes)).from_buffer(block)
+    base = ctypes.addressof(view)
+    for g in range(wl.G):
+        kt.kt_host_register(base + g * nbytes, nbytes)
+    crossed = None
+    try:
+        send = torch.full((wl.G, n), float("nan"), device="cuda")
+        recv = torch.full((wl.G, n), float("nan"), device="cuda")
+        pinned = kt.PtrArray.from_addresses([base + g * nbytes for g in range(wl.G)], keep=block)
+        down, up = torch.cuda.Stream(), torch.cuda.Stream()
+        kt.kt_hier_reduce(ctx, kt.KT_INTRA, list(send))
+        kt.kt_relay_through_host(ctx, list(send), pinned, list(recv), down, up, bucket=-1, chunk_bytes=4096)
+        kt.kt_stage_wait(ctx, kt.KT_H2D, bucket=-1)
+        torch.cuda.synchronize()
+        _, o_parts, _, _ = H.run_oracle_path(oracle, wl, host, wl.shares)
+        crossed = np.frombuffer(view, dtype=np.float32).reshape(wl.G, n)
+        for g in range(wl.G):
+            H.assert_bit_equal(recv[g], o_parts[g], "received partial %d" % g)
+            assert np.array_equal(H.bits(crossed[g].copy()), H.bits(o_parts[g])), "host copy of partial %d" % g
+    finally:
+        torch.cuda.synchronize()
+        for g in range(wl.G):
+            kt.kt_host_unregister(base + g * nbytes)
+        kt.kt_destroy(ctx)
+        del crossed, view
+        block.close()
+
+
 def test_whole_transport_goes_up_only_after_every_bucket_came_down(kt, oracle):
     """Mixed granularity on different copy streams: the partials go down bucket by bucket on one
     stream, the whole transport comes back up in one call on another.  The way up must wait
