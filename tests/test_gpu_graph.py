@@ -190,3 +190,105 @@ def test_destination_table_uploaded_on_one_stream_is_safe_to_use_on_another(kt, 
         H.assert_bit_equal(out[0][t], want[t], "out[%d] written from stream B" % t)
     torch.cuda.synchronize()
     kt.kt_destroy(ctx)
+
+
+def random_table_traffic(kt, oracle, rnd, bursts):
+    """Random traffic over a context's destination tables: more sets of output tensors than the
+    context keeps tables for, written by the combine+unpack, by the one-pass kernel and by
+    replayed recordings, on three streams, in bursts without any synchronisation inside a burst
+    (so tables are replaced while kernels that read their neighbours are still queued), with new
+    recordings, destroyed recordings and new plans in between.  After every burst each targeted
+    set must hold the oracle's result and every other set must be untouched."""
+    import test_gpu_random as TR
+    wl = TR.random_problem(rnd)
+    host, dev = H.device_gradients(wl, misalign=rnd.choice([0, 0, 1, 3]))
+    ctx = kt.kt_groups_init(wl.group_of, wl.shares, wl.G)
+    kt.kt_bucket_pack(ctx, dev, wl.bucket_cap_bytes)
+    n = kt.kt_plan_query(ctx).transport_numel
+    transport = [torch.full((n,), float("nan"), device="cuda") for _ in range(wl.G)]
+    streams = [torch.cuda.Stream() for _ in range(3)]
+    kt.kt_hier_reduce(ctx, kt.KT_INTRA, transport, stream=streams[0])
+    torch.cuda.synchronize()
+    scales = [1.0, 1.0 / 3.0]
+    want = {}
+    for code, dt in ((0, torch.float32), (1, torch.bfloat16)):
+        for s in scales:
+            want[dt, s] = H.run_oracle_path(oracle, wl, host, wl.shares, out_dtype=code, scale=s)[0]
+    n_sets = 14
+    sets = []
+    for _ in range(n_sets):
+        dt, R = rnd.choice([torch.float32, torch.bfloat16]), rnd.randint(1, min(2, wl.K))
+        sets.append(dict(dtype=dt, tensors=[[torch.full((m,), float("nan"), dtype=dt, device="cuda") for m in wl.numel]
+                                            for _ in range(R)]))
+    graphs = []                                      # (graph, set index, scale)
+    recorded_sets = set()
+
+    def launch(i, scale, stream, one_pass):
+        if one_pass:
+            kt.kt_sync_direct(ctx, sets[i]["tensors"], scale=scale, stream=stream)
+        else:
+            kt.kt_unpack_scale(ctx, transport, sets[i]["tensors"], scale=scale, stream=stream)
+
+    def verify(written):
+        torch.cuda.synchronize()
+        for i, st in enumerate(sets):
+            for copy in st["tensors"]:
+                for t in range(wl.T):
+                    if i in written:
+                        H.assert_bit_equal(copy[t], want[st["dtype"], written[i]][t], "set %d out[%d]" % (i, t))
+                        copy[t].fill_(float("nan"))
+                    else:
+                        assert bool(torch.isnan(copy[t].float()).all()), "set %d was written by a call for another set" % i
+        torch.cuda.synchronize()
+
+    for _ in range(bursts):
+        move = rnd.random()
+        if move < 0.12 and len(recorded_sets) < 6:
+            # a new recording: the set must have been used once, outside a recording
+            i, scale, one_pass, s = rnd.randrange(n_sets), rnd.choice(scales), rnd.random() < 0.5, rnd.choice(streams)
+            launch(i, scale, s, one_pass)
+            verify({i: scale})
+            kt.kt_graph_begin(ctx, s)
+            launch(i, scale, s, one_pass)
+            graphs.append((kt.kt_graph_end(ctx, s), i, scale))
+            recorded_sets.add(i)
+            verify({})                               # recording runs nothing
+        elif move < 0.16 and graphs:
+            g, _, _ = graphs.pop(rnd.randrange(len(graphs)))
+            torch.cuda.synchronize()
+            kt.kt_graph_destroy(g)
+        elif move < 0.19:
+            # a new plan: recordings are void (destroyed first), every table is free again
+            torch.cuda.synchronize()
+            for g, _, _ in graphs:
+                kt.kt_graph_destroy(g)
+            graphs, recorded_sets = [], set()
+            kt.kt_bucket_pack(ctx, dev, wl.bucket_cap_bytes)
+        else:
+            written = {}
+            for _ in range(rnd.randint(1, 7)):
+                s = rnd.choice(streams)
+                if graphs and rnd.random() < 0.3:
+                    g, i, scale = rnd.choice(graphs)
+                    if i in written:
+                        continue
+                    kt.kt_graph_launch(g, s)
+                else:
+                    i, scale = rnd.randrange(n_sets), rnd.choice(scales)
+                    if i in written:
+                        continue
+                    launch(i, scale, s, rnd.random() < 0.5)
+                written[i] = scale
+            verify(written)
+    torch.cuda.synchronize()
+    for g, _, _ in graphs:
+        kt.kt_graph_destroy(g)
+    kt.kt_destroy(ctx)
+
+
+@pytest.mark.parametrize("seed", range(4))
+def test_random_traffic_over_the_destination_tables(kt, oracle, seed):
+    import random
+    rnd = random.Random(4100 + seed)
+    for _ in range(3):
+        random_table_traffic(kt, oracle, rnd, bursts=40)
