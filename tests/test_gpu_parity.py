@@ -3,6 +3,8 @@ same seeded inputs.  Bars: bit-exact for pack / unpack / casts / shares / plan; 
 reductions the kernels follow the oracle's operation order, so results are compared bit
 for bit as well, and the stated tolerances (1e-6 relative for fp32 sources, 1e-2 for
 bf16-sourced gradients) are checked against an fp64 weighted mean on top."""
+import random
+
 import numpy as np
 import pytest
 import torch
@@ -577,6 +579,87 @@ def test_whole_transport_goes_up_only_after_every_bucket_came_down(kt, oracle):
     for g in range(wl.G):
         H.assert_bit_equal(recv[g], o_parts[g], "receive buffer %d" % g)
     kt.kt_destroy(ctx)
+
+
+def random_staging_traffic(kt, oracle, rnd, rounds):
+    """Steps queued back to back without any synchronisation, each choosing its own granularity
+    for every phase (whole transport or bucket by bucket, for the reduce, the way down, the way
+    up -- as two calls or as the chunked relay -- and the combine+unpack) and its own copy
+    streams out of a pool of three.  From step to step the gradients are scaled by another power of two
+    (exact), so a phase that ran ahead of the data it depends on, or picked up the data of the
+    step before, shows in the result."""
+    import test_gpu_random as TR
+    wl = TR.random_problem(rnd)
+    if rnd.random() < 0.5:        # more and larger buckets
+        wl = W.Workload("random_long", wl.config_id, [(rnd.choice([5000, 20000, 70001, 300000]),) for _ in range(rnd.randint(2, 5))],
+                        wl.dtype, wl.group_of, wl.shares, bucket_cap_bytes=rnd.choice([40000, 400000, 1 << 40]))
+    host, dev = H.device_gradients(wl)
+    base = [[t.clone() for t in row] for row in dev]
+    ctx = kt.kt_groups_init(wl.group_of, wl.shares, wl.G)
+    kt.kt_bucket_pack(ctx, dev, wl.bucket_cap_bytes)
+    plan = kt.kt_plan_query(ctx)
+    n, nb = plan.transport_numel, plan.n_buckets
+    rows = rnd.random() < 0.5
+    def buffers(pinned=False):
+        if rows:
+            whole = torch.zeros(wl.G, n)
+            return list(whole.pin_memory() if pinned else whole.cuda())
+        return [torch.zeros(n).pin_memory() if pinned else torch.zeros(n, device="cuda") for _ in range(wl.G)]
+    tr, pinned, recv = buffers(), buffers(True), buffers()
+    out_dtype = rnd.choice([torch.float32, torch.bfloat16])
+    out = [[torch.zeros(m, dtype=out_dtype, device="cuda") for m in wl.numel]]
+    want, _, _, _ = H.run_oracle_path(oracle, wl, host, wl.shares, out_dtype={torch.float32: F32, torch.bfloat16: BF16}[out_dtype])
+    main = torch.cuda.Stream()
+    pool = [torch.cuda.Stream() for _ in range(3)]
+    every, whole = list(range(nb)), [-1]
+    snapshots = []
+    torch.cuda.synchronize()
+    for r in range(rounds):
+        factor = float(2 ** rnd.randint(-4, 4))
+        with torch.cuda.stream(main):
+            for row, brow in zip(dev, base):           # this step's gradients: the seeded ones times a power of two
+                for t, b in zip(row, brow):
+                    torch.mul(b, factor, out=t)
+        reduce_by, down_by, up_by, unpack_by = (rnd.choice([every, whole]) for _ in range(4))
+        relay = rnd.random() < 0.4
+        for b in reduce_by:
+            kt.kt_hier_reduce(ctx, kt.KT_INTRA, tr, bucket=b, stream=main)
+        if relay:
+            a, c = rnd.sample(pool, 2)
+            for b in down_by:
+                kt.kt_relay_through_host(ctx, tr, pinned, recv, a, c, bucket=b, chunk_bytes=rnd.choice([256, 4096, 65536, 1 << 20]),
+                                         main_stream=main)
+            up_by = down_by
+        else:
+            for b in down_by:
+                kt.kt_stage_to_host(ctx, kt.KT_D2H, tr, pinned, bucket=b, main_stream=main, side_stream=rnd.choice(pool))
+            for b in up_by:
+                kt.kt_stage_to_host(ctx, kt.KT_H2D, recv, pinned, bucket=b, main_stream=main, side_stream=rnd.choice(pool))
+        for b in up_by:
+            kt.kt_stage_wait(ctx, kt.KT_H2D, bucket=b, main_stream=main)
+        for b in unpack_by:
+            kt.kt_unpack_scale(ctx, recv, out, bucket=b, stream=main)
+        with torch.cuda.stream(main):
+            snapshots.append((factor, [t.clone() for t in out[0]]))
+        if len(snapshots) >= 6 or r == rounds - 1:
+            torch.cuda.synchronize()
+            for factor, got in snapshots:
+                for t in range(wl.T):
+                    w = want[t]
+                    if w.dtype == np.uint16:
+                        w = oracle.f32_to_bf16(oracle.bf16_to_f32(w) * np.float32(factor))
+                    else:
+                        w = w * np.float32(factor)
+                    H.assert_bit_equal(got[t], w, "step with factor %g, out[%d]" % (factor, t))
+            snapshots = []
+    kt.kt_destroy(ctx)
+
+
+@pytest.mark.parametrize("seed", range(4))
+def test_random_staging_granularities_and_streams(kt, oracle, seed):
+    rnd = random.Random(8800 + seed)
+    for _ in range(5):
+        random_staging_traffic(kt, oracle, rnd, rounds=14)
 
 
 # ------------------------------------------------------------------ error paths
