@@ -116,3 +116,35 @@ def test_output_guard_bytes_untouched(kt, oracle):
         for b, m in zip(obuf, wl.numel):
             assert bool((b[:guard] == -777.0).all()) and bool((b[guard + m:] == -777.0).all())
         kt.kt_destroy(ctx)
+
+
+def test_contexts_on_different_host_threads(kt, oracle):
+    """Different contexts may be used from different host threads at the same time (the
+    header's promise): four threads, each with contexts, streams and buffers of its own, run
+    random problems side by side; every result equals the oracle's, and a failing call on one
+    thread leaves its message on that thread only."""
+    import threading
+    failures = []
+
+    def worker(i):
+        try:
+            torch.cuda.set_device(0)
+            rnd = random.Random(31000 + i)
+            with torch.cuda.stream(torch.cuda.Stream()):
+                for _ in range(12):
+                    run_case(kt, oracle, rnd)
+                    if i == 0:                          # one thread keeps failing calls going
+                        with pytest.raises(kt.KtError):
+                            kt.kt_groups_init([0, 2], [1, 1], 3)
+                        assert "outside" in kt.kt_last_error()
+                    else:
+                        assert kt.kt_last_error() == ""
+        except BaseException as e:                      # reported by the main thread
+            failures.append((i, repr(e)))
+
+    threads = [threading.Thread(target=worker, args=(i,)) for i in range(4)]
+    for t in threads:
+        t.start()
+    for t in threads:
+        t.join()
+    assert not failures, failures
