@@ -295,7 +295,8 @@ int kt_host_barrier(void *shared, int n_ranks, int timeout_ms);
  * the same element range of the other groups' partials up (up_stream, while later ranges are
  * still going down), combine + scale + cast + unpack of the share into the R = M output sets
  * (this rank's and, peer-mapped, its group mates') -> wait for the own stream, barrier.  With
- * one group the middle is kt_sync_direct.
+ * one group the middle is kt_sync_direct: nothing is stored in a transport, so the transport's
+ * element type (kt_set_transport_dtype) has no effect on the result.
  *   barrier_block (host): the kt_host_barrier block shared by all K ranks of kt_groups_init.
  *   partials: host array of G device pointers, this rank's rows of transport_numel elements
  *        (row of its own group: the share it reduces; other rows: what it receives).

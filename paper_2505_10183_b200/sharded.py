@@ -44,7 +44,8 @@ class ShardedSync:
         rank wants the reduced gradients (None: in place, over `grads`); host_group: a
         torch.distributed group whose collectives run on the host (gloo) and whose ranks are
         numbered like `group_of`; narrow_transport: the library's bf16 transport (an extension:
-        half the bytes through host memory, one extra rounding of every group partial)."""
+        half the bytes through host memory, one extra rounding of every group partial; without
+        effect when all ranks are one group, where no partial is stored)."""
         self.rank, self.group_of, self.K = rank, list(group_of), len(group_of)
         self.G = max(group_of) + 1
         self.g = group_of[rank]

@@ -286,6 +286,10 @@ CASES = [
 
 
 def case_workload(case, world):
+    if "numel" in case:          # a drawn problem: flat tensors of the listed sizes
+        wl = W.Workload(case["name"], case["config_id"], [(m,) for m in case["numel"]], case["dtype"],
+                        list(case["group_of"]), list(case["shares"]), bucket_cap_bytes=case["cap"])
+        return wl if wl.K == world else None
     wl = W.by_name(case["wl"])
     if "dtype" in case:
         wl.dtype = case["dtype"]
@@ -328,8 +332,9 @@ def rank_main(rank, world, port, cases):
         shares = list(wl.shares)
         for scale in scales:
             job.step(scale=scale)
+            # with one group no partial is ever stored: the narrow transport has nothing to round
             want, _, _, _ = oracle.sync_step(host, wl.numel, dt, wl.group_of, shares, wl.G, wl.bucket_cap_bytes,
-                                             scale, H.ORACLE_DT[odt_name], 1 if narrow else 0)
+                                             scale, H.ORACLE_DT[odt_name], 1 if narrow and wl.G > 1 else 0)
             # the scheduler moves samples from the first rank to the last between steps: new weights
             shares = [shares[0] - 1] + shares[1:-1] + [shares[-1] + 1] if shares[0] > 1 and wl.K > 1 else shares
             job.set_shares(shares)
@@ -339,6 +344,38 @@ def rank_main(rank, world, port, cases):
         job.close()
     dist.barrier()
     dist.destroy_process_group()
+
+
+def random_cases(rnd, world, count):
+    """Drawn problems for `world` ranks: ragged tensor lists, group layouts, shares, dtypes,
+    bucket caps, output dtypes, in place or not, bucket by bucket or not, either transport."""
+    cases = []
+    while len(cases) < count:
+        wl = TR.random_problem(rnd)
+        if wl.K != world:
+            continue
+        numel = list(wl.numel)
+        if rnd.random() < 0.3:
+            numel = [rnd.choice([5000, 20000, 70001]) for _ in range(rnd.randint(1, 3))]
+        in_place = rnd.random() < 0.4
+        case = dict(name="drawn_%d" % len(cases), numel=numel, config_id=wl.config_id, dtype=wl.dtype, group_of=wl.group_of,
+                    shares=wl.shares, cap=wl.bucket_cap_bytes, per_bucket=rnd.random() < 0.5, in_place=in_place,
+                    narrow=rnd.random() < 0.25)
+        if not in_place:
+            case["out_dtype"] = rnd.choice(["f32", "bf16"])
+        cases.append(case)
+    return cases
+
+
+@pytest.mark.parametrize("world", [3])
+def test_ranks_as_processes_on_drawn_problems(world):
+    import random
+    import torch.multiprocessing as mp
+    if not torch.cuda.is_available():
+        pytest.fail("this test needs a CUDA device")
+    cases = random_cases(random.Random(5150), world, 14)
+    port = 29600 + (os.getpid() * 13 + world) % 2000
+    mp.spawn(rank_main, args=(world, port, cases), nprocs=world, join=True)
 
 
 @pytest.mark.parametrize("world", [4, 5])
