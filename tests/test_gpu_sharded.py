@@ -460,12 +460,18 @@ def bcast_rank_main(rank, world, port, cases):
     torch.cuda.set_device(0)
     dist.init_process_group("gloo", rank=rank, world_size=world)
     for case in cases:
-        wl = W.by_name(case["wl"])
-        wl.dtype = case.get("dtype", wl.dtype)
-        if "group_of" in case:
-            wl.group_of = list(case["group_of"])
-        if wl.K != world:
-            continue
+        if "numel" in case:
+            wl = case_workload(case, world)
+            if wl is None:
+                continue
+            case = dict(case, wl=case["name"])
+        else:
+            wl = W.by_name(case["wl"])
+            wl.dtype = case.get("dtype", wl.dtype)
+            if "group_of" in case:
+                wl.group_of = list(case["group_of"])
+            if wl.K != world:
+                continue
         dt = H.ORACLE_DT[wl.dtype]
         host = [[W.as_numpy(t) for t in W.split_tensors(W.rank_gradients(wl, r, "cpu"), wl.numel)] for r in range(wl.K)]
         params = [t.cuda() for t in W.split_tensors(W.rank_gradients(wl, rank, "cpu"), wl.numel)]     # every rank starts with its own values
@@ -480,6 +486,15 @@ def bcast_rank_main(rank, world, port, cases):
         job.close()
     dist.barrier()
     dist.destroy_process_group()
+
+
+def test_broadcast_with_ranks_as_processes_on_drawn_problems():
+    import torch.multiprocessing as mp
+    if not torch.cuda.is_available():
+        pytest.fail("this test needs a CUDA device")
+    rnd = random.Random(6160)
+    cases = [dict(c, root=rnd.randrange(3)) for c in random_cases(rnd, 3, 14)]
+    mp.spawn(bcast_rank_main, args=(3, 29600 + (os.getpid() * 17 + 3) % 2000, cases), nprocs=3, join=True)
 
 
 @pytest.mark.parametrize("world", [4, 5])
