@@ -171,3 +171,46 @@ def test_shared_memory_calls_validate_arguments(kt):
         with pytest.raises(kt.KtError) as e:
             call()
         assert e.value.status == kt.KT_ERR_INVALID
+
+
+def test_host_arithmetic_at_extreme_values_matches_the_oracle(kt, oracle):
+    """Sizes beyond 2^31 and 2^40 elements, caps from 4 bytes to 2^63 - 1, step times from the
+    smallest subnormal to the largest double, batches up to 2^31 - 1: the library's host
+    functions and the oracle must agree on every result and on what they reject."""
+    rnd = random.Random(99)
+    big = [0, 1, 7, 8, 9, 63, 64, 65, 2047, 2048, 2049, 4096, (1 << 31) - 1, 1 << 31, (1 << 31) + 1, (1 << 33) + 5,
+           (1 << 40) + 3, 1 << 45]
+    caps = [4, 63, 64, 256, 4096, 1 << 20, 25 << 20, 1 << 40, 1 << 62, (1 << 63) - 1]
+
+    def outcome(fn):
+        try:
+            return fn()
+        except (kt.KtError, oracle.OracleError):
+            return "rejected"
+
+    for _ in range(1500):
+        T = rnd.randint(1, 8)
+        numel = [rnd.choice(big) if rnd.random() < 0.6 else rnd.randint(0, 100000) for _ in range(T)]
+        if sum(numel) == 0:
+            numel[0] = 3
+        cap = rnd.choice(caps)
+        po, pl = outcome(lambda: oracle.bucket_plan(numel, cap)), outcome(lambda: kt.kt_plan_buckets(numel, cap))
+        assert (po == "rejected") == (pl == "rejected"), (numel, cap)
+        if po == "rejected":
+            continue
+        assert (pl.n_buckets, pl.tensor_offset, pl.bucket_of, pl.bucket_start, pl.bucket_numel, pl.transport_numel) == \
+            (po.n_buckets, po.tensor_offset.tolist(), po.bucket_of.tolist(), po.bucket_start.tolist(),
+             po.bucket_numel.tolist(), po.transport_numel), (numel, cap)
+        if sum(numel) <= 1 << 34:                    # the oracle walks the range unit by unit
+            unit, M, b = rnd.choice([2048, 4096]), rnd.randint(1, 9), rnd.randint(-1, po.n_buckets - 1)
+            assert outcome(lambda: oracle.shard_ranges(numel, cap, unit, b, M)) == \
+                outcome(lambda: kt.kt_shard_ranges(numel, cap, unit, b, M)), (numel, cap, unit, b, M)
+    times = [5e-324, 1e-300, 1e-30, 1e-9, 0.5, 1.0, 1.0000000000000002, 3.0, 1e9, 1e30, 1e300, 1.7976931348623157e308]
+    for _ in range(1500):
+        K = rnd.randint(1, 64)
+        ts = [rnd.choice(times) if rnd.random() < 0.5 else rnd.uniform(0.001, 1000) for _ in range(K)]
+        B = rnd.choice([K, K + 1, 2 * K, 256, 65536, (1 << 31) - 1, rnd.randint(K, 100000)])
+        a = outcome(lambda: oracle.schedule(ts, B).tolist())
+        assert a == outcome(lambda: kt.kt_schedule(ts, B)), (ts, B)
+        assert a == "rejected" or (sum(a) == B and min(a) >= 1)
+        assert outcome(lambda: oracle.scores(ts).tolist()) == outcome(lambda: kt.kt_scores(ts))
