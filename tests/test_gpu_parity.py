@@ -110,6 +110,39 @@ def test_relay_with_group_buffers_as_rows_of_one_allocation(kt, oracle):
     compare_all(kt, oracle, W.tiny(), staged="relay_all", relay_chunk=256, rows=True)
 
 
+def test_relay_merges_the_groups_copies_only_for_rows_of_one_allocation(kt):
+    """Seen from outside through a recording's node count: with the G buffers of every set as
+    rows of one allocation a chunk of all groups is one copy each way; with separately
+    allocated buffers it is G copies each way."""
+    wl = W.mobilenet_v2()                                   # three groups
+    host, dev = H.device_gradients(wl)
+    ctx = kt.kt_groups_init(wl.group_of, H.shares_of(wl, kt), wl.G)
+    kt.kt_bucket_pack(ctx, dev, wl.bucket_cap_bytes)
+    n = kt.kt_plan_query(ctx).transport_numel
+    main, a, b = torch.cuda.Stream(), torch.cuda.Stream(), torch.cuda.Stream()
+    chunk = 1 << 30
+    nodes = {}
+    for layout in ("rows", "separate"):
+        def buffers(pinned):
+            if layout == "rows":
+                whole = torch.zeros(wl.G, n)
+                return list(whole.pin_memory() if pinned else whole.cuda())
+            # separate allocations, with a gap so that they cannot be neighbours
+            return [(torch.zeros(n + 4096).pin_memory() if pinned else torch.zeros(n + 4096, device="cuda"))[:n]
+                    for _ in range(wl.G)]
+        send, pinned, recv = buffers(False), buffers(True), buffers(False)
+        torch.cuda.synchronize()
+        kt.kt_graph_begin(ctx, main)
+        kt.kt_relay_through_host(ctx, send, pinned, recv, a, b, bucket=-1, chunk_bytes=chunk, main_stream=main)
+        kt.kt_stage_wait(ctx, kt.KT_H2D, bucket=-1, main_stream=main)
+        g = kt.kt_graph_end(ctx, main)
+        nodes[layout] = kt.kt_graph_nodes(g)
+        kt.kt_graph_destroy(g)
+    # one chunk covers everything: one copy down and one up when merged, G of each otherwise
+    assert nodes["separate"] - nodes["rows"] == 2 * (wl.G - 1), nodes
+    kt.kt_destroy(ctx)
+
+
 @pytest.mark.parametrize("name", ["resnet18", "resnet50", "mobilenet_v2"])
 def test_host_resident_step_as_benchmarked(kt, oracle, name):
     """The benchmark's end-to-end arm (gradients start in pinned host memory, buckets pipelined
