@@ -119,3 +119,37 @@ def test_static_scratch_entry_rejects_what_does_not_fit(kt):
     assert bool((out == 1.0).all())
     with pytest.raises(kt.KtError):
         kt.kt_sync_flat_static([0, 2], [1, 1], g, out)      # group 1 is empty
+
+
+def drawn_static_calls(kt, oracle, rnd, calls):
+    """`calls` drawn problems (rank counts, group layouts, shares, lengths around the tile and
+    vector sizes, dtypes, element misalignment of sources and of the output, scales) through
+    the entry point back to back on one stream, then each result against the oracle."""
+    sizes = [1, 3, 7, 8, 9, 63, 64, 65, 511, 2047, 2048, 2049, 4095, 4096, 4097, 10000, 100003, 262144]
+    todo = []
+    for i in range(calls):
+        K = rnd.randint(1, 16)
+        G = rnd.randint(1, min(K, 4))
+        group_of = list(range(G)) + [rnd.randrange(G) for _ in range(K - G)]
+        rnd.shuffle(group_of)
+        c = dict(group_of=group_of, shares=[rnd.randint(1, 200) for _ in range(K)], n=rnd.choice(sizes),
+                 dtype=rnd.choice([torch.float32, torch.bfloat16]), out_dtype=rnd.choice([torch.float32, torch.bfloat16]),
+                 scale=rnd.choice([1.0, 0.5, 1.0 / 3.0]), misalign=rnd.choice([0, 0, 1, 3]))
+        if G * ((c["n"] + 63) // 64 * 64) > kt.KT_STATIC_MAX_ELEMS:
+            c["n"] = 4097
+        grads = make_grads(K, c["n"], c["dtype"], 5000 + i + rnd.randrange(1 << 20), c["misalign"])
+        shift = rnd.choice([0, 0, 1, 2])
+        out = torch.full((c["n"] + shift,), float("nan"), dtype=c["out_dtype"], device="cuda")[shift:]
+        todo.append((c, grads, out))
+    torch.cuda.synchronize()
+    for c, grads, out in todo:
+        kt.kt_sync_flat_static(c["group_of"], c["shares"], grads, out, scale=c["scale"])
+    torch.cuda.synchronize()
+    for c, grads, out in todo:
+        H.assert_bit_equal(out, oracle_result(oracle, c, grads), "drawn call %r" % {k: v for k, v in c.items() if k != "shares"})
+
+
+@pytest.mark.parametrize("seed", range(3))
+def test_static_scratch_entry_on_drawn_problems(kt, oracle, seed):
+    import random
+    drawn_static_calls(kt, oracle, random.Random(1200 + seed), 20)
